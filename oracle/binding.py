@@ -1,0 +1,168 @@
+"""ctypes access to ``llmem_oracle.c`` (TEST INFRASTRUCTURE ONLY).
+
+Argument marshalling only; every number comes from the C file.  Inputs are
+numpy arrays of 64-byte configuration records (any structured dtype of
+itemsize 64 with the documented field order).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "llmem_oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+
+SELECT_ALLZERO = 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc if the shared object is missing or stale."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(
+            ["gcc", "-O2", "-std=c11", "-Wall", "-Wextra", "-shared", "-fPIC", "-o", tmp, _SRC,
+             "-lpthread"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.oracle_max_batch.restype = ctypes.c_int32
+        _lib.oracle_max_batch_bisect.restype = ctypes.c_int32
+    return _lib
+
+
+def _cfgs(cfg: np.ndarray) -> np.ndarray:
+    cfg = np.ascontiguousarray(cfg)
+    if cfg.dtype.itemsize != 64:
+        raise ValueError("configuration records must be 64 bytes")
+    return cfg.reshape(-1)
+
+
+def _p(a: np.ndarray | None):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _rec(cfg: np.ndarray, i: int = 0):
+    return ctypes.c_void_p(cfg.ctypes.data + 64 * i)
+
+
+# ---- single-configuration calls ------------------------------------------
+def validate(cfg: np.ndarray) -> int:
+    cfg = _cfgs(cfg)
+    return int(lib().oracle_validate(_rec(cfg)))
+
+
+def inventory(cfg: np.ndarray) -> dict:
+    cfg = _cfgs(cfg)
+    out = np.zeros(10, dtype=np.int64)
+    st = lib().oracle_inventory(_rec(cfg), _p(out))
+    if st:
+        raise ValueError(f"invalid configuration (status {st})")
+    keys = ("e_n", "K", "C", "embed_p", "other_p", "lm_p", "tok_p", "pos_p", "hh_p", "hf_p")
+    return dict(zip(keys, (int(v) for v in out)))
+
+
+def event_count(cfg: np.ndarray, formula: bool = False) -> tuple[int, int]:
+    """(status, number of events)."""
+    cfg = _cfgs(cfg)
+    n = ctypes.c_int64(0)
+    f = lib().oracle_event_count_formula if formula else lib().oracle_event_count
+    st = f(_rec(cfg), ctypes.byref(n))
+    return int(st), int(n.value)
+
+
+def expand_events(cfg: np.ndarray) -> np.ndarray:
+    """Raw signed byte deltas of one configuration."""
+    cfg = _cfgs(cfg)
+    st, n = event_count(cfg)
+    if st:
+        raise ValueError(f"status {st}")
+    out = np.zeros(n, dtype=np.int64)
+    st = lib().oracle_expand_events(_rec(cfg), _p(out), ctypes.c_int64(n))
+    assert st == 0
+    return out
+
+
+def round_events(delta: np.ndarray) -> np.ndarray:
+    out = np.ascontiguousarray(delta, dtype=np.int64).copy()
+    lib().oracle_round_events(_p(out), ctypes.c_int64(out.size))
+    return out
+
+
+def scan_peak(delta: np.ndarray) -> tuple[int, int]:
+    """(max prefix sum, first index attaining it); (0, -1) for an empty list."""
+    d = np.ascontiguousarray(delta, dtype=np.int64)
+    best, arg = ctypes.c_int64(0), ctypes.c_int64(0)
+    lib().oracle_scan_peak(_p(d), ctypes.c_int64(d.size), ctypes.byref(best), ctypes.byref(arg))
+    return int(best.value), int(arg.value)
+
+
+def peak_offset(cfg: np.ndarray) -> tuple[int, int]:
+    cfg = _cfgs(cfg)
+    off = ctypes.c_int64(0)
+    st = lib().oracle_peak_offset(_rec(cfg), ctypes.byref(off))
+    return int(st), int(off.value)
+
+
+# ---- batched calls ---------------------------------------------------------
+def estimate(cfg: np.ndarray, level: int = 1, threads: int = 1):
+    """Returns dict(peak, index, status, count); index and count are level-1 only."""
+    cfg = _cfgs(cfg)
+    n = cfg.size
+    peak = np.full(n, -1, dtype=np.int64)
+    index = np.full(n, -1, dtype=np.int64)
+    status = np.zeros(n, dtype=np.uint8)
+    count = np.zeros(n, dtype=np.int64)
+    lib().oracle_estimate_many(_p(cfg), ctypes.c_int64(n), _p(peak), _p(index), _p(status),
+                               _p(count), ctypes.c_int(level), ctypes.c_int(threads))
+    return {"peak": peak, "index": index, "status": status, "count": count}
+
+
+def max_batch(cfg: np.ndarray, capacities, bmax: int, level: int = 1, threads: int = 1):
+    """Returns (bs[n, n_cap] int32, status[n] uint8)."""
+    cfg = _cfgs(cfg)
+    caps = np.ascontiguousarray(capacities, dtype=np.int64).reshape(-1)
+    n = cfg.size
+    bs = np.full((n, caps.size), -1, dtype=np.int32)
+    status = np.zeros(n, dtype=np.uint8)
+    lib().oracle_max_batch_many(_p(cfg), ctypes.c_int64(n), _p(caps), ctypes.c_int32(caps.size),
+                                ctypes.c_int32(bmax), _p(bs), _p(status), ctypes.c_int(level),
+                                ctypes.c_int(threads))
+    return bs, status
+
+
+def select_method(cfg: np.ndarray, capacities, bmax: int, flags: int = 0, level: int = 1,
+                  threads: int = 1):
+    """Returns dict(method[n, n_cap], batch[n, n_cap], bs_list[n, n_cap, 4], status[n])."""
+    cfg = _cfgs(cfg)
+    caps = np.ascontiguousarray(capacities, dtype=np.int64).reshape(-1)
+    n = cfg.size
+    method = np.full((n, caps.size), -1, dtype=np.int32)
+    batch = np.full((n, caps.size), -1, dtype=np.int32)
+    bs_list = np.full((n, caps.size, 4), -1, dtype=np.int32)
+    status = np.zeros(n, dtype=np.uint8)
+    lib().oracle_select_many(_p(cfg), ctypes.c_int64(n), _p(caps), ctypes.c_int32(caps.size),
+                             ctypes.c_int32(bmax), ctypes.c_uint32(flags), _p(method), _p(batch),
+                             _p(bs_list), _p(status), ctypes.c_int(level), ctypes.c_int(threads))
+    return {"method": method, "batch": batch, "bs_list": bs_list, "status": status}
+
+
+def decide(bs_list, gpu_n: int, tp_n: int, flags: int = 0) -> tuple[int, int]:
+    """Decision step of Algorithm 1 for given per-method largest batches."""
+    bl = np.ascontiguousarray(bs_list, dtype=np.int32)
+    assert bl.size == 4
+    m, b = ctypes.c_int32(0), ctypes.c_int32(0)
+    lib().oracle_decide(_p(bl), ctypes.c_int32(gpu_n), ctypes.c_int32(tp_n),
+                        ctypes.c_uint32(flags), ctypes.byref(m), ctypes.byref(b))
+    return int(m.value), int(b.value)

@@ -1,0 +1,580 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+Nothing here compares the oracle with itself re-typed: the closed forms are
+the paper's equations (Sections 4.2 and 5) evaluated in exact rational
+arithmetic from an independently enumerated tensor list; the allocator
+simulation works from tensor lifetimes, not from the event order; parameter
+counts are public facts; Algorithm 1 cases are worked by hand.
+"""
+from fractions import Fraction
+from math import ceil
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2404_10933_b200 import grids
+
+G = 2 * 1024 * 1024  # cu_p, Section 4.2
+B16, B32 = 2, 4      # Table 1
+
+
+def mk(**kw):
+    c = grids.empty(1)
+    base = dict(layers=4, hidden=2048, heads=16, ffn=8192, vocab=65536, pos_len=0, seq=1024,
+                batch=32, chunk_elems=1 << 24, base_bytes=123456789, method=0, gpu_n=1, tp_n=0,
+                lm_bytes=2, ffn_kind=0, has_bias=0, iters=2)
+    base.update(kw)
+    for k, v in base.items():
+        c[k] = v
+    return c
+
+
+def cfg_fields(c):
+    return {k: int(c[k][0]) for k in c.dtype.names if k != "reserved"}
+
+
+# --------------------------------------------------------------------------
+# an independent parameter inventory: enumerate the tensors of a standard
+# decoder the way a framework's named_parameters() would list them
+# --------------------------------------------------------------------------
+def enumerate_tensors(f):
+    """List of (kind, n_elements); kind in {'E', 'L', 'bias', 'norm'}."""
+    H, F, V, P = f["hidden"], f["ffn"], f["vocab"], f["pos_len"]
+    bias = f["has_bias"]
+    t = [("E", V * H)]
+    if P > 0:
+        t.append(("E", P * H))
+    for _ in range(f["layers"]):
+        t.append(("norm", H))
+        if bias:
+            t.append(("norm", H))
+        for _proj in ("q", "k", "v", "o"):
+            t.append(("L", H * H))
+            if bias:
+                t.append(("bias", H))
+        t.append(("norm", H))
+        if bias:
+            t.append(("norm", H))
+        ups = ("gate", "up") if f["ffn_kind"] else ("fc1",)
+        for _u in ups:
+            t.append(("L", H * F))
+            if bias:
+                t.append(("bias", F))
+        t.append(("L", F * H))
+        if bias:
+            t.append(("bias", H))
+    t.append(("norm", H))
+    if bias:
+        t.append(("norm", H))
+    return t
+
+
+def rnd(x):
+    """ceil(x / cu_p) * cu_p for a rational x."""
+    return ceil(Fraction(x) / G) * G
+
+
+def paper_closed_forms(f):
+    """m_peak^s, m_peak^dp, m_peak^tp, m_peak^dp+tp of Sections 4.2 and 5, exact rationals."""
+    tensors = enumerate_tensors(f)
+    embed_p = sum(n for k, n in tensors if k == "E")
+    other_p = sum(n for k, n in tensors if k != "E")
+    cs, bs, sl = f["chunk_elems"], f["batch"], f["seq"]
+    o_n, l_n, dict_n = f["hidden"], f["layers"], f["vocab"]
+    e_n = sum(1 for k, _ in tensors if k == "E")
+    n, t = f["gpu_n"], f["tp_n"]
+    B = f["lm_bytes"]
+    lm_p = dict_n * o_n * B
+    chunked = embed_p + ceil(Fraction(other_p, cs)) * cs
+    m_p = rnd(chunked * (B16 + B32))
+    m_p16 = rnd(chunked * B16)
+    m_p32 = rnd(chunked * B32)
+    m_os = sum(rnd(p * (B32 + B32)) for k, p in tensors if k in ("E", "L"))
+    m_out = rnd((e_n + l_n) * (bs * sl * o_n) * B16)
+    m_lm = rnd(bs * sl * dict_n * B) + 2 * rnd(bs * (sl - 1) * dict_n * B) + lm_p
+    base = f["base_bytes"]
+
+    def m_back(tp):
+        return rnd(Fraction(l_n * (bs * sl * o_n) * (tp - 1), tp) * B16)
+
+    m_s = base + m_p + m_os + m_out + m_lm
+    m_dp = base + m_p16 + Fraction(m_p32 + m_os, n) + m_out + m_lm
+    m_tp = base + Fraction(m_p + m_os, n) + m_out + m_lm + m_back(n)
+    m_dptp = (m_dp - Fraction(m_p16 * t, n) + m_back(t)) if t else None
+    return {"s": m_s, "dp": m_dp, "tp": m_tp, "dptp": m_dptp, "m_p": m_p, "m_os": m_os,
+            "m_out": m_out, "m_lm": m_lm, "embed_p": embed_p, "other_p": other_p,
+            "lm_p": lm_p, "e_n": e_n, "C": ceil(Fraction(other_p, cs))}
+
+
+def oracle_peak(c, level=1):
+    r = oracle.estimate(c, level=level)
+    assert r["status"][0] == 0, r["status"][0]
+    return int(r["peak"][0])
+
+
+# --------------------------------------------------------------------------
+# P6: rounding, from the definition ceil(x/cu_p)*cu_p
+# --------------------------------------------------------------------------
+def test_round_hand_cases():
+    d = np.array([0, 1, G - 1, G, G + 1, 3 * G, -1, -G, -(G + 1), 5 * G - 7], dtype=np.int64)
+    want = [0, G, G, G, 2 * G, 3 * G, -G, -G, -2 * G, 5 * G]
+    assert oracle.round_events(d).tolist() == want
+
+
+def test_scan_hand_cases():
+    assert oracle.scan_peak(np.array([], dtype=np.int64)) == (0, -1)
+    assert oracle.scan_peak(np.array([5, -5, 5], dtype=np.int64)) == (5, 0)       # first of equals
+    assert oracle.scan_peak(np.array([1, 2, -4, 6, -1], dtype=np.int64)) == (5, 3)
+    assert oracle.scan_peak(np.array([-3, -2], dtype=np.int64)) == (-3, 0)        # all negative
+    assert oracle.scan_peak(np.array([4, 0, 0], dtype=np.int64)) == (4, 0)        # zero events
+
+
+# --------------------------------------------------------------------------
+# parameter inventory against public parameter counts
+# --------------------------------------------------------------------------
+def test_inventory_public_param_counts(golden_dir):
+    rows = [l.split() for l in open(f"{golden_dir}/public_param_counts.txt")
+            if l.strip() and not l.startswith("#")]
+    assert len(rows) == 2
+    for name, L, H, A, F, V, P, kind, bias, tied, total in rows:
+        c = mk(layers=int(L), hidden=int(H), heads=int(A), ffn=int(F), vocab=int(V),
+               pos_len=int(P), ffn_kind=int(kind), has_bias=int(bias), lm_bytes=2)
+        inv = oracle.inventory(c)
+        lm_elems = inv["lm_p"] // 2
+        assert lm_elems == int(V) * int(H)
+        got = inv["embed_p"] + inv["other_p"] + (0 if int(tied) else lm_elems)
+        assert got == int(total), name
+
+
+def test_inventory_matches_tensor_enumeration():
+    for kw in (dict(), dict(has_bias=1), dict(ffn_kind=1, ffn=5632), dict(pos_len=2048, has_bias=1),
+               dict(layers=1, hidden=64, heads=1, ffn=192, vocab=1000, ffn_kind=1, has_bias=1)):
+        c = mk(**kw)
+        f = cfg_fields(c)
+        t = enumerate_tensors(f)
+        inv = oracle.inventory(c)
+        assert inv["embed_p"] == sum(n for k, n in t if k == "E")
+        assert inv["other_p"] == sum(n for k, n in t if k != "E")
+        assert inv["e_n"] == sum(1 for k, _ in t if k == "E")
+        assert inv["K"] * f["layers"] == sum(1 for k, _ in t if k == "L")
+        assert inv["C"] == ceil(Fraction(inv["other_p"], f["chunk_elems"]))
+
+
+# --------------------------------------------------------------------------
+# P1: page-aligned family: per-event rounding == per-term rounding, so the event
+# model must reproduce the paper's four peak equations exactly
+# --------------------------------------------------------------------------
+ALIGNED = [
+    dict(method=0, gpu_n=1), dict(method=0, gpu_n=4),
+    dict(method=1, gpu_n=2), dict(method=1, gpu_n=4), dict(method=1, gpu_n=16),
+    dict(method=2, gpu_n=4), dict(method=2, gpu_n=8),
+    dict(method=3, gpu_n=4, tp_n=2), dict(method=3, gpu_n=8, tp_n=2),
+    dict(method=3, gpu_n=8, tp_n=4), dict(method=3, gpu_n=16, tp_n=4),
+]
+ALIGNED_SHAPES = [
+    dict(),
+    dict(pos_len=8192, lm_bytes=4),
+    dict(ffn_kind=1, ffn=8192, layers=3, batch=16, seq=2048),
+]
+
+
+@pytest.mark.parametrize("shape", ALIGNED_SHAPES)
+@pytest.mark.parametrize("meth", ALIGNED)
+def test_aligned_family_equals_paper_equations(shape, meth):
+    c = mk(**shape, **meth)
+    f = cfg_fields(c)
+    forms = paper_closed_forms(f)
+    key = ("s", "dp", "tp", "dptp")[f["method"]]
+    want = forms[key]
+    assert want.denominator == 1, "family is not aligned"
+    # every event of the family is already a multiple of the page
+    raw = oracle.expand_events(c)
+    assert (raw % G == 0).all()
+    assert oracle_peak(c) == int(want)
+    assert oracle_peak(c, level=2) == int(want)
+    # iterations beyond the second change nothing; one iteration peaks lower
+    c3 = c.copy(); c3["iters"] = 3
+    c1 = c.copy(); c1["iters"] = 1
+    assert oracle_peak(c3) == int(want)
+    assert oracle_peak(c1) < int(want)
+
+
+def test_aligned_single_iteration_value():
+    # one iteration: max(before optimizer states: init + outputs; after: init + m_os)
+    c = mk(method=2, gpu_n=4, iters=1)
+    f = cfg_fields(c)
+    forms = paper_closed_forms(f)
+    n = 4
+    no_os = forms["tp"] - Fraction(forms["m_os"], n)
+    back = rnd(Fraction(f["layers"] * f["batch"] * f["seq"] * f["hidden"] * 3, 4) * B16)
+    only_os = forms["tp"] - forms["m_out"] - (forms["m_lm"] - forms["lm_p"]) - back
+    assert oracle_peak(c) == int(max(no_os, only_os))
+
+
+# --------------------------------------------------------------------------
+# P3: static model-state bytes = what is still allocated after the last free
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("meth", ALIGNED)
+def test_static_bytes_closed_form(meth):
+    c = mk(**meth)
+    f = cfg_fields(c)
+    forms = paper_closed_forms(f)
+    final = int(oracle.round_events(oracle.expand_events(c)).sum())
+    n = f["gpu_n"]
+    want = forms["m_p"] + forms["m_os"] if f["method"] == 0 else Fraction(forms["m_p"] + forms["m_os"], n)
+    assert final == want
+
+
+# --------------------------------------------------------------------------
+# P2: unaligned shapes: the event model differs from the paper's per-term
+# rounding by a bounded number of pages
+# --------------------------------------------------------------------------
+def test_cdp_two_sided_bound():
+    cfgs = grids.g2_shapes(0, 48)
+    for i in range(len(cfgs)):
+        for b in (1, 7, 32):
+            c = cfgs[i:i + 1].copy()
+            c["batch"] = b
+            f = cfg_fields(c)
+            forms = paper_closed_forms(f)
+            diff = oracle_peak(c) - forms["s"]
+            pages = (2 * forms["C"] + 2 - 1) + (forms["e_n"] + f["layers"] - 1)
+            assert 0 <= diff <= pages * G, (i, b, diff)
+
+
+def test_g1_shape_bound_example():
+    c = grids.g1_small()[6:7]          # batch 7
+    f = cfg_fields(c)
+    forms = paper_closed_forms(f)
+    diff = oracle_peak(c) - forms["s"]
+    assert 0 <= diff <= ((2 * 82 + 1) + (2 + 12 - 1)) * G
+    assert diff % G == 0
+
+
+def test_all_methods_bounded_distance_from_paper():
+    cfgs = grids.g3_sweep(0, 200)
+    for i in range(len(cfgs)):
+        c = cfgs[i:i + 1]
+        f = cfg_fields(c)
+        forms = paper_closed_forms(f)
+        want = forms[("s", "dp", "tp", "dptp")[f["method"]]]
+        C, L, e_n = forms["C"], f["layers"], forms["e_n"]
+        n_alloc = (2 + 2 * C) + (1 + C) + (e_n + L + 3) + L + (e_n + 6 * L + L)
+        assert abs(oracle_peak(c) - want) <= n_alloc * (G + 1), i
+
+
+# --------------------------------------------------------------------------
+# P5: allocator simulation from tensor lifetimes (not from the event order)
+# --------------------------------------------------------------------------
+def lifetime_table(f):
+    """(bytes, first_step, last_step) per allocation.  Steps: 0 = initialisation,
+    2k-1 = compute of iteration k, 2k = between iterations (optimizer step of k)."""
+    inf = 10 ** 9
+    n, t, m = f["gpu_n"], f["tp_n"], f["method"]
+    H, V, L, P = f["hidden"], f["vocab"], f["layers"], f["pos_len"]
+    tensors = enumerate_tensors(f)
+    embed_p = sum(x for k, x in tensors if k == "E")
+    other_p = sum(x for k, x in tensors if k != "E")
+    cs = f["chunk_elems"]
+    C = -(-other_p // cs)
+    units = [embed_p] + [cs] * C
+
+    def part(x):
+        return x if m == 0 else -(-x // n)
+
+    rows = []
+    for x in units:
+        rows.append((part(2 * x), 0, inf))
+        rows.append((part(4 * x), 0, inf))
+    for k, x in tensors:
+        if k in ("E", "L"):
+            rows.append((part(8 * x), 2, inf))       # appears with the first optimizer step
+    out = 2 * f["batch"] * f["seq"] * H
+    e_n = sum(1 for k, _ in tensors if k == "E")
+    for it in range(1, f["iters"] + 1):
+        s = 2 * it - 1
+        for x in units:
+            if m == 1:
+                rows.append((2 * x - part(2 * x), s, s))
+            elif m == 3:
+                rows.append((2 * x - (2 * x * t) // n - part(2 * x), s, s))
+        for _ in range(e_n + L):
+            rows.append((out, s, s))
+        rows.append((f["lm_bytes"] * f["batch"] * f["seq"] * V, s, s))
+        for _ in range(2):
+            rows.append((f["lm_bytes"] * f["batch"] * (f["seq"] - 1) * V, s, s))
+        if m in (2, 3):
+            tp = n if m == 2 else t
+            for _ in range(L):
+                rows.append((-(-(out * (tp - 1)) // tp), s, s))
+    return rows
+
+
+def sweep_peak(rows, steps):
+    best = 0
+    for s in range(steps):
+        live = sum(-(-b // G) * G for b, a, z in rows if a <= s <= z)
+        best = max(best, live)
+    return best
+
+
+TINY = [
+    dict(layers=1, hidden=64, heads=1, ffn=256, vocab=1000, chunk_elems=20000, batch=3, seq=17),
+    dict(layers=3, hidden=128, heads=2, ffn=384, vocab=3001, pos_len=77, chunk_elems=150000,
+         batch=2, seq=33, ffn_kind=1, has_bias=1, lm_bytes=4),
+    dict(layers=2, hidden=192, heads=3, ffn=768, vocab=5000, chunk_elems=1 << 18, batch=5, seq=1,
+         has_bias=1),
+]
+TINY_METHODS = [dict(method=0, gpu_n=1), dict(method=0, gpu_n=3), dict(method=1, gpu_n=1),
+                dict(method=1, gpu_n=3), dict(method=2, gpu_n=1), dict(method=2, gpu_n=5),
+                dict(method=3, gpu_n=4, tp_n=2), dict(method=3, gpu_n=12, tp_n=3)]
+
+
+@pytest.mark.parametrize("iters", [1, 2, 3])
+@pytest.mark.parametrize("meth", TINY_METHODS)
+@pytest.mark.parametrize("shape", TINY)
+def test_lifetime_sweep_matches_event_scan(shape, meth, iters):
+    c = mk(**shape, **meth, iters=iters, base_bytes=999)
+    f = cfg_fields(c)
+    rows = lifetime_table(f)
+    want = sweep_peak(rows, 2 * iters + 1) + 999 + f["vocab"] * f["hidden"] * f["lm_bytes"]
+    assert oracle_peak(c) == want
+    assert oracle_peak(c, level=2) == want
+    # the event list allocates and frees exactly this multiset of sizes
+    ev = oracle.expand_events(c)
+    allocs = sorted(int(x) for x in ev if x > 0)
+    assert int((ev == 0).sum()) % 2 == 0
+    frees = sorted(int(-x) for x in ev if x < 0)
+    assert allocs == sorted(b for b, a, z in rows if b > 0)
+    assert frees == sorted(b for b, a, z in rows if z < 10 ** 9 and b > 0)
+
+
+def test_explicit_allocator_replay():
+    """Replay the oracle's event list on an id -> size map: every free releases the
+    most recent live allocation (stack discipline), nothing temporary survives.
+    Zero-byte events (a gather on one device, a shifted logit of a length-1 sequence)
+    hold no memory and are skipped."""
+    for shape in TINY:
+        for meth in TINY_METHODS:
+            c = mk(**shape, **meth, iters=3)
+            ev = oracle.round_events(oracle.expand_events(c)).tolist()
+            live, order, peak, total = {}, [], 0, 0
+            for i, d in enumerate(ev):
+                if d > 0:
+                    live[i] = d
+                    order.append(i)
+                elif d < 0:
+                    j = order.pop()
+                    assert live.pop(j) == -d, (i, j)
+                total += d
+                assert total >= 0
+                peak = max(peak, total)
+            assert sum(live.values()) == sum(ev)
+            # what survives is exactly the initialisation and the optimizer states
+            inv = oracle.inventory(c)
+            n_persistent = 2 + 2 * inv["C"] + inv["e_n"] + inv["K"] * int(c["layers"][0])
+            assert len(live) == n_persistent
+            st, off = oracle.peak_offset(c)
+            assert oracle_peak(c) == peak + off
+
+
+# --------------------------------------------------------------------------
+# P4: invariants
+# --------------------------------------------------------------------------
+def test_invariants_on_seeded_configs():
+    cfgs = grids.g3_sweep(1000, 160)
+    # smaller chunk counts keep level 1 quick
+    cfgs["chunk_elems"] = 1 << 25
+    r = oracle.estimate(cfgs, threads=4)
+    assert (r["status"] == 0).all()
+    for i in range(len(cfgs)):
+        c = cfgs[i:i + 1]
+        f = cfg_fields(c)
+        peak = int(r["peak"][i])
+        st, off = oracle.peak_offset(c)
+        ev = oracle.round_events(oracle.expand_events(c))
+        prefix = np.cumsum(ev)
+        assert (prefix >= 0).all()                               # (vi)
+        assert (peak - off) % G == 0                             # (vii)
+        assert peak >= off + int(ev.sum())                       # (i) static states
+        assert int(prefix.max()) + off == peak
+        assert int(np.argmax(prefix)) == int(r["index"][i])      # first maximum
+        st2, n_formula = oracle.event_count(c, formula=True)
+        assert n_formula == len(ev) == int(r["count"][i])
+        # (ii) monotone in batch and sequence length
+        for key in ("batch", "seq"):
+            c2 = c.copy(); c2[key] = f[key] + 1
+            assert oracle_peak(c2) >= peak
+            c2[key] = f[key] * 2
+            assert oracle_peak(c2) >= peak
+        # (viii) heads do not matter
+        c2 = c.copy(); c2["heads"] = 1
+        assert oracle_peak(c2) == peak
+        # (v) iterations
+        c2 = c.copy(); c2["iters"] = 5
+        assert oracle_peak(c2) == peak
+        c2["iters"] = 1
+        assert oracle_peak(c2) <= peak
+        # level 2 agrees
+        assert oracle_peak(c, level=2) == peak
+
+
+def test_degree_one_methods_coincide_and_sharding_never_costs_more():
+    cfgs = grids.g2_shapes(100, 40)
+    cfgs["batch"] = 3
+    for i in range(len(cfgs)):
+        c = cfgs[i:i + 1].copy()
+        c["method"], c["gpu_n"] = 0, 1
+        cdp = oracle_peak(c)
+        cdp_events = oracle.expand_events(c)
+        for m in (1, 2):
+            c["method"], c["gpu_n"] = m, 1
+            assert oracle_peak(c) == cdp                         # (iv)
+        inv = oracle.inventory(c)
+        n_init = 2 + 2 * inv["C"]
+        for m, n, t in ((1, 4, 0), (2, 4, 0), (3, 4, 2), (1, 7, 0), (2, 8, 0), (3, 8, 4)):
+            c["method"], c["gpu_n"], c["tp_n"] = m, n, t
+            ev = oracle.expand_events(c)
+            # (iii) persistent events: initialisation and optimizer states
+            assert (ev[:n_init] <= cdp_events[:n_init]).all()
+            static = int(oracle.round_events(ev).sum())
+            static_cdp = int(oracle.round_events(cdp_events).sum())
+            assert static <= static_cdp
+
+
+# --------------------------------------------------------------------------
+# status codes and guards
+# --------------------------------------------------------------------------
+def test_status_codes():
+    assert oracle.validate(mk()) == 0
+    for bad in (dict(layers=0), dict(hidden=0), dict(heads=3), dict(heads=0), dict(ffn=0),
+                dict(vocab=0), dict(pos_len=-1), dict(seq=0), dict(batch=0), dict(chunk_elems=0),
+                dict(base_bytes=-1), dict(method=4), dict(gpu_n=0), dict(lm_bytes=3),
+                dict(ffn_kind=2), dict(has_bias=2), dict(iters=0), dict(hidden=(1 << 20) + 1, heads=1),
+                dict(layers=(1 << 16) + 1), dict(chunk_elems=(1 << 40) + 1)):
+        assert oracle.validate(mk(**bad)) == 1, bad
+    c = mk(); c["reserved"][0, 3] = 1
+    assert oracle.validate(c) == 1
+    for n, t in ((4, 0), (4, 1), (4, 4), (4, 3), (6, 4), (1, 1), (2, 2), (7, 2)):
+        assert oracle.validate(mk(method=3, gpu_n=n, tp_n=t)) == 2, (n, t)
+    for n, t in ((4, 2), (6, 2), (6, 3), (8, 2), (8, 4), (16, 8), (255, 5)):
+        assert oracle.validate(mk(method=3, gpu_n=n, tp_n=t)) == 0, (n, t)
+    # tp_n is ignored by the other methods
+    assert oracle.validate(mk(method=2, gpu_n=4, tp_n=77)) == 0
+
+
+def test_overflow_guard():
+    # 2^31 events: tiny chunks of a big model
+    c = mk(layers=1 << 16, hidden=1 << 20, heads=1, ffn=1 << 22, chunk_elems=1)
+    assert oracle.event_count(c)[0] == 3
+    r = oracle.estimate(c)
+    assert r["status"][0] == 3 and r["peak"][0] == -1 and r["index"][0] == -1
+    # peak >= 2^62 bytes with few events
+    c = mk(batch=1 << 26, seq=1 << 26, vocab=1 << 26)
+    assert oracle.event_count(c)[0] == 3
+    # just large, still fine
+    c = mk(batch=1 << 10, seq=1 << 16, vocab=1 << 17)
+    assert oracle.event_count(c)[0] == 0
+
+
+# --------------------------------------------------------------------------
+# P7: largest batch
+# --------------------------------------------------------------------------
+def test_max_batch_definition_and_bisect():
+    cfgs = grids.g4_search_grid(0, 6)                 # 6 shapes x 64 (method, degree)
+    cfgs["chunk_elems"] = 1 << 25
+    caps = grids.g4_capacities()
+    bmax = 48
+    lin, st1 = oracle.max_batch(cfgs, caps, bmax, level=1, threads=8)
+    bis, st2 = oracle.max_batch(cfgs, caps, bmax, level=2, threads=8)
+    assert (lin == bis).all() and (st1 == st2).all()
+    assert set(np.unique(st1)) <= {0, 2}
+    assert (lin[st1 == 2] == -1).all()
+    seen_zero = seen_mid = seen_cap = False
+    for i in np.flatnonzero(st1 == 0)[::5]:
+        for m, cap in enumerate(caps):
+            b = int(lin[i, m])
+            c = cfgs[i:i + 1].copy()
+            if b >= 1:
+                c["batch"] = b
+                assert oracle_peak(c) <= cap
+            if b < bmax:
+                c["batch"] = b + 1
+                assert oracle_peak(c) > cap
+            seen_zero |= b == 0
+            seen_mid |= 0 < b < bmax
+            seen_cap |= b == bmax
+    assert seen_zero and seen_mid and seen_cap
+
+
+def test_max_batch_full_range_bisect_sampled():
+    cfgs = grids.g4_search_grid(7, 2)
+    caps = grids.g4_capacities()
+    bis, st = oracle.max_batch(cfgs, caps, grids.G4_BMAX, level=2)
+    for i in np.flatnonzero(st == 0)[::9]:
+        for m in (0, 4, 8):
+            b = int(bis[i, m])
+            c = cfgs[i:i + 1].copy()
+            if b >= 1:
+                c["batch"] = b
+                assert oracle_peak(c, level=2) <= caps[m]
+            if b < grids.G4_BMAX:
+                c["batch"] = b + 1
+                assert oracle_peak(c, level=2) > caps[m]
+
+
+# --------------------------------------------------------------------------
+# P8: the decision of Algorithm 1
+# --------------------------------------------------------------------------
+def test_algorithm1_hand_cases(golden_dir):
+    n_cases = 0
+    for line in open(f"{golden_dir}/algorithm1_decisions.txt"):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        lhs, rhs = line.split("->")
+        b0, b1, b2, b3, n, t, flags = (int(x) for x in lhs.split())
+        want = tuple(int(x) for x in rhs.split())
+        assert oracle.decide([b0, b1, b2, b3], n, t, flags) == want, line
+        n_cases += 1
+    assert n_cases >= 15
+
+
+def test_select_is_max_batch_plus_decision():
+    cfgs = grids.g4_select_grid(3, 5)
+    cfgs["chunk_elems"] = 1 << 25
+    caps = grids.g4_capacities()[[0, 3, 7]]
+    bmax = 24
+    for flags in (0, oracle.SELECT_ALLZERO):
+        sel = oracle.select_method(cfgs, caps, bmax, flags=flags, level=1, threads=8)
+        sel2 = oracle.select_method(cfgs, caps, bmax, flags=flags, level=2, threads=8)
+        for k in ("method", "batch", "bs_list"):
+            assert (sel[k] == sel2[k]).all()
+        for i in range(len(cfgs)):
+            n, t = int(cfgs["gpu_n"][i]), int(cfgs["tp_n"][i])
+            for m in range(len(caps)):
+                bl = sel["bs_list"][i, m]
+                for meth in range(4):
+                    c = cfgs[i:i + 1].copy()
+                    c["method"] = meth
+                    b, st = oracle.max_batch(c, caps[m:m + 1], bmax)
+                    assert bl[meth] == max(int(b[0, 0]), 0)
+                assert (int(sel["method"][i, m]), int(sel["batch"][i, m])) == \
+                    oracle.decide(bl, n, t, flags)
+    methods = set(np.unique(sel["method"]).tolist())
+    assert len(methods) >= 3
+
+
+def test_llama7b_on_four_16gib_devices_offloads(golden_dir):
+    # Table 3, last row: llama-7b on 4 x 16384 MB -> CPU offloading.  With 6 + 8 bytes of
+    # parameter and optimizer state per parameter, a quarter of a 6.6e9-parameter model
+    # already exceeds 16 GiB, whatever m_base, the chunk size or the batch.
+    for cs in (1 << 22, 1 << 26):
+        for base in (0, 700 << 20):
+            c = mk(layers=32, hidden=4096, heads=32, ffn=11008, vocab=32000, ffn_kind=1,
+                   has_bias=0, gpu_n=4, tp_n=2, seq=512, chunk_elems=cs, base_bytes=base)
+            for flags in (0, 1):
+                sel = oracle.select_method(c, [16384 << 20], 8, flags=flags, level=2)
+                assert (int(sel["method"][0, 0]), int(sel["batch"][0, 0])) == (4, 0)
+                assert sel["bs_list"][0, 0].tolist() == [0, 0, 0, 0]
