@@ -1,0 +1,407 @@
+#!/usr/bin/env python
+"""Benchmark of the batched LLMem estimator on B200.
+
+One "step" is one pass of the whole hot path over the stress grid (65,536 deep/wide
+decoders, about 5.8e9 allocate/free events, materialised as int64):
+
+    event counts + offsets  ->  expansion with fused page rounding  ->  segmented
+    prefix-sum + max  ->  largest batch per capacity  ->  Algorithm 1 selection
+
+`value` is alloc-events per second over all ranks with the configurations already
+resident in HBM; `e2e` is the same pass through the public API starting from pinned
+host buffers, with the host<->device copies inside the timed region.  The roofline
+block reports the dominant kernel against the measured HBM copy bandwidth.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Under torchrun every rank runs the same work on its own seeded grid (no exchange
+step exists in this method); times are the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2404_10933_b200 import grids  # noqa: E402
+
+METRIC = "alloc-events/sec (configs/sec in configs_per_sec, % of HBM roofline in roofline)"
+UNIT = "events/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            d = json.load(open(path))
+            return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_id: str):
+        self.device_index = device_id
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.device_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [x.strip() for x in line.split(",")]))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        rows = [r for t, r in self.rows if t0 - 0.05 <= t <= t1 + 0.15 and len(r) >= 9] or \
+               [r for _, r in self.rows if len(r) >= 9]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm = [float(r[1]) for r in rows]
+        reasons = set()
+        for r in rows:
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                               r[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": float(rows[0][2]), "reasons": sorted(reasons),
+                "samples": len(rows), "power_w_max": max(float(r[3]) for r in rows)}
+
+
+# ---------------------------------------------------------------------------
+# CPU oracle legs (the only places that may execute oracle/)
+# ---------------------------------------------------------------------------
+def oracle_sample(sample_configs: int):
+    cfgs = grids.g5_stress(0, sample_configs)
+    return cfgs
+
+
+def time_oracle(cfgs, threads: int):
+    import oracle
+    oracle.lib()
+    t0 = time.perf_counter()
+    r = oracle.estimate(cfgs, level=1, threads=threads)
+    dt = time.perf_counter() - t0
+    return int(r["count"].sum()), dt
+
+
+def cpu_baseline(sample_configs: int = 16384):
+    cores = os.cpu_count() or 1
+    events, dt = time_oracle(oracle_sample(sample_configs), cores)
+    return {"value": events / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "configs_per_sec": sample_configs / dt,
+            "sample": f"first {sample_configs} of the 65536 stress-grid configurations "
+                      f"({events} events), level-1 oracle (explicit list, round, scan), "
+                      f"{cores} threads, {dt:.2f} s"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    cores = os.cpu_count() or 1
+    sample = 4096
+    cfgs = oracle_sample(sample)
+    for _ in range(max(args.warmup, 0)):
+        time_oracle(cfgs[:256], cores)
+    t_total, ev_total = 0.0, 0
+    for _ in range(args.steps):
+        ev, dt = time_oracle(cfgs, cores)
+        t_total += dt
+        ev_total += ev
+    value = ev_total / t_total
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
+        "data": "synthetic", "configs_per_sec": sample * args.steps / t_total,
+        "config": {"workload": "G5 stress grid (materialised int64 event lists), bounded sample",
+                   "sample_configs": sample, "events_per_step": ev_total // args.steps},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"each step: first {sample} stress-grid configurations, level-1 oracle, "
+                                   f"{cores} threads"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ---------------------------------------------------------------------------
+# the CUDA arm
+# ---------------------------------------------------------------------------
+class HotPath:
+    """Holds device buffers for one grid and runs one step of the hot path."""
+
+    KERNELS_PER_STEP = 8  # counts(3) + expand(1) + scan(2) + max_batch(1) + select(1)
+
+    def __init__(self, llmem, torch, cfgs: np.ndarray, caps: np.ndarray, bmax: int):
+        self.llmem, self.torch = llmem, torch
+        self.n = len(cfgs)
+        self.bmax = bmax
+        self.host_cfg = torch.from_numpy(cfgs.view(np.uint8).reshape(-1, 64)).pin_memory()
+        self.host_caps = torch.from_numpy(caps).pin_memory()
+        self.cfg = self.host_cfg.cuda()
+        self.caps = self.host_caps.cuda()
+        offsets, _ = llmem.event_counts(self.cfg)
+        self.total = int(offsets[-1].item())
+        self.delta = torch.empty(self.total, dtype=torch.int64, device="cuda")
+        self.scan_scratch = torch.empty(llmem.scratch_bytes(llmem.OP_SCAN_PEAK, self.n, self.total),
+                                        dtype=torch.uint8, device="cuda")
+        self.ev = {k: [] for k in ("expand", "scan")}
+        self.host_out = {
+            "peak": torch.empty(self.n, dtype=torch.int64).pin_memory(),
+            "method": torch.empty((self.n, len(caps)), dtype=torch.int32).pin_memory(),
+            "batch": torch.empty((self.n, len(caps)), dtype=torch.int32).pin_memory(),
+        }
+
+    def step(self, cfg=None, caps=None, total=None, record=True):
+        llmem, torch = self.llmem, self.torch
+        cfg = self.cfg if cfg is None else cfg
+        caps = self.caps if caps is None else caps
+        offsets, status = llmem.event_counts(cfg)
+        if total is None:
+            total = self.total
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)] if record else None
+        if record:
+            e[0].record()
+        delta = llmem.expand_events(cfg, offsets, total, fuse_round=True, out=self.delta)
+        if record:
+            e[1].record()
+        r = llmem.scan_peak(delta, offsets, cfg, scratch=self.scan_scratch)
+        if record:
+            e[2].record()
+            self.ev["expand"].append((e[0], e[1]))
+            self.ev["scan"].append((e[1], e[2]))
+        bs, _ = llmem.max_batch(cfg, caps, self.bmax, want_status=False)
+        sel = llmem.select_method(cfg, caps, self.bmax, want_bs_list=False, want_status=False)
+        return {"peak": r["peak"], "index": r["index"], "bs": bs, "method": sel["method"],
+                "batch": sel["batch"], "offsets": offsets}
+
+    def step_e2e(self):
+        """Host buffers in, host results out: H2D of the configurations and capacities, the
+        device-to-host read of the event total that sizes the list, every kernel, and the
+        D2H of peaks and selections."""
+        torch = self.torch
+        cfg = self.host_cfg.to("cuda", non_blocking=True)
+        caps = self.host_caps.to("cuda", non_blocking=True)
+        offsets, _ = self.llmem.event_counts(cfg)
+        total = int(offsets[-1].item())                      # 8-byte D2H + sync
+        if total > self.delta.numel():
+            self.delta = torch.empty(total, dtype=torch.int64, device="cuda")
+        delta = self.llmem.expand_events(cfg, offsets, total, fuse_round=True, out=self.delta)
+        r = self.llmem.scan_peak(delta, offsets, cfg, scratch=self.scan_scratch)
+        self.llmem.max_batch(cfg, caps, self.bmax, want_status=False)
+        sel = self.llmem.select_method(cfg, caps, self.bmax, want_bs_list=False, want_status=False)
+        self.host_out["peak"].copy_(r["peak"], non_blocking=True)
+        self.host_out["method"].copy_(sel["method"], non_blocking=True)
+        self.host_out["batch"].copy_(sel["batch"], non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        return total
+
+    @property
+    def h2d_bytes(self):
+        return self.host_cfg.numel() + self.host_caps.numel() * 8
+
+    @property
+    def d2h_bytes(self):
+        return 8 + sum(t.numel() * t.element_size() for t in self.host_out.values())
+
+
+def run_ours(args):
+    import torch
+    if not torch.cuda.is_available():
+        print(json.dumps({"error": "no CUDA device: the estimator has no CPU fallback"}))
+        return 2
+    import paper_2404_10933_b200 as llmem
+    llmem.lib()  # fail loudly if the CUDA library is missing
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def sum_over_ranks(x: float) -> float:
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        return float(t.item())
+
+    n_cfg = args.configs
+    cfgs = grids.g5_stress(0, n_cfg, seed_offset=rank)     # weak scaling: one full grid per rank
+    caps = grids.g4_capacities()
+    hp = HotPath(llmem, torch, cfgs, caps, grids.G4_BMAX)
+
+    # ---- device-resident timing ----
+    for _ in range(args.warmup):
+        hp.step(record=False)
+    hp.ev = {k: [] for k in hp.ev}
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(torch.cuda.current_device()).uuid)
+    except Exception:
+        gpu_id = str(torch.cuda.current_device())
+    sampler = ClockSampler(gpu_id)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    wall0 = time.time()
+    start.record()
+    for _ in range(args.steps):
+        out = hp.step()
+    stop.record()
+    barrier()
+    wall1 = time.time()
+    ms = max_over_ranks(start.elapsed_time(stop))
+    clocks = sampler.stop(wall0, wall1) if rank == 0 else None
+    total_events_all = sum_over_ranks(float(hp.total))
+    configs_all = sum_over_ranks(float(hp.n))
+    value = total_events_all * args.steps / (ms * 1e-3)
+
+    kernel_ms = {k: statistics.mean(a.elapsed_time(b) for a, b in v) for k, v in hp.ev.items()}
+    status = llmem.lib().llmem_scratch_status(int(hp.scan_scratch.data_ptr()), None)
+    if status != 0:
+        print(json.dumps({"error": f"device status {status}"}))
+        return 3
+    # the two paths must agree on the device (cheap self-check outside the timed region)
+    fused = llmem.estimate_batch(hp.cfg, want_status=False)
+    agree = bool(torch.equal(fused["peak"], out["peak"]) and torch.equal(fused["index"], out["index"]))
+
+    # ---- end to end from host buffers ----
+    for _ in range(min(args.warmup, 3)):
+        hp.step_e2e()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    e2e_steps = max(1, min(args.steps, 10))
+    for _ in range(e2e_steps):
+        hp.step_e2e()
+    e1.record()
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1))
+    e2e_value = total_events_all * e2e_steps / (e2e_ms * 1e-3)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
+
+    peak_gbs, peak_src = measured_peaks()
+    dom = max(kernel_ms, key=kernel_ms.get)
+    bytes_per_launch = 8.0 * hp.total          # 8 algorithmic bytes per event for either kernel
+    achieved = bytes_per_launch / (kernel_ms[dom] * 1e-3) / 1e9
+    roofline = {
+        "bound": "hbm", "kernel": {"expand": "expand_kernel (8 B written / event)",
+                                   "scan": "scan_kernel (8 B read / event)"}[dom],
+        "achieved": achieved, "peak": peak_gbs, "unit": "GB/s", "frac": achieved / peak_gbs,
+        "peak_source": peak_src, "traffic": None,
+        "per_kernel": {k: {"ms": kernel_ms[k], "gbs": bytes_per_launch / (kernel_ms[k] * 1e-3) / 1e9,
+                           "frac": bytes_per_launch / (kernel_ms[k] * 1e-3) / 1e9 / peak_gbs}
+                       for k in kernel_ms},
+        "materialised_path_gbs": 2 * bytes_per_launch / ((kernel_ms["expand"] + kernel_ms["scan"]) * 1e-3) / 1e9,
+        "frac_of_nominal_8000": achieved / 8000.0,
+    }
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+        "configs_per_sec": configs_all * args.steps / (ms * 1e-3),
+        "config": {"workload": "G5 stress grid: deep/wide decoders, materialised int64 event lists",
+                   "configs_per_gpu": hp.n, "events_per_gpu": hp.total, "capacities": len(caps),
+                   "bmax": grids.G4_BMAX, "parallelism": f"replicas x{world} (independent configs, no collective)",
+                   "l2": "event list (8 B/event) far larger than the 126 MB L2; no flush needed",
+                   "step": "event_counts + expand(fused rounding) + scan_peak + max_batch + select_method"},
+        "roofline": roofline,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": hp.h2d_bytes,
+                "d2h_bytes_per_step": hp.d2h_bytes, "ms_per_step": e2e_ms / e2e_steps},
+        "gpu_launches": HotPath.KERNELS_PER_STEP * args.steps,
+        "clocks": clocks,
+        "fused_equals_materialised": agree,
+    }
+    if args.cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline()
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0 if agree else 4
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
+    ap.add_argument("--configs", type=int, default=grids.G5_CONFIGS,
+                    help="configurations of the stress grid per GPU (default: the full grid)")
+    ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world == 1 and args.gpus > 1:
+        # launched without torchrun: re-launch one rank per GPU
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", "29511", os.path.abspath(__file__)] + sys.argv[1:]
+        return subprocess.call(cmd)
+    if int(os.environ.get("RANK", "0")) != 0:
+        args.cpu_baseline = False
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

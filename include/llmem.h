@@ -1,0 +1,195 @@
+/*
+ * llmem.h -- C ABI of the batched LLMem peak-memory estimator for NVIDIA B200 (sm_100a).
+ *
+ * The library evaluates, for very many fine-tuning configurations at once, the
+ * peak per-device memory model of Kim et al., "LLMem: Estimating GPU Memory
+ * Usage for Fine-Tuning Pre-Trained LLMs" (arXiv 2404.10933):
+ *
+ *   Section 4.2   m_peak^s = m_base + m_p + m_os + m_out + m_lm        (single device / CDP)
+ *   Section 5     m_peak^dp, m_peak^tp, m_peak^dp+tp and m_back^tp     (ZeRO-3, 1-D TP, DP+TP)
+ *   Section 6     Algorithm 1: largest batch per method, scores, selection
+ *
+ * Every term is expanded into allocate/free events in the phase order of
+ * Sections 4.1 and 5 (initialisation, gather, output phase, TP backward
+ * buffers, frees, optimizer states in the first iteration); every event is
+ * rounded up to the CUDA page size cu_p = 2 * 1024^2 bytes (Section 4.2); the
+ * peak is m_base + lm_p + the largest prefix sum of the rounded list.
+ *
+ * Conventions
+ *   - "DEV" pointers are device pointers owned by the caller; "HOST" are host
+ *     pointers.  The library allocates no device memory and keeps no state
+ *     between calls except the text returned by llmem_last_error().
+ *   - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*, NULL =
+ *     default stream) and return without synchronising.  Outputs are valid once
+ *     the stream has reached the end of the enqueued work.
+ *   - The return code reports call-level problems (bad pointer, size, scratch,
+ *     launch failure).  Problems of a single configuration are reported per
+ *     element: status_out[i] != 0 and the element's outputs are -1.  Nothing
+ *     traps, asserts or aborts on the device.
+ *   - All byte quantities are int64.  Supported results are < 2^62 bytes and
+ *     < 2^31 events per configuration; beyond that the element gets status 3.
+ *   - `scratch` must be 256-byte aligned, at least llmem_scratch_bytes() long,
+ *     and must not be shared by calls that may overlap on the device.
+ */
+#ifndef LLMEM_H_
+#define LLMEM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DEV
+#define HOST
+
+/* One fine-tuning configuration: the symbols of Table 1 that the equations use,
+ * plus the method and its modelled partition degrees.  64 bytes, no padding. */
+typedef struct __attribute__((aligned(16))) llmem_config {
+  int32_t layers;      /* l_n, 1 .. 2^16 */
+  int32_t hidden;      /* o_n, 1 .. 2^20 */
+  int32_t heads;       /* >= 1 and a divisor of hidden; no term of the model depends on it */
+  int32_t ffn;         /* inner width of the feed-forward block, 1 .. 2^22 */
+  int32_t vocab;       /* dict_n, 1 .. 2^26 */
+  int32_t pos_len;     /* rows of a learned position Embedding, 0 = none; 0 .. 2^26 (fixes e_n) */
+  int32_t seq;         /* sl, 1 .. 2^26 */
+  int32_t batch;       /* bs, 1 .. 2^26; ignored by llmem_max_batch / llmem_select_method */
+  int64_t chunk_elems; /* cs in elements, 1 .. 2^40 */
+  int64_t base_bytes;  /* m_base, 0 .. 2^60, added without rounding */
+  uint8_t method;      /* LLMEM_METHOD_*; ignored by llmem_select_method */
+  uint8_t gpu_n;       /* >= 1; a plain number, nothing runs across devices */
+  uint8_t tp_n;        /* DP+TP only: 2 <= tp_n <= gpu_n/2 and tp_n | gpu_n */
+  uint8_t lm_bytes;    /* B of the m_lm equation: 2 or 4 */
+  uint8_t ffn_kind;    /* 0: two feed-forward matrices, 1: three (gated) */
+  uint8_t has_bias;    /* 0 / 1: Linear biases and norm biases present */
+  uint8_t iters;       /* fine-tuning iterations spanned by the event list, >= 1;
+                          2 or more gives the paper's peak */
+  uint8_t reserved[9]; /* must be 0 */
+} llmem_config;
+
+enum { LLMEM_METHOD_CDP = 0, LLMEM_METHOD_ADP = 1, LLMEM_METHOD_TP = 2, LLMEM_METHOD_DPTP = 3,
+       LLMEM_METHOD_OFFLOAD = 4 /* only ever an output of llmem_select_method */ };
+
+typedef enum {
+  LLMEM_OK = 0,
+  LLMEM_ERR_ARG = 1,     /* null / misaligned pointer, negative size, bmax out of range */
+  LLMEM_ERR_SCRATCH = 2, /* scratch missing, misaligned or too small */
+  LLMEM_ERR_CUDA = 3,    /* a CUDA runtime call failed; text in llmem_last_error() */
+  LLMEM_ERR_TIMEOUT = 4  /* a bounded device-side wait ran out (llmem_scratch_status only) */
+} llmem_status;
+
+/* per-configuration status bytes */
+enum { LLMEM_CFG_OK = 0, LLMEM_CFG_FIELD = 1 /* a field outside its range */,
+       LLMEM_CFG_COMBO = 2 /* method / gpu_n / tp_n not admissible */,
+       LLMEM_CFG_OVERFLOW = 3 /* >= 2^31 events or >= 2^62 bytes */ };
+
+/* operations, for llmem_scratch_bytes */
+enum { LLMEM_OP_ESTIMATE = 0, LLMEM_OP_EVENT_COUNTS = 1, LLMEM_OP_EXPAND = 2, LLMEM_OP_ROUND = 3,
+       LLMEM_OP_SCAN_PEAK = 4, LLMEM_OP_MAX_BATCH = 5, LLMEM_OP_SELECT = 6 };
+
+/* call flags */
+#define LLMEM_SELECT_ALLZERO 1u /* llmem_select_method: offload only if every score is 0 */
+#define LLMEM_FUSE_ROUND 2u     /* llmem_expand_events: write page-rounded deltas;
+                                   llmem_scan_peak: round each delta while reading */
+
+/* Bytes of scratch the operation needs for n configurations and total_events
+ * events (0 where it needs none; such calls accept scratch = NULL). */
+size_t llmem_scratch_bytes(int op, int64_t n, int64_t total_events);
+
+/* Sections 4.2 and 5, fused: peak of each configuration without materialising
+ * its event list (identical runs of events are summed in registers).
+ *   cfg            DEV [n]
+ *   peak_out       DEV [n]   m_base + lm_p + largest prefix sum of the rounded events, -1 on status != 0
+ *   peak_index_out DEV [n]   nullable; 0-based index of the first event whose prefix attains the peak
+ *   status_out     DEV [n]   nullable; LLMEM_CFG_* */
+llmem_status llmem_estimate_batch(const llmem_config* DEV cfg, int64_t n, int64_t* DEV peak_out,
+                                  int64_t* DEV peak_index_out, uint8_t* DEV status_out,
+                                  void* DEV scratch, size_t scratch_bytes, uint32_t flags,
+                                  void* cuda_stream);
+
+/* Sections 4.1 and 5: number of allocate/free events of each configuration
+ * (0 on status != 0) as an exclusive prefix sum.
+ *   offsets_out    DEV [n+1] offsets_out[0] = 0, offsets_out[n] = total number of events
+ *   status_out     DEV [n]   nullable */
+llmem_status llmem_event_counts(const llmem_config* DEV cfg, int64_t n, int64_t* DEV offsets_out,
+                                uint8_t* DEV status_out, void* DEV scratch, size_t scratch_bytes,
+                                uint32_t flags, void* cuda_stream);
+
+/* Sections 4.1 and 5: the signed byte count of every event, allocations
+ * positive and frees negative, configuration i occupying
+ * delta_out[offsets[i] .. offsets[i+1]).  Order: initialisation (embedding unit,
+ * then each chunk: fp16, fp32); per iteration gather, embedding and layer
+ * outputs, logits, two shifted copies, TP backward buffers, then the frees in
+ * reverse; optimizer states (per Embedding / Linear tensor) after the first
+ * iteration.  With LLMEM_FUSE_ROUND the magnitudes are page-rounded.
+ *   offsets        DEV [n+1] as written by llmem_event_counts for the same cfg
+ *   total_events   HOST value of offsets[n]
+ *   delta_out      DEV [total_events], 8-byte aligned (16-byte alignment enables bulk stores) */
+llmem_status llmem_expand_events(const llmem_config* DEV cfg, int64_t n, const int64_t* DEV offsets,
+                                 int64_t total_events, int64_t* DEV delta_out, void* DEV scratch,
+                                 size_t scratch_bytes, uint32_t flags, void* cuda_stream);
+
+/* Section 4.2, every ceil(x / cu_p) * cu_p: round each magnitude up to a
+ * multiple of 2 MiB in place, keeping the sign. */
+llmem_status llmem_round_events(int64_t* DEV delta, int64_t total_events, void* DEV scratch,
+                                size_t scratch_bytes, uint32_t flags, void* cuda_stream);
+
+/* Sections 4.2 and 5 (the peaks are these sums): per segment, the largest
+ * prefix sum of delta[offsets[i] .. offsets[i+1]) and the first index attaining
+ * it, plus m_base + lm_p of cfg[i] when cfg is given.  An empty segment yields
+ * offset + 0 and index -1; with cfg, an inadmissible cfg[i] yields -1 / -1.
+ *   delta          DEV [total_events]; any signed values whose prefix sums stay within int64
+ *   cfg            DEV [n], nullable (then the offset is 0)
+ *   scratch        required; holds a device status word readable with llmem_scratch_status */
+llmem_status llmem_scan_peak(const int64_t* DEV delta, const int64_t* DEV offsets, int64_t n,
+                             int64_t total_events, const llmem_config* DEV cfg,
+                             int64_t* DEV peak_out, int64_t* DEV peak_index_out, void* DEV scratch,
+                             size_t scratch_bytes, uint32_t flags, void* cuda_stream);
+
+/* Algorithm 1, the inner loop of every method: the largest batch b in 1..bmax
+ * whose peak does not exceed the capacity (0 if even b = 1 does not fit, -1 on
+ * status != 0).  The paper increments b; the peak is non-decreasing in b, so the
+ * library bisects.
+ *   shape          DEV [n]      method, gpu_n, tp_n used; batch ignored
+ *   capacity_bytes DEV [n_cap]  m_total values
+ *   bmax           1 .. 2^26
+ *   bs_out         DEV [n][n_cap] */
+llmem_status llmem_max_batch(const llmem_config* DEV shape, int64_t n,
+                             const int64_t* DEV capacity_bytes, int32_t n_cap, int32_t bmax,
+                             int32_t* DEV bs_out, uint8_t* DEV status_out, void* DEV scratch,
+                             size_t scratch_bytes, uint32_t flags, void* cuda_stream);
+
+/* Algorithm 1 in full: the four largest batches, the scores
+ * [1.5 bs gpu_n, bs gpu_n, bs, bs gpu_n/tp_n], the first maximum in the order
+ * CDP, ADP, TP, DP+TP, and (LLMEM_METHOD_OFFLOAD, 0) when the TP score is 0
+ * (with LLMEM_SELECT_ALLZERO: when all four are 0).  A method that is not
+ * admissible for (gpu_n, tp_n) scores 0.
+ *   method_out, batch_out DEV [n][n_cap]
+ *   bs_list_out           DEV [n][n_cap][4], nullable */
+llmem_status llmem_select_method(const llmem_config* DEV shape, int64_t n,
+                                 const int64_t* DEV capacity_bytes, int32_t n_cap, int32_t bmax,
+                                 int32_t* DEV method_out, int32_t* DEV batch_out,
+                                 int32_t* DEV bs_list_out, uint8_t* DEV status_out,
+                                 void* DEV scratch, size_t scratch_bytes, uint32_t flags,
+                                 void* cuda_stream);
+
+/* Synchronises cuda_stream and returns the device status word that
+ * llmem_scan_peak keeps at the start of its scratch: LLMEM_OK, or
+ * LLMEM_ERR_TIMEOUT if a bounded wait inside a kernel gave up (outputs are then
+ * undefined). */
+llmem_status llmem_scratch_status(const void* DEV scratch, void* cuda_stream);
+
+/* Text of the last error on the calling thread ("" if none). */
+const char* llmem_last_error(void);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int llmem_version(void);
+
+#undef DEV
+#undef HOST
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LLMEM_H_ */

@@ -1,0 +1,252 @@
+"""Batched LLMem peak-memory estimation on NVIDIA B200.
+
+Thin Python binding of ``csrc/libllmem.so`` (C ABI declared in
+``include/llmem.h``).  The functions here only marshal arguments: they allocate
+output and scratch tensors with PyTorch, pass raw device pointers and the current
+CUDA stream, and check return codes.  Every step of the estimation runs in the
+library's CUDA kernels.  There is no CPU fallback: if the shared library is
+missing or fails to load, importing a function that needs it raises.
+
+Configurations are 64-byte records (``grids.CONFIG_DTYPE``); on the device they
+are ``torch.uint8`` tensors of shape ``[n, 64]``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+
+from . import grids  # noqa: F401  (input generators; no part of the model)
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "csrc", "libllmem.so")
+
+OK, ERR_ARG, ERR_SCRATCH, ERR_CUDA, ERR_TIMEOUT = 0, 1, 2, 3, 4
+OP_ESTIMATE, OP_EVENT_COUNTS, OP_EXPAND, OP_ROUND, OP_SCAN_PEAK, OP_MAX_BATCH, OP_SELECT = range(7)
+SELECT_ALLZERO = 1
+FUSE_ROUND = 2
+METHOD_OFFLOAD = 4
+
+EXPORTS = (
+    "llmem_scratch_bytes", "llmem_estimate_batch", "llmem_event_counts", "llmem_expand_events",
+    "llmem_round_events", "llmem_scan_peak", "llmem_max_batch", "llmem_select_method",
+    "llmem_scratch_status", "llmem_last_error", "llmem_version",
+)
+
+
+class LlmemError(RuntimeError):
+    def __init__(self, code: int, text: str):
+        super().__init__(f"llmem status {code}: {text}")
+        self.code = code
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C-ABI library.  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2404_10933_b200._build` "
+                "(needs nvcc); this package has no CPU fallback")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i64, i32, u32, sz = (ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_uint32,
+                                 ctypes.c_size_t)
+        L.llmem_scratch_bytes.restype = sz
+        L.llmem_scratch_bytes.argtypes = [ctypes.c_int, i64, i64]
+        L.llmem_estimate_batch.argtypes = [vp, i64, vp, vp, vp, vp, sz, u32, vp]
+        L.llmem_event_counts.argtypes = [vp, i64, vp, vp, vp, sz, u32, vp]
+        L.llmem_expand_events.argtypes = [vp, i64, vp, i64, vp, vp, sz, u32, vp]
+        L.llmem_round_events.argtypes = [vp, i64, vp, sz, u32, vp]
+        L.llmem_scan_peak.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, sz, u32, vp]
+        L.llmem_max_batch.argtypes = [vp, i64, vp, i32, i32, vp, vp, vp, sz, u32, vp]
+        L.llmem_select_method.argtypes = [vp, i64, vp, i32, i32, vp, vp, vp, vp, vp, sz, u32, vp]
+        L.llmem_scratch_status.argtypes = [vp, vp]
+        L.llmem_last_error.restype = ctypes.c_char_p
+        L.llmem_version.restype = ctypes.c_int
+        for name in EXPORTS:
+            getattr(L, name)  # every declared entry point must be exported
+        _lib = L
+    return _lib
+
+
+def _check(code: int) -> None:
+    if code != OK:
+        raise LlmemError(code, lib().llmem_last_error().decode())
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def _stream_ptr(stream) -> int:
+    torch = _torch()
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else int(t.data_ptr())
+
+
+def to_device(cfg: np.ndarray, device="cuda", non_blocking: bool = False):
+    """Copy 64-byte configuration records to a ``[n, 64]`` uint8 device tensor."""
+    torch = _torch()
+    cfg = np.ascontiguousarray(cfg)
+    if cfg.dtype.itemsize != 64:
+        raise ValueError("configuration records must be 64 bytes")
+    host = torch.from_numpy(cfg.reshape(-1).view(np.uint8).reshape(-1, 64))
+    return host.to(device, non_blocking=non_blocking)
+
+
+def _as_cfg(cfg):
+    torch = _torch()
+    if isinstance(cfg, np.ndarray):
+        cfg = to_device(cfg)
+    if cfg.dtype != torch.uint8 or cfg.dim() != 2 or cfg.shape[1] != 64 or not cfg.is_cuda:
+        raise ValueError("cfg must be a CUDA uint8 tensor of shape [n, 64]")
+    return cfg.contiguous()
+
+
+def scratch_bytes(op: int, n: int, total_events: int = 0) -> int:
+    return int(lib().llmem_scratch_bytes(op, n, total_events))
+
+
+def _scratch(op: int, n: int, total: int, device):
+    torch = _torch()
+    nbytes = scratch_bytes(op, n, total)
+    if nbytes == 0:
+        return None, 0
+    return torch.empty(nbytes, dtype=torch.uint8, device=device), nbytes
+
+
+def estimate_batch(cfg, *, want_index: bool = True, want_status: bool = True, stream=None):
+    """Fused estimate.  Returns dict(peak[n] int64, index[n] int64 | None, status[n] uint8 | None)."""
+    torch = _torch()
+    cfg = _as_cfg(cfg)
+    n = cfg.shape[0]
+    peak = torch.empty(n, dtype=torch.int64, device=cfg.device)
+    index = torch.empty(n, dtype=torch.int64, device=cfg.device) if want_index else None
+    status = torch.empty(n, dtype=torch.uint8, device=cfg.device) if want_status else None
+    _check(lib().llmem_estimate_batch(_ptr(cfg), n, _ptr(peak), _ptr(index), _ptr(status), None, 0, 0,
+                                      _stream_ptr(stream)))
+    return {"peak": peak, "index": index, "status": status}
+
+
+def event_counts(cfg, *, want_status: bool = True, stream=None):
+    """Returns (offsets[n+1] int64 exclusive scan of event counts, status[n] | None)."""
+    torch = _torch()
+    cfg = _as_cfg(cfg)
+    n = cfg.shape[0]
+    offsets = torch.empty(n + 1, dtype=torch.int64, device=cfg.device)
+    status = torch.empty(n, dtype=torch.uint8, device=cfg.device) if want_status else None
+    scratch, nbytes = _scratch(OP_EVENT_COUNTS, n, 0, cfg.device)
+    _check(lib().llmem_event_counts(_ptr(cfg), n, _ptr(offsets), _ptr(status), _ptr(scratch), nbytes, 0,
+                                    _stream_ptr(stream)))
+    return offsets, status
+
+
+def expand_events(cfg, offsets, total_events: Optional[int] = None, *, fuse_round: bool = False,
+                  out=None, stream=None):
+    """Materialise the signed event list.  ``total_events`` defaults to ``offsets[-1]`` (one
+    device-to-host read)."""
+    torch = _torch()
+    cfg = _as_cfg(cfg)
+    n = cfg.shape[0]
+    if total_events is None:
+        total_events = int(offsets[-1].item())
+    if out is None:
+        out = torch.empty(total_events, dtype=torch.int64, device=cfg.device)
+    elif out.numel() < total_events or out.dtype != torch.int64:
+        raise ValueError("out must be an int64 tensor with at least total_events elements")
+    _check(lib().llmem_expand_events(_ptr(cfg), n, _ptr(offsets), total_events, _ptr(out), None, 0,
+                                     FUSE_ROUND if fuse_round else 0, _stream_ptr(stream)))
+    return out[:total_events] if out.numel() != total_events else out
+
+
+def round_events(delta, stream=None):
+    """Round every magnitude up to the 2 MiB page, in place."""
+    _check(lib().llmem_round_events(_ptr(delta), delta.numel(), None, 0, 0, _stream_ptr(stream)))
+    return delta
+
+
+def scan_peak(delta, offsets, cfg=None, *, fuse_round: bool = False, want_index: bool = True,
+              scratch=None, stream=None, check_status: bool = False):
+    """Segmented prefix-sum + max.  Returns dict(peak[n], index[n] | None, scratch)."""
+    torch = _torch()
+    n = offsets.numel() - 1
+    total = delta.numel()
+    if cfg is not None:
+        cfg = _as_cfg(cfg)
+    peak = torch.empty(n, dtype=torch.int64, device=offsets.device)
+    index = torch.empty(n, dtype=torch.int64, device=offsets.device) if want_index else None
+    if scratch is None:
+        scratch, nbytes = _scratch(OP_SCAN_PEAK, n, total, offsets.device)
+    else:
+        nbytes = scratch.numel()
+    _check(lib().llmem_scan_peak(_ptr(delta), _ptr(offsets), n, total, _ptr(cfg), _ptr(peak), _ptr(index),
+                                 _ptr(scratch), nbytes, FUSE_ROUND if fuse_round else 0,
+                                 _stream_ptr(stream)))
+    if check_status:
+        _check(lib().llmem_scratch_status(_ptr(scratch), _stream_ptr(stream)))
+    return {"peak": peak, "index": index, "scratch": scratch}
+
+
+def max_batch(shape, capacities, bmax: int, *, want_status: bool = True, stream=None):
+    """Largest fitting batch.  Returns (bs[n, n_cap] int32, status[n] | None)."""
+    torch = _torch()
+    shape = _as_cfg(shape)
+    n = shape.shape[0]
+    caps = _caps(capacities, shape.device)
+    bs = torch.empty((n, caps.numel()), dtype=torch.int32, device=shape.device)
+    status = torch.empty(n, dtype=torch.uint8, device=shape.device) if want_status else None
+    _check(lib().llmem_max_batch(_ptr(shape), n, _ptr(caps), caps.numel(), bmax, _ptr(bs), _ptr(status),
+                                 None, 0, 0, _stream_ptr(stream)))
+    return bs, status
+
+
+def select_method(shape, capacities, bmax: int, *, allzero: bool = False, want_bs_list: bool = True,
+                  want_status: bool = True, stream=None):
+    """Algorithm 1.  Returns dict(method[n, n_cap], batch[n, n_cap], bs_list[n, n_cap, 4] | None,
+    status[n] | None)."""
+    torch = _torch()
+    shape = _as_cfg(shape)
+    n = shape.shape[0]
+    caps = _caps(capacities, shape.device)
+    m = caps.numel()
+    method = torch.empty((n, m), dtype=torch.int32, device=shape.device)
+    batch = torch.empty((n, m), dtype=torch.int32, device=shape.device)
+    bs_list = torch.empty((n, m, 4), dtype=torch.int32, device=shape.device) if want_bs_list else None
+    status = torch.empty(n, dtype=torch.uint8, device=shape.device) if want_status else None
+    _check(lib().llmem_select_method(_ptr(shape), n, _ptr(caps), m, bmax, _ptr(method), _ptr(batch),
+                                     _ptr(bs_list), _ptr(status), None, 0,
+                                     SELECT_ALLZERO if allzero else 0, _stream_ptr(stream)))
+    return {"method": method, "batch": batch, "bs_list": bs_list, "status": status}
+
+
+def _caps(capacities, device):
+    torch = _torch()
+    if isinstance(capacities, torch.Tensor):
+        caps = capacities.to(device=device, dtype=torch.int64).contiguous().reshape(-1)
+    else:
+        caps = torch.as_tensor(np.asarray(capacities, dtype=np.int64).reshape(-1)).to(device)
+    return caps
+
+
+def estimate_materialized(cfg, *, fuse_round: bool = True, stream=None):
+    """The materialised path end to end: event counts -> expansion -> (rounding) ->
+    segmented scan.  Returns dict(peak, index, status, offsets, total_events)."""
+    cfg = _as_cfg(cfg)
+    offsets, status = event_counts(cfg, stream=stream)
+    total = int(offsets[-1].item())
+    delta = expand_events(cfg, offsets, total, fuse_round=fuse_round, stream=stream)
+    if not fuse_round:
+        round_events(delta, stream=stream)
+    r = scan_peak(delta, offsets, cfg, stream=stream)
+    return {"peak": r["peak"], "index": r["index"], "status": status, "offsets": offsets,
+            "total_events": total}

@@ -1,0 +1,243 @@
+// Fused kernels: peak estimation without a materialised event list, largest-batch
+// search and Algorithm 1.  One thread evaluates one configuration (four threads per
+// shape in the selection kernel); identical consecutive events are summed as
+// count * rounded size, which is exact because all allocations of an iteration
+// precede its frees.  The work is plain 64-bit integer arithmetic; global traffic is
+// 64 bytes in and a few bytes out per configuration.
+#include "llmem_host.h"
+#include "llmem_model.cuh"
+
+namespace llmem {
+
+// Peak of one admissible plan at a given batch: m_base + lm_p + largest prefix sum.
+// Returns kSat when the value does not fit below 2^62.
+struct Search {
+  Plan p;
+  StaticSums s;
+  __device__ __forceinline__ u64 peak(u64 batch, Dyn* d_out, bool* first_wins) const {
+    Dyn d = make_dyn(p, batch);
+    if (d_out) *d_out = d;
+    u64 rel = relative_peak(p, s, sat_add(s.gather, dyn_sum(p, d)), first_wins);
+    return sat_add(p.offset, rel);
+  }
+  // Section 6: the largest b in 1..bmax with peak(b) <= capacity.  Algorithm 1
+  // increments b until the peak exceeds m_total; the peak never decreases with b,
+  // so bisection finds the same b.
+  __device__ __forceinline__ int largest_batch(i64 capacity, int bmax) const {
+    int lo = 0, hi = bmax;
+    while (lo < hi) {
+      int mid = lo + (hi - lo + 1) / 2;
+      bool fw;
+      u64 pk = peak((u64)mid, nullptr, &fw);
+      if (pk < kSat && (i64)pk <= capacity)
+        lo = mid;
+      else
+        hi = mid - 1;
+    }
+    return lo;
+  }
+};
+
+// ---------------------------------------------------------------------------
+// llmem_estimate_batch
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+estimate_kernel(const llmem_config* __restrict__ cfg, i64 n, i64* __restrict__ peak_out,
+                i64* __restrict__ index_out, uint8_t* __restrict__ status_out) {
+  for (i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (i64)gridDim.x * blockDim.x) {
+    Cfg f = load_cfg(cfg + i);
+    int st = check_fields(f, true, true);
+    i64 pk = -1, ix = -1;
+    if (st == LLMEM_CFG_OK) {
+      Search q;
+      q.p = make_plan(f, f.method);
+      st = q.p.status;
+      if (st == LLMEM_CFG_OK) {
+        q.s = make_static_sums(q.p, f.pos_len > 0);
+        Dyn d;
+        bool first_wins;
+        u64 total = q.peak((u64)f.batch, &d, &first_wins);
+        if (total >= kSat) {
+          st = LLMEM_CFG_OVERFLOW;
+        } else {
+          pk = (i64)total;
+          const Plan& p = q.p;
+          // position of the peak: the last allocation of non-zero size in the
+          // iteration that attains it, or the last optimizer-state allocation
+          const u64 init_n = 2 + 2 * (u64)p.C;
+          const u64 gpart = p.gather ? 1 + (u64)p.C : 0;
+          const u64 allocs = gpart + (u64)p.e_n + (u64)p.L + 3 + (p.tpback ? (u64)p.L : 0);
+          const u64 os_n = (u64)p.e_n + (u64)p.K * (u64)p.L;
+          const u64 last = (p.tpback && d.back > 0) ? allocs - 1
+                           : (d.shift > 0 ? gpart + p.e_n + p.L + 2 : gpart + p.e_n + p.L);
+          if (p.iters >= 2) ix = (i64)(init_n + 2 * allocs + os_n + last);
+          else if (first_wins) ix = (i64)(init_n + last);
+          else ix = (i64)(init_n + 2 * allocs + os_n - 1);
+        }
+      }
+    }
+    peak_out[i] = pk;
+    if (index_out) index_out[i] = ix;
+    if (status_out) status_out[i] = (uint8_t)st;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// llmem_max_batch: one thread per shape, capacities innermost (the peak curve
+// does not depend on the capacity, so the plan is built once)
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+max_batch_kernel(const llmem_config* __restrict__ shape, i64 n, const i64* __restrict__ caps,
+                 int n_cap, int bmax, int* __restrict__ bs_out, uint8_t* __restrict__ status_out) {
+  for (i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (i64)gridDim.x * blockDim.x) {
+    Cfg f = load_cfg(shape + i);
+    int st = check_fields(f, false, true);
+    Search q;
+    if (st == LLMEM_CFG_OK) {
+      q.p = make_plan(f, f.method);
+      st = q.p.status;
+    }
+    int* out = bs_out + i * n_cap;
+    if (st != LLMEM_CFG_OK) {
+      for (int m = 0; m < n_cap; ++m) out[m] = -1;
+    } else {
+      q.s = make_static_sums(q.p, f.pos_len > 0);
+      for (int m = 0; m < n_cap; ++m) out[m] = q.largest_batch(__ldg(caps + m), bmax);
+    }
+    if (status_out) status_out[i] = (uint8_t)st;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// llmem_select_method: four lanes per shape, lane k searching method k; the
+// quad exchanges its four batches by shuffle and lane 0 takes the decision.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+select_kernel(const llmem_config* __restrict__ shape, i64 n, const i64* __restrict__ caps, int n_cap,
+              int bmax, u32 flags, int* __restrict__ method_out, int* __restrict__ batch_out,
+              int* __restrict__ bs_list_out, uint8_t* __restrict__ status_out) {
+  const i64 quads_per_grid = ((i64)gridDim.x * blockDim.x) >> 2;
+  const u32 k = threadIdx.x & 3;  // method of this lane
+  const u32 quad_base = (threadIdx.x & 31) & ~3u;
+  // n rounded up so that whole warps stay in the loop (shuffles need all lanes)
+  const i64 n_warp_rounded = (n + 7) & ~(i64)7;
+  for (i64 i = ((i64)blockIdx.x * blockDim.x + threadIdx.x) >> 2; i < n_warp_rounded; i += quads_per_grid) {
+    const bool live = i < n;
+    int st = LLMEM_CFG_FIELD;
+    Search q;
+    bool usable = false;
+    u32 gpu_n = 1, tp_n = 1;
+    if (live) {
+      Cfg f = load_cfg(shape + i);
+      st = check_fields(f, false, false);
+      gpu_n = f.gpu_n;
+      tp_n = f.tp_n;
+      if (st == LLMEM_CFG_OK) {
+        q.p = make_plan(f, k);
+        usable = q.p.status == LLMEM_CFG_OK;  // a method that cannot be configured scores 0
+        if (usable) q.s = make_static_sums(q.p, f.pos_len > 0);
+      }
+    }
+    for (int m = 0; m < n_cap; ++m) {
+      int bs = 0;
+      if (usable) bs = q.largest_batch(__ldg(caps + m), bmax);
+      int b0 = __shfl_sync(0xffffffffu, bs, quad_base + 0);
+      int b1 = __shfl_sync(0xffffffffu, bs, quad_base + 1);
+      int b2 = __shfl_sync(0xffffffffu, bs, quad_base + 2);
+      int b3 = __shfl_sync(0xffffffffu, bs, quad_base + 3);
+      if (!live) continue;
+      const i64 o = i * n_cap + m;
+      if (st != LLMEM_CFG_OK) {
+        if (k == 0) { method_out[o] = -1; batch_out[o] = -1; }
+        if (bs_list_out) bs_list_out[4 * o + k] = -1;
+        continue;
+      }
+      if (bs_list_out) bs_list_out[4 * o + k] = bs;
+      if (k == 0) {
+        // scores doubled so that CDP's factor 1.5 stays integral; dp_n = gpu_n / tp_n
+        const i64 nn = gpu_n;
+        i64 e0 = 3 * (i64)b0 * nn, e1 = 2 * (i64)b1 * nn, e2 = 2 * (i64)b2;
+        i64 e3 = b3 > 0 ? 2 * (i64)b3 * (nn / tp_n) : 0;
+        int idx = 0, bb = b0;
+        i64 best = e0;
+        if (e1 > best) { best = e1; idx = 1; bb = b1; }
+        if (e2 > best) { best = e2; idx = 2; bb = b2; }
+        if (e3 > best) { best = e3; idx = 3; bb = b3; }
+        const bool keep = (flags & LLMEM_SELECT_ALLZERO) ? (best != 0) : (e2 != 0);
+        method_out[o] = keep ? idx : LLMEM_METHOD_OFFLOAD;
+        batch_out[o] = keep ? bb : 0;
+      }
+    }
+    if (live && k == 0 && status_out) status_out[i] = (uint8_t)st;
+  }
+}
+
+static int grid_for(i64 threads_needed, int block, int ctas_per_sm) {
+  i64 blocks = (threads_needed + block - 1) / block;
+  i64 cap = (i64)sm_count() * ctas_per_sm;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  return (int)blocks;
+}
+
+}  // namespace llmem
+
+using namespace llmem;
+
+extern "C" llmem_status llmem_estimate_batch(const llmem_config* cfg, int64_t n, int64_t* peak_out,
+                                             int64_t* peak_index_out, uint8_t* status_out,
+                                             void* scratch, size_t scratch_bytes, uint32_t flags,
+                                             void* cuda_stream) {
+  (void)scratch; (void)scratch_bytes; (void)flags;
+  clear_error();
+  if (n < 0) { set_error("llmem_estimate_batch: n < 0"); return LLMEM_ERR_ARG; }
+  if (n == 0) return LLMEM_OK;
+  if (!cfg || !peak_out) { set_error("llmem_estimate_batch: cfg and peak_out are required"); return LLMEM_ERR_ARG; }
+  if (!aligned_to(cfg, 16) || !aligned_to(peak_out, 8) || !aligned_to(peak_index_out, 8)) {
+    set_error("llmem_estimate_batch: cfg must be 16-byte and outputs 8-byte aligned");
+    return LLMEM_ERR_ARG;
+  }
+  estimate_kernel<<<grid_for(n, 256, 8), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      cfg, n, reinterpret_cast<i64*>(peak_out), reinterpret_cast<i64*>(peak_index_out), status_out);
+  return check_launch("llmem_estimate_batch");
+}
+
+static llmem_status check_search_args(const char* who, const llmem_config* shape, int64_t n,
+                                      const int64_t* caps, int32_t n_cap, int32_t bmax) {
+  if (n < 0 || n_cap < 0) { set_error("%s: negative size", who); return LLMEM_ERR_ARG; }
+  if (bmax < 1 || bmax > (1 << 26)) { set_error("%s: bmax must be in 1 .. 2^26", who); return LLMEM_ERR_ARG; }
+  if (n == 0 || n_cap == 0) return LLMEM_OK;
+  if (!shape || !caps) { set_error("%s: shape and capacity_bytes are required", who); return LLMEM_ERR_ARG; }
+  if (!aligned_to(shape, 16) || !aligned_to(caps, 8)) { set_error("%s: misaligned input", who); return LLMEM_ERR_ARG; }
+  return LLMEM_OK;
+}
+
+extern "C" llmem_status llmem_max_batch(const llmem_config* shape, int64_t n,
+                                        const int64_t* capacity_bytes, int32_t n_cap, int32_t bmax,
+                                        int32_t* bs_out, uint8_t* status_out, void* scratch,
+                                        size_t scratch_bytes, uint32_t flags, void* cuda_stream) {
+  (void)scratch; (void)scratch_bytes; (void)flags;
+  clear_error();
+  llmem_status st = check_search_args("llmem_max_batch", shape, n, capacity_bytes, n_cap, bmax);
+  if (st != LLMEM_OK || n == 0 || n_cap == 0) return st;
+  if (!bs_out || !aligned_to(bs_out, 4)) { set_error("llmem_max_batch: bs_out is required"); return LLMEM_ERR_ARG; }
+  max_batch_kernel<<<grid_for(n, 256, 8), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      shape, n, reinterpret_cast<const i64*>(capacity_bytes), n_cap, bmax, bs_out, status_out);
+  return check_launch("llmem_max_batch");
+}
+
+extern "C" llmem_status llmem_select_method(const llmem_config* shape, int64_t n,
+                                            const int64_t* capacity_bytes, int32_t n_cap,
+                                            int32_t bmax, int32_t* method_out, int32_t* batch_out,
+                                            int32_t* bs_list_out, uint8_t* status_out, void* scratch,
+                                            size_t scratch_bytes, uint32_t flags, void* cuda_stream) {
+  (void)scratch; (void)scratch_bytes;
+  clear_error();
+  llmem_status st = check_search_args("llmem_select_method", shape, n, capacity_bytes, n_cap, bmax);
+  if (st != LLMEM_OK || n == 0 || n_cap == 0) return st;
+  if (!method_out || !batch_out) { set_error("llmem_select_method: method_out and batch_out are required"); return LLMEM_ERR_ARG; }
+  select_kernel<<<grid_for(4 * n, 256, 8), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      shape, n, reinterpret_cast<const i64*>(capacity_bytes), n_cap, bmax, flags, method_out,
+      batch_out, bs_list_out, status_out);
+  return check_launch("llmem_select_method");
+}

@@ -1,0 +1,494 @@
+// Materialised event lists: per-configuration event counts and their exclusive
+// scan, the expansion kernel that writes every signed delta, and in-place page
+// rounding.  The expansion is bound by HBM writes (8 bytes per event): each CTA
+// builds a tile of deltas in shared memory and hands it to the TMA engine as one
+// bulk store, double-buffered so that filling the next tile overlaps the store.
+#include "llmem_host.h"
+#include "llmem_model.cuh"
+
+namespace llmem {
+
+// ---------------------------------------------------------------------------
+// event counts + exclusive scan
+// ---------------------------------------------------------------------------
+constexpr int kCountThreads = 256;
+constexpr int kCountItems = 4;
+constexpr int kCountBlock = kCountThreads * kCountItems;  // configurations per CTA
+
+__device__ __forceinline__ u64 warp_inclusive_scan(u64 v, int lane) {
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    u64 o = __shfl_up_sync(0xffffffffu, v, d);
+    if (lane >= d) v += o;
+  }
+  return v;
+}
+
+// Exclusive scan of one value per thread across a CTA of kCountThreads threads;
+// returns the exclusive prefix and the CTA total.
+__device__ __forceinline__ u64 block_exclusive_scan(u64 v, u64* total, u64* smem /* >= 9 */) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  u64 inc = warp_inclusive_scan(v, lane);
+  if (lane == 31) smem[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    u64 w = lane < (kCountThreads / 32) ? smem[lane] : 0;
+    u64 winc = warp_inclusive_scan(w, lane);
+    if (lane < (kCountThreads / 32)) smem[lane] = winc - w;
+    if (lane == (kCountThreads / 32) - 1) smem[kCountThreads / 32] = winc;
+  }
+  __syncthreads();
+  u64 r = smem[warp] + inc - v;
+  *total = smem[kCountThreads / 32];
+  __syncthreads();
+  return r;
+}
+
+// Pass 1: counts, CTA-local exclusive offsets, per-CTA totals.
+__global__ void __launch_bounds__(kCountThreads)
+count_kernel(const llmem_config* __restrict__ cfg, i64 n, i64* __restrict__ offsets,
+             uint8_t* __restrict__ status_out, u64* __restrict__ block_sums) {
+  __shared__ u64 smem[16];
+  const i64 base = (i64)blockIdx.x * kCountBlock + (i64)threadIdx.x * kCountItems;
+  u64 c[kCountItems];
+  u64 sum = 0;
+#pragma unroll
+  for (int j = 0; j < kCountItems; ++j) {
+    c[j] = 0;
+    const i64 i = base + j;
+    if (i < n) {
+      Cfg f = load_cfg(cfg + i);
+      int st = check_fields(f, true, true);
+      if (st == LLMEM_CFG_OK) {
+        Plan p = make_plan(f, f.method);
+        st = p.status;
+        if (st == LLMEM_CFG_OK) {
+          // the byte guard: the peak itself must stay below 2^62
+          StaticSums s = make_static_sums(p, f.pos_len > 0);
+          Dyn d = make_dyn(p, (u64)f.batch);
+          bool fw;
+          u64 rel = relative_peak(p, s, sat_add(s.gather, dyn_sum(p, d)), &fw);
+          if (sat_add(p.offset, rel) >= kSat) st = LLMEM_CFG_OVERFLOW;
+          else c[j] = p.count;
+        }
+      }
+      if (status_out) status_out[i] = (uint8_t)st;
+    }
+    sum += c[j];
+  }
+  u64 total;
+  u64 excl = block_exclusive_scan(sum, &total, smem);
+#pragma unroll
+  for (int j = 0; j < kCountItems; ++j) {
+    const i64 i = base + j;
+    if (i < n) offsets[i] = (i64)excl;
+    excl += c[j];
+  }
+  if (threadIdx.x == 0) block_sums[blockIdx.x] = total;
+}
+
+// Pass 2 (one CTA): exclusive scan of the per-CTA totals in place; the grand total
+// goes to block_sums[nblocks].
+__global__ void __launch_bounds__(kCountThreads)
+scan_block_sums_kernel(u64* __restrict__ block_sums, i64 nblocks) {
+  __shared__ u64 smem[16];
+  u64 carry = 0;
+  for (i64 base = 0; base < nblocks; base += kCountThreads) {
+    const i64 i = base + threadIdx.x;
+    u64 v = i < nblocks ? block_sums[i] : 0;
+    u64 total;
+    u64 excl = block_exclusive_scan(v, &total, smem);
+    if (i < nblocks) block_sums[i] = carry + excl;
+    carry += total;
+  }
+  if (threadIdx.x == 0) block_sums[nblocks] = carry;
+}
+
+// Pass 3: add each CTA's base; write offsets[n].
+__global__ void __launch_bounds__(256)
+add_block_base_kernel(i64* __restrict__ offsets, i64 n, const u64* __restrict__ block_sums, i64 nblocks) {
+  for (i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x; i <= n; i += (i64)gridDim.x * blockDim.x) {
+    if (i == n) offsets[n] = (i64)block_sums[nblocks];
+    else offsets[i] += (i64)block_sums[i / kCountBlock];
+  }
+}
+
+// ---------------------------------------------------------------------------
+// expansion
+// ---------------------------------------------------------------------------
+constexpr int kExpThreads = 256;
+// 18 events = 144 bytes = nine 16-byte words per thread: an odd word count makes
+// the per-thread spans fall on distinct shared-memory banks.
+constexpr int kExpPerThread = 18;
+constexpr int kExpTile = kExpThreads * kExpPerThread;  // 4608 events, 36 KiB
+constexpr int kDescBatch = 8;
+constexpr int kRuns = 17;
+
+// A run of events that repeat with a short period: the first `split` events of each
+// period have value a, the others b.  Constant runs use period 1.
+struct Run {
+  int cnt, period, split, pad;
+  i64 a, b;
+};
+
+// The event list of one configuration as runs.  Order: 0-1 initialisation,
+// 2-13 one iteration (allocations, then frees mirrored), 14-16 optimizer states,
+// which follow the first iteration only.
+struct SegDesc {
+  i64 gstart, gend;  // global event range of the segment
+  u32 init_n, dyn_n, os_n;
+  int invalid;
+  Run run[kRuns];
+};
+
+__device__ __forceinline__ void set_run(Run& r, int cnt, int period, int split, i64 a, i64 b) {
+  r.cnt = cnt; r.period = period; r.split = split; r.pad = 0; r.a = a; r.b = b;
+}
+
+__device__ void build_desc(SegDesc& d, const llmem_config* __restrict__ cfg, i64 gstart, i64 gend, bool round) {
+  d.gstart = gstart;
+  d.gend = gend;
+  d.invalid = 1;
+  d.init_n = d.dyn_n = d.os_n = 0;
+  if (gend <= gstart) return;
+  Cfg f = load_cfg(cfg);
+  if (check_fields(f, true, true) != LLMEM_CFG_OK) return;
+  Plan p = make_plan(f, f.method);
+  if (p.status != LLMEM_CFG_OK) return;
+  Dyn y = make_dyn(p, (u64)f.batch);
+  if (y.out >= kSat || y.logit >= kSat || y.shift >= kSat) return;
+  d.invalid = 0;
+#define LLMEM_V(x) ((i64)(round ? page_round(x) : (x)))
+  const int C = (int)p.C, L = p.L;
+  const int G = p.gather ? 1 : 0, T = p.tpback ? 1 : 0;
+  set_run(d.run[0], 2, 2, 1, LLMEM_V(p.p16_embed), LLMEM_V(p.p32_embed));
+  set_run(d.run[1], 2 * C, 2, 1, LLMEM_V(p.p16_chunk), LLMEM_V(p.p32_chunk));
+  const i64 ge = LLMEM_V(p.gat_embed), gc = LLMEM_V(p.gat_chunk), out = LLMEM_V(y.out);
+  const i64 lg = LLMEM_V(y.logit), sh = LLMEM_V(y.shift), bk = LLMEM_V(y.back);
+  set_run(d.run[2], G, 1, 1, ge, ge);
+  set_run(d.run[3], G * C, 1, 1, gc, gc);
+  set_run(d.run[4], p.e_n + L, 1, 1, out, out);
+  set_run(d.run[5], 1, 1, 1, lg, lg);
+  set_run(d.run[6], 2, 1, 1, sh, sh);
+  set_run(d.run[7], T * L, 1, 1, bk, bk);
+  set_run(d.run[8], T * L, 1, 1, -bk, -bk);
+  set_run(d.run[9], 2, 1, 1, -sh, -sh);
+  set_run(d.run[10], 1, 1, 1, -lg, -lg);
+  set_run(d.run[11], p.e_n + L, 1, 1, -out, -out);
+  set_run(d.run[12], G * C, 1, 1, -gc, -gc);
+  set_run(d.run[13], G, 1, 1, -ge, -ge);
+  const i64 ot = LLMEM_V(p.os_tok), op = LLMEM_V(p.os_pos);
+  set_run(d.run[14], 1, 1, 1, ot, ot);
+  set_run(d.run[15], f.pos_len > 0 ? 1 : 0, 1, 1, op, op);
+  set_run(d.run[16], p.K * L, p.K, 4, LLMEM_V(p.os_hh), LLMEM_V(p.os_hf));
+#undef LLMEM_V
+  d.init_n = 2u + 2u * (u32)C;
+  const u32 allocs = (u32)(G * (1 + C) + p.e_n + L + 3 + T * L);
+  d.dyn_n = 2 * allocs;
+  d.os_n = (u32)(p.e_n + p.K * L);
+}
+
+// Cursor of one thread inside a segment.
+struct Cursor {
+  int r, it, rem, phase, period, split;
+  i64 a, b;
+};
+
+__device__ __forceinline__ void enter_run(Cursor& c, const SegDesc& d, int r, int o) {
+  const Run& rn = d.run[r];
+  c.r = r;
+  c.rem = rn.cnt - o;
+  c.period = rn.period;
+  c.split = rn.split;
+  c.a = rn.a;
+  c.b = rn.b;
+  c.phase = rn.period == 1 ? 0 : (rn.period == 2 ? (o & 1) : (int)((u32)o % (u32)rn.period));
+}
+
+// Position the cursor on event `pos` (0-based inside the segment).
+__device__ __forceinline__ void seek(Cursor& c, const SegDesc& d, u32 pos) {
+  c.it = 1;
+  if (pos < d.init_n) {
+    if (pos < 2) enter_run(c, d, 0, (int)pos);
+    else enter_run(c, d, 1, (int)(pos - 2));
+    return;
+  }
+  u32 q = pos - d.init_n;
+  int r = 2;
+  if (q >= d.dyn_n) {
+    q -= d.dyn_n;
+    if (q < d.os_n) {
+      r = 14;
+    } else {
+      q -= d.os_n;
+      c.it = 2 + (int)(q / d.dyn_n);
+      q = q % d.dyn_n;
+    }
+  }
+  while (r < kRuns - 1 && q >= (u32)d.run[r].cnt) {
+    q -= (u32)d.run[r].cnt;
+    ++r;
+  }
+  enter_run(c, d, r, (int)q);
+}
+
+// Move to the next non-empty run.  After the frees of iteration 1 come the optimizer
+// states; after them, and after the frees of every later iteration, the next iteration.
+__device__ __forceinline__ void next_run(Cursor& c, const SegDesc& d) {
+  int r = c.r;
+  for (int guard = 0; guard < 2 * kRuns; ++guard) {
+    if (r == 13) {
+      if (c.it == 1) r = 14;
+      else { r = 2; ++c.it; }
+    } else if (r == 16) {
+      r = 2;
+      c.it = 2;
+    } else {
+      ++r;
+    }
+    if (d.run[r].cnt > 0) break;
+  }
+  enter_run(c, d, r, 0);
+}
+
+__device__ __forceinline__ i64 emit(Cursor& c, const SegDesc& d) {
+  const i64 v = c.phase < c.split ? c.a : c.b;
+  if (++c.phase == c.period) c.phase = 0;
+  if (--c.rem == 0) next_run(c, d);
+  return v;
+}
+
+__device__ __forceinline__ u32 smem_addr(const void* p) { return (u32)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void bulk_store(void* gdst, const void* ssrc, u32 bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;\n" ::"l"(gdst),
+               "r"(smem_addr(ssrc)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;\n" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
+
+// smallest s in [lo, n] with offsets[s + 1] > pos (n if none)
+__device__ i64 first_segment_after(const i64* __restrict__ offsets, i64 n, i64 pos) {
+  i64 lo = 0, hi = n;
+  while (lo < hi) {
+    i64 mid = lo + (hi - lo) / 2;
+    if (__ldg(offsets + mid + 1) > pos) hi = mid;
+    else lo = mid + 1;
+  }
+  return lo;
+}
+
+struct ExpandSmem {
+  alignas(128) i64 tile[2][kExpTile];
+  SegDesc desc[kDescBatch];
+  i64 tag[kDescBatch];
+  i64 seg0;
+};
+
+__global__ void __launch_bounds__(kExpThreads)
+expand_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict__ offsets, i64 total,
+              i64* __restrict__ out, i64 tiles_per_cta, int round, int bulk_ok) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  ExpandSmem& sm = *reinterpret_cast<ExpandSmem*>(smem_raw);
+  const int tid = threadIdx.x;
+  const i64 ntiles = (total + kExpTile - 1) / kExpTile;
+  const i64 tile_lo = (i64)blockIdx.x * tiles_per_cta;
+  const i64 tile_hi = tile_lo + tiles_per_cta < ntiles ? tile_lo + tiles_per_cta : ntiles;
+  if (tile_lo >= tile_hi) return;
+
+  if (tid < kDescBatch) sm.tag[tid] = -1;
+  if (tid == 0) sm.seg0 = first_segment_after(offsets, n, tile_lo * kExpTile);
+  __syncthreads();
+  i64 seg = sm.seg0;  // smallest segment index whose end lies beyond the current position
+
+  int parity = 0;
+  for (i64 tile = tile_lo; tile < tile_hi; ++tile, parity ^= 1) {
+    const i64 tb = tile * kExpTile;
+    const i64 te = tb + kExpTile < total ? tb + kExpTile : total;
+    i64* buf = sm.tile[parity];
+    // the bulk store issued from this buffer two tiles ago must have read it
+    if (tid == 0) bulk_wait_read<1>();
+    __syncthreads();
+    const i64 span_lo = tb + (i64)tid * kExpPerThread;
+    const i64 span_hi = span_lo + kExpPerThread < te ? span_lo + kExpPerThread : te;
+    i64 pos = tb;
+    while (pos < te) {
+      // descriptors of the next kDescBatch segments that begin before the tile ends
+      if (tid < kDescBatch) {
+        const i64 s = seg + tid;
+        i64 gs = INT64_MAX, ge = INT64_MAX;
+        if (s < n) {
+          gs = __ldg(offsets + s);
+          ge = __ldg(offsets + s + 1);
+        }
+        if (s < n && gs < te) {
+          if (sm.tag[tid] != s) {
+            build_desc(sm.desc[tid], cfg + s, gs, ge, round != 0);
+            sm.tag[tid] = s;
+          }
+        } else {
+          sm.desc[tid].gstart = INT64_MAX;
+          sm.desc[tid].gend = INT64_MAX;
+          sm.tag[tid] = -1;
+        }
+      }
+      __syncthreads();
+      int nb = 0;
+      while (nb < kDescBatch && sm.desc[nb].gstart != INT64_MAX) ++nb;
+      if (nb == 0) {
+        // offsets do not cover the rest of the tile: define it as zeros
+        for (i64 e = (span_lo > pos ? span_lo : pos); e < span_hi; ++e) buf[e - tb] = 0;
+        pos = te;
+        __syncthreads();
+        break;
+      }
+      const i64 last_end = sm.desc[nb - 1].gend;
+      const i64 batch_end = last_end < te ? last_end : te;
+      i64 e = span_lo > pos ? span_lo : pos;
+      const i64 e_end = span_hi < batch_end ? span_hi : batch_end;
+      if (e < e_end) {
+        int di = 0;
+        while (di + 1 < nb && sm.desc[di + 1].gstart <= e) ++di;
+        while (di + 1 < nb && sm.desc[di].gend <= e) ++di;
+        Cursor c;
+        bool inval = sm.desc[di].invalid != 0;
+        if (!inval) seek(c, sm.desc[di], (u32)(e - sm.desc[di].gstart));
+        for (; e < e_end; ++e) {
+          if (e >= sm.desc[di].gend) {
+            do { ++di; } while (di + 1 < nb && sm.desc[di].gend <= e);
+            inval = sm.desc[di].invalid != 0;
+            if (!inval) seek(c, sm.desc[di], (u32)(e - sm.desc[di].gstart));
+          }
+          buf[e - tb] = inval ? 0 : emit(c, sm.desc[di]);
+        }
+      }
+      pos = batch_end;
+      seg += (last_end <= te) ? nb : nb - 1;
+      __syncthreads();  // descriptors are rebuilt by the next round
+    }
+    // hand the tile to the TMA engine (generic-proxy writes -> async-proxy read)
+    const u32 cnt = (u32)(te - tb);
+    if (bulk_ok) {
+      fence_async_shared();
+      __syncthreads();
+      if (tid == 0) {
+        const u32 even = cnt & ~1u;
+        if (even) bulk_store(out + tb, buf, even * 8u);
+        bulk_commit();
+        if (cnt & 1u) out[tb + cnt - 1] = buf[cnt - 1];
+      }
+    } else {
+      __syncthreads();
+      for (u32 i = tid; i < cnt; i += kExpThreads) out[tb + i] = buf[i];
+    }
+  }
+  if (tid == 0) bulk_wait_read<0>();
+}
+
+// ---------------------------------------------------------------------------
+// rounding in place
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+round_kernel(i64* __restrict__ delta, i64 total) {
+  // 16-byte vectors over the aligned middle, scalars for a ragged first / last element
+  const i64 head = ((reinterpret_cast<uintptr_t>(delta) & 15) != 0 && total > 0) ? 1 : 0;
+  const i64 nvec = (total - head) / 2;
+  longlong2* v = reinterpret_cast<longlong2*>(delta + head);
+  const i64 stride = (i64)gridDim.x * blockDim.x;
+  const i64 t0 = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+  for (i64 i = t0; i < nvec; i += stride) {
+    longlong2 x = v[i];
+    x.x = page_round_signed(x.x);
+    x.y = page_round_signed(x.y);
+    v[i] = x;
+  }
+  if (t0 == 0) {
+    if (head) delta[0] = page_round_signed(delta[0]);
+    const i64 tail = head + 2 * nvec;
+    if (tail < total) delta[tail] = page_round_signed(delta[tail]);
+  }
+}
+
+}  // namespace llmem
+
+using namespace llmem;
+
+extern "C" llmem_status llmem_event_counts(const llmem_config* cfg, int64_t n, int64_t* offsets_out,
+                                           uint8_t* status_out, void* scratch, size_t scratch_bytes,
+                                           uint32_t flags, void* cuda_stream) {
+  (void)flags;
+  clear_error();
+  if (n < 0) { set_error("llmem_event_counts: n < 0"); return LLMEM_ERR_ARG; }
+  if (!offsets_out || !aligned_to(offsets_out, 8)) { set_error("llmem_event_counts: offsets_out is required"); return LLMEM_ERR_ARG; }
+  if (n > 0 && (!cfg || !aligned_to(cfg, 16))) { set_error("llmem_event_counts: cfg must be a 16-byte aligned device pointer"); return LLMEM_ERR_ARG; }
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (n == 0) {
+    if (cudaMemsetAsync(offsets_out, 0, sizeof(int64_t), s) != cudaSuccess) return check_launch("llmem_event_counts");
+    return LLMEM_OK;
+  }
+  if (!scratch || !aligned_to(scratch, 256) ||
+      scratch_bytes < llmem_scratch_bytes(LLMEM_OP_EVENT_COUNTS, n, 0)) {
+    set_error("llmem_event_counts: scratch missing, misaligned or smaller than llmem_scratch_bytes()");
+    return LLMEM_ERR_SCRATCH;
+  }
+  u64* block_sums = reinterpret_cast<u64*>(static_cast<unsigned char*>(scratch) + kScratchHeader);
+  const i64 nblocks = (n + kCountBlock - 1) / kCountBlock;
+  count_kernel<<<(unsigned)nblocks, kCountThreads, 0, s>>>(cfg, n, reinterpret_cast<i64*>(offsets_out), status_out, block_sums);
+  scan_block_sums_kernel<<<1, kCountThreads, 0, s>>>(block_sums, nblocks);
+  i64 blocks3 = (n + 1 + 255) / 256;
+  const i64 cap3 = (i64)sm_count() * 8;
+  if (blocks3 > cap3) blocks3 = cap3;
+  add_block_base_kernel<<<(unsigned)blocks3, 256, 0, s>>>(reinterpret_cast<i64*>(offsets_out), n, block_sums, nblocks);
+  return check_launch("llmem_event_counts");
+}
+
+extern "C" llmem_status llmem_expand_events(const llmem_config* cfg, int64_t n, const int64_t* offsets,
+                                            int64_t total_events, int64_t* delta_out, void* scratch,
+                                            size_t scratch_bytes, uint32_t flags, void* cuda_stream) {
+  (void)scratch; (void)scratch_bytes;
+  clear_error();
+  if (n < 0 || total_events < 0) { set_error("llmem_expand_events: negative size"); return LLMEM_ERR_ARG; }
+  if (total_events == 0) return LLMEM_OK;
+  if (!cfg || !offsets || !delta_out) { set_error("llmem_expand_events: cfg, offsets and delta_out are required"); return LLMEM_ERR_ARG; }
+  if (!aligned_to(cfg, 16) || !aligned_to(offsets, 8) || !aligned_to(delta_out, 8)) {
+    set_error("llmem_expand_events: misaligned pointer");
+    return LLMEM_ERR_ARG;
+  }
+  static thread_local int configured_dev = -1;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (configured_dev != dev) {
+    if (cudaFuncSetAttribute(expand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ExpandSmem)) != cudaSuccess)
+      return check_launch("llmem_expand_events (shared memory opt-in)");
+    configured_dev = dev;
+  }
+  const i64 ntiles = (total_events + kExpTile - 1) / kExpTile;
+  i64 grid = (i64)sm_count() * 2;
+  if (grid > ntiles) grid = ntiles;
+  const i64 tiles_per_cta = (ntiles + grid - 1) / grid;
+  grid = (ntiles + tiles_per_cta - 1) / tiles_per_cta;
+  expand_kernel<<<(unsigned)grid, kExpThreads, sizeof(ExpandSmem), static_cast<cudaStream_t>(cuda_stream)>>>(
+      cfg, n, reinterpret_cast<const i64*>(offsets), total_events, reinterpret_cast<i64*>(delta_out),
+      tiles_per_cta, (flags & LLMEM_FUSE_ROUND) ? 1 : 0, aligned_to(delta_out, 16) ? 1 : 0);
+  return check_launch("llmem_expand_events");
+}
+
+extern "C" llmem_status llmem_round_events(int64_t* delta, int64_t total_events, void* scratch,
+                                           size_t scratch_bytes, uint32_t flags, void* cuda_stream) {
+  (void)scratch; (void)scratch_bytes; (void)flags;
+  clear_error();
+  if (total_events < 0) { set_error("llmem_round_events: negative size"); return LLMEM_ERR_ARG; }
+  if (total_events == 0) return LLMEM_OK;
+  if (!delta || !aligned_to(delta, 8)) { set_error("llmem_round_events: delta must be an 8-byte aligned device pointer"); return LLMEM_ERR_ARG; }
+  i64 blocks = (total_events / 2 + 255) / 256;
+  const i64 cap = (i64)sm_count() * 16;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  round_kernel<<<(unsigned)blocks, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(reinterpret_cast<i64*>(delta), total_events);
+  return check_launch("llmem_round_events");
+}

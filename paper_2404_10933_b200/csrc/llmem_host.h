@@ -1,0 +1,31 @@
+// Host-side helpers shared by the translation units of the library: error text,
+// argument checks, launch geometry.
+#pragma once
+
+#include <cstdarg>
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "../../include/llmem.h"
+
+namespace llmem {
+
+// Records the text returned by llmem_last_error() for the calling thread.
+void set_error(const char* fmt, ...);
+void clear_error();
+
+inline bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// Number of SMs of the current device (cached per thread; 148 on B200).
+int sm_count();
+
+// Returns LLMEM_ERR_CUDA and records the text if the last launch failed.
+llmem_status check_launch(const char* what);
+
+// Layout of the scratch buffer used by llmem_scan_peak and llmem_event_counts:
+// a 256-byte header whose first word is the device status, then the payload.
+constexpr size_t kScratchHeader = 256;
+constexpr int kMaxScanCtas = 1024;  // upper bound on the persistent grid of the scan
+
+}  // namespace llmem

@@ -1,0 +1,254 @@
+// Device-side memory model shared by every kernel of the library: configuration
+// checks, parameter inventory (Table 1 of the paper), raw event sizes per method
+// (Sections 4.1, 4.2 and 5) and the per-phase sums used by the fused kernels.
+//
+// All arithmetic is unsigned 64-bit and saturates at 2^62: every quantity is a
+// sum or product of non-negative terms, so "the exact value is >= 2^62" and "the
+// saturating value is 2^62" are the same statement, which is how the overflow
+// status is decided without wider integers.
+#pragma once
+
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "../../include/llmem.h"
+
+namespace llmem {
+
+typedef unsigned long long u64;
+typedef long long i64;
+typedef unsigned int u32;
+
+constexpr u64 kPage = 2ull * 1024ull * 1024ull;  // cu_p, Section 4.2
+constexpr u64 kSat = 1ull << 62;                 // bytes limit (exclusive)
+constexpr u64 kCountLimit = 1ull << 31;          // events limit (exclusive)
+
+__host__ __device__ __forceinline__ u64 sat_add(u64 a, u64 b) {
+  u64 s = a + b;  // a, b <= 2^62: no wrap
+  return s > kSat ? kSat : s;
+}
+
+__device__ __forceinline__ u64 sat_mul(u64 a, u64 b) {
+  u64 hi = __umul64hi(a, b);
+  u64 lo = a * b;
+  return (hi != 0 || lo >= kSat) ? kSat : lo;
+}
+
+// ceil(x / cu_p) * cu_p; x <= 2^62 keeps the result <= 2^62
+__host__ __device__ __forceinline__ u64 page_round(u64 x) { return (x + (kPage - 1)) & ~(kPage - 1); }
+
+// signed variant: the magnitude is rounded, the sign kept
+__host__ __device__ __forceinline__ i64 page_round_signed(i64 d) {
+  u64 mag = d < 0 ? (u64)0 - (u64)d : (u64)d;
+  u64 r = (mag + (kPage - 1)) & ~(kPage - 1);
+  return d < 0 ? (i64)((u64)0 - r) : (i64)r;
+}
+
+__device__ __forceinline__ u64 ceil_div(u64 a, u64 b) { return (a + b - 1) / b; }
+
+// A configuration record loaded into registers (four 16-byte loads).
+struct Cfg {
+  int layers, hidden, heads, ffn, vocab, pos_len, seq, batch;
+  i64 chunk_elems, base_bytes;
+  u32 method, gpu_n, tp_n, lm_bytes, ffn_kind, has_bias, iters;
+  bool reserved_zero;
+};
+
+__device__ __forceinline__ Cfg load_cfg(const llmem_config* __restrict__ p) {
+  const int4* q = reinterpret_cast<const int4*>(p);
+  int4 a = __ldg(q), b = __ldg(q + 1), c = __ldg(q + 2), d = __ldg(q + 3);
+  Cfg f;
+  f.layers = a.x; f.hidden = a.y; f.heads = a.z; f.ffn = a.w;
+  f.vocab = b.x; f.pos_len = b.y; f.seq = b.z; f.batch = b.w;
+  f.chunk_elems = (i64)(((u64)(u32)c.y << 32) | (u32)c.x);
+  f.base_bytes = (i64)(((u64)(u32)c.w << 32) | (u32)c.z);
+  u32 w0 = (u32)d.x, w1 = (u32)d.y;
+  f.method = w0 & 0xff; f.gpu_n = (w0 >> 8) & 0xff; f.tp_n = (w0 >> 16) & 0xff; f.lm_bytes = w0 >> 24;
+  f.ffn_kind = w1 & 0xff; f.has_bias = (w1 >> 8) & 0xff; f.iters = (w1 >> 16) & 0xff;
+  f.reserved_zero = ((w1 >> 24) == 0) && d.z == 0 && d.w == 0;
+  return f;
+}
+
+// Field ranges (status 1).  `check_batch` is false for the search entry points,
+// which choose the batch themselves; `check_method` is false for selection.
+__device__ __forceinline__ int check_fields(const Cfg& f, bool check_batch, bool check_method) {
+  bool ok = f.layers >= 1 && f.layers <= (1 << 16) && f.hidden >= 1 && f.hidden <= (1 << 20) &&
+            f.heads >= 1 && f.ffn >= 1 && f.ffn <= (1 << 22) && f.vocab >= 1 &&
+            f.vocab <= (1 << 26) && f.pos_len >= 0 && f.pos_len <= (1 << 26) && f.seq >= 1 &&
+            f.seq <= (1 << 26) && f.chunk_elems >= 1 && f.chunk_elems <= (1ll << 40) &&
+            f.base_bytes >= 0 && f.base_bytes <= (1ll << 60) && f.gpu_n >= 1 &&
+            (f.lm_bytes == 2 || f.lm_bytes == 4) && f.ffn_kind <= 1 && f.has_bias <= 1 &&
+            f.iters >= 1 && f.reserved_zero;
+  if (ok) ok = (f.hidden % f.heads) == 0;
+  if (ok && check_batch) ok = f.batch >= 1 && f.batch <= (1 << 26);
+  if (ok && check_method) ok = f.method <= 3;
+  return ok ? LLMEM_CFG_OK : LLMEM_CFG_FIELD;
+}
+
+// Section 5, DP+TP: needs both a DP and a TP dimension (status 2 otherwise).
+__device__ __forceinline__ int check_combo(u32 method, u32 gpu_n, u32 tp_n) {
+  if (method == LLMEM_METHOD_DPTP && (tp_n < 2 || 2 * tp_n > gpu_n || gpu_n % tp_n != 0))
+    return LLMEM_CFG_COMBO;
+  return LLMEM_CFG_OK;
+}
+
+// Everything that does not depend on the batch size.
+struct Plan {
+  int status;
+  int e_n;        // Embedding operators: token, + learned position
+  int K;          // Linear operators per layer (q,k,v,o + 2 or 3 feed-forward matrices)
+  int gather;     // phase 2 present: ADP, DP+TP
+  int tpback;     // phase 4 present: TP, DP+TP
+  int L, iters;
+  u32 tp;         // TP degree of the backward buffers: gpu_n for TP, tp_n for DP+TP
+  u32 C;          // chunks = ceil(other_p / cs); < 2^31 when status == 0
+  u64 count;      // number of events
+  u64 offset;     // m_base + lm_p (added unrounded, Section 4.2)
+  // raw byte sizes of the batch-independent event kinds
+  u64 p16_embed, p32_embed, p16_chunk, p32_chunk, gat_embed, gat_chunk;
+  u64 os_tok, os_pos, os_hh, os_hf;
+  // per-sample factors of the batch-dependent kinds: out = batch * out1, ...
+  u64 out1, logit1, shift1;
+};
+
+__device__ __forceinline__ u64 shard_bytes(u64 bytes, u32 method, u32 n) {
+  return method == LLMEM_METHOD_CDP ? bytes : ceil_div(bytes, n);
+}
+
+// fp16 bytes of a unit of x elements that exist only while computing:
+// ADP holds the whole of param fp16 (m_p,16 undivided in m_peak^dp);
+// DP+TP holds m_p,16 * (1 - tp_n/gpu_n) (m_peak^dp+tp).
+__device__ __forceinline__ u64 gathered_bytes(u64 x, u32 method, u32 n, u32 t) {
+  u64 whole = 2 * x;
+  u64 kept = ceil_div(whole, n);
+  if (method == LLMEM_METHOD_ADP) return whole - kept;
+  if (method == LLMEM_METHOD_DPTP) return whole - (whole * t) / n - kept;
+  return 0;
+}
+
+// a1: parameter inventory and event sizes.  `f` has passed check_fields.
+__device__ __forceinline__ Plan make_plan(const Cfg& f, u32 method) {
+  Plan p;
+  p.status = check_combo(method, f.gpu_n, f.tp_n);
+  const u64 H = (u64)f.hidden, F = (u64)f.ffn, V = (u64)f.vocab, P = (u64)f.pos_len;
+  const u64 bias = f.has_bias, n = f.gpu_n;
+  p.e_n = 1 + (f.pos_len > 0);
+  p.K = f.ffn_kind ? 7 : 6;
+  p.gather = (method == LLMEM_METHOD_ADP || method == LLMEM_METHOD_DPTP);
+  p.tpback = (method == LLMEM_METHOD_TP || method == LLMEM_METHOD_DPTP);
+  p.tp = method == LLMEM_METHOD_TP ? f.gpu_n : f.tp_n;
+  if (p.tp == 0) p.tp = 1;  // only reachable with status 2; keeps divisions defined
+  p.L = f.layers;
+  p.iters = (int)f.iters;
+  const u64 tok_p = V * H, pos_p = P * H, hh_p = H * H, hf_p = H * F;
+  const u64 embed_p = tok_p + pos_p;                       // <= 2^47
+  const u64 nffn = (u64)(p.K - 4);
+  const u64 bias_p = bias * (4 * H + (nffn - 1) * F + H);
+  const u64 norm_p = 2 * H * (1 + bias);
+  const u64 other_p = (u64)p.L * (4 * hh_p + nffn * hf_p + bias_p + norm_p) + H * (1 + bias);  // < 2^61
+  const u64 cs = (u64)f.chunk_elems;
+  const u64 chunks = ceil_div(other_p, cs);
+  p.offset = (u64)f.base_bytes + tok_p * (u64)f.lm_bytes;  // < 2^60 + 2^49
+  p.p16_embed = shard_bytes(2 * embed_p, method, f.gpu_n);
+  p.p32_embed = shard_bytes(4 * embed_p, method, f.gpu_n);
+  p.p16_chunk = shard_bytes(2 * cs, method, f.gpu_n);
+  p.p32_chunk = shard_bytes(4 * cs, method, f.gpu_n);
+  p.gat_embed = gathered_bytes(embed_p, method, f.gpu_n, p.tp);
+  p.gat_chunk = gathered_bytes(cs, method, f.gpu_n, p.tp);
+  p.os_tok = shard_bytes(8 * tok_p, method, f.gpu_n);
+  p.os_pos = shard_bytes(8 * pos_p, method, f.gpu_n);
+  p.os_hh = shard_bytes(8 * hh_p, method, f.gpu_n);
+  p.os_hf = shard_bytes(8 * hf_p, method, f.gpu_n);
+  p.out1 = 2 * (u64)f.seq * H;                              // <= 2^47
+  p.logit1 = (u64)f.lm_bytes * (u64)f.seq * V;              // <= 2^54
+  p.shift1 = (u64)f.lm_bytes * (u64)(f.seq - 1) * V;
+  (void)n;
+  if (chunks >= kCountLimit) {
+    p.C = 0;
+    p.count = kCountLimit;
+    if (p.status == LLMEM_CFG_OK) p.status = LLMEM_CFG_OVERFLOW;
+  } else {
+    p.C = (u32)chunks;
+    const u64 allocs = (p.gather ? 1 + chunks : 0) + (u64)p.e_n + (u64)p.L + 3 +
+                       (p.tpback ? (u64)p.L : 0);
+    p.count = 2 + 2 * chunks + (u64)p.e_n + (u64)p.K * (u64)p.L + (u64)p.iters * 2 * allocs;
+    if (p.count >= kCountLimit && p.status == LLMEM_CFG_OK) p.status = LLMEM_CFG_OVERFLOW;
+  }
+  return p;
+}
+
+// Batch-dependent raw sizes (saturating).
+struct Dyn {
+  u64 out, logit, shift, back;
+};
+
+__device__ __forceinline__ Dyn make_dyn(const Plan& p, u64 batch) {
+  Dyn d;
+  d.out = sat_mul(batch, p.out1);
+  d.logit = sat_mul(batch, p.logit1);
+  d.shift = sat_mul(batch, p.shift1);
+  // ceil(out * (tp-1) / tp) = out - floor(out / tp)   (m_back^tp, one layer's share)
+  d.back = p.tpback ? d.out - d.out / p.tp : 0;
+  return d;
+}
+
+// Batch-independent sums of rounded events.
+struct StaticSums {
+  u64 init, gather, os;
+};
+
+__device__ __forceinline__ StaticSums make_static_sums(const Plan& p, bool has_pos) {
+  StaticSums s;
+  s.init = sat_add(sat_add(page_round(p.p16_embed), page_round(p.p32_embed)),
+                   sat_mul(p.C, page_round(p.p16_chunk) + page_round(p.p32_chunk)));
+  s.gather = p.gather ? sat_add(page_round(p.gat_embed), sat_mul(p.C, page_round(p.gat_chunk))) : 0;
+  const u64 per_layer = 4 * page_round(p.os_hh) + (u64)(p.K - 4) * page_round(p.os_hf);  // < 2^48
+  s.os = sat_add(page_round(p.os_tok) + (has_pos ? page_round(p.os_pos) : 0),
+                 sat_mul((u64)p.L, per_layer));
+  return s;
+}
+
+// Sum of the rounded batch-dependent allocations of one iteration (phases 3 and 4).
+__device__ __forceinline__ u64 dyn_sum(const Plan& p, const Dyn& d) {
+  u64 s = sat_mul((u64)(p.e_n + p.L), page_round(d.out));
+  s = sat_add(s, page_round(d.logit));
+  s = sat_add(s, sat_mul(2, page_round(d.shift)));
+  if (p.tpback) s = sat_add(s, sat_mul((u64)p.L, page_round(d.back)));
+  return s;
+}
+
+// Largest prefix sum (without the offset) given the phase sums.  Iteration 1
+// peaks before the optimizer states exist; they are allocated after its frees and
+// stay; every later iteration peaks on top of them.
+__device__ __forceinline__ u64 relative_peak(const Plan& p, const StaticSums& s, u64 dyn_total,
+                                             bool* first_iteration_wins) {
+  const u64 first = sat_add(s.init, dyn_total);
+  const u64 after = sat_add(s.init, s.os);
+  const u64 later = sat_add(after, dyn_total);
+  if (p.iters >= 2) {
+    *first_iteration_wins = false;
+    return later;
+  }
+  *first_iteration_wins = first >= after;
+  return first >= after ? first : after;
+}
+
+// Complete admissibility check of a configuration for estimation: field ranges,
+// method / degree combination, event-count limit and byte limit.  On LLMEM_CFG_OK
+// *plan_out holds the plan and *peak_out the peak (offset included).
+__device__ __forceinline__ int full_status(const Cfg& f, Plan* plan_out, u64* peak_out) {
+  int st = check_fields(f, true, true);
+  if (st != LLMEM_CFG_OK) return st;
+  *plan_out = make_plan(f, f.method);
+  if (plan_out->status != LLMEM_CFG_OK) return plan_out->status;
+  StaticSums s = make_static_sums(*plan_out, f.pos_len > 0);
+  Dyn d = make_dyn(*plan_out, (u64)f.batch);
+  bool fw;
+  u64 rel = relative_peak(*plan_out, s, sat_add(s.gather, dyn_sum(*plan_out, d)), &fw);
+  u64 total = sat_add(plan_out->offset, rel);
+  if (total >= kSat) return LLMEM_CFG_OVERFLOW;
+  *peak_out = total;
+  return LLMEM_CFG_OK;
+}
+
+}  // namespace llmem

@@ -1,0 +1,114 @@
+"""CPU-side checks: the C-ABI library loads and exports what the header declares,
+the input generators are deterministic and well-formed, and argument errors are
+reported by return code without touching a GPU."""
+import ctypes
+import os
+import re
+
+import numpy as np
+
+import paper_2404_10933_b200 as llmem
+from paper_2404_10933_b200 import grids
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "llmem.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(llmem_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_2404_10933_b200 import _build
+    _build.build()
+    L = llmem.lib()
+    names = declared_symbols()
+    assert len(names) >= 11
+    for name in names:
+        assert hasattr(L, name), name
+    assert sorted(llmem.EXPORTS) == names
+    assert L.llmem_version() >= 100
+
+
+def test_scratch_bytes_and_argument_errors_need_no_gpu():
+    L = llmem.lib()
+    assert L.llmem_scratch_bytes(llmem.OP_ESTIMATE, 1000, 0) == 0
+    assert L.llmem_scratch_bytes(llmem.OP_EXPAND, 1000, 10 ** 9) == 0
+    assert L.llmem_scratch_bytes(llmem.OP_EVENT_COUNTS, 5000, 0) >= 256 + 8 * 6
+    assert L.llmem_scratch_bytes(llmem.OP_SCAN_PEAK, 5000, 10 ** 9) >= 256 + 64
+    # call-level errors are detected before any CUDA call
+    assert L.llmem_estimate_batch(None, -1, None, None, None, None, 0, 0, None) == llmem.ERR_ARG
+    assert b"n < 0" in L.llmem_last_error()
+    assert L.llmem_estimate_batch(None, 5, None, None, None, None, 0, 0, None) == llmem.ERR_ARG
+    assert L.llmem_max_batch(ctypes.c_void_p(16), 5, ctypes.c_void_p(16), 1, 0, ctypes.c_void_p(16),
+                             None, None, 0, 0, None) == llmem.ERR_ARG          # bmax < 1
+    assert L.llmem_estimate_batch(ctypes.c_void_p(8), 5, ctypes.c_void_p(16), None, None, None, 0, 0,
+                                  None) == llmem.ERR_ARG                        # cfg misaligned
+    assert L.llmem_scan_peak(ctypes.c_void_p(16), ctypes.c_void_p(16), 5, 10, None, ctypes.c_void_p(16),
+                             None, None, 0, 0, None) == llmem.ERR_SCRATCH
+    assert L.llmem_event_counts(ctypes.c_void_p(16), 5, ctypes.c_void_p(16), None, ctypes.c_void_p(256), 8,
+                                0, None) == llmem.ERR_SCRATCH
+    # empty calls succeed
+    assert L.llmem_estimate_batch(None, 0, None, None, None, None, 0, 0, None) == llmem.OK
+    assert L.llmem_round_events(None, 0, None, 0, 0, None) == llmem.OK
+    assert L.llmem_last_error() == b""
+
+
+def test_record_layout_matches_header():
+    text = open(os.path.join(ROOT, "include", "llmem.h")).read()
+    body = text[text.index("typedef struct __attribute__((aligned(16))) llmem_config {"):text.index("} llmem_config;")]
+    fields = re.findall(r"^\s*(int32_t|int64_t|uint8_t)\s+(\w+)(\[\d+\])?;", body, flags=re.M)
+    assert [f[1] for f in fields] == list(grids.CONFIG_DTYPE.names)
+    size = {"int32_t": 4, "int64_t": 8, "uint8_t": 1}
+    off = 0
+    for ctype, name, arr in fields:
+        assert grids.CONFIG_DTYPE.fields[name][1] == off, name
+        off += size[ctype] * (int(arr[1:-1]) if arr else 1)
+    assert off == 64 == grids.CONFIG_DTYPE.itemsize
+
+
+def test_grids_are_deterministic_and_sliceable():
+    a = grids.g3_sweep(1000, 50)
+    b = grids.g3_sweep(0, 2000)[1000:1050]
+    assert a.tobytes() == b.tobytes()
+    assert grids.g5_stress(10, 5).tobytes() == grids.g5_stress(0, 20)[10:15].tobytes()
+    assert grids.g5_stress(0, 8, seed_offset=1).tobytes() != grids.g5_stress(0, 8).tobytes()
+
+
+def test_grid_shapes_and_ranges():
+    g1 = grids.g1_small()
+    assert len(g1) == 64 and g1["batch"].tolist() == list(range(1, 65))
+    combos = grids.g2_combos()
+    assert len(combos) == 29
+    assert [(n, t) for m, n, t in combos if m == 3] == [(4, 2), (6, 2), (6, 3), (8, 2), (8, 4)]
+    g2 = grids.g2_shape_grid(0, 3)
+    assert len(g2) == 3 * 32 * 29
+    assert set(np.unique(g2["hidden"]) % 256) == {0}
+    assert g2["layers"].min() >= 4 and g2["layers"].max() <= 48
+    assert ((g2["hidden"] % g2["heads"]) == 0).all()
+    g3 = grids.g3_sweep(0, 20000)
+    assert g3["gpu_n"].min() == 1 and g3["gpu_n"].max() == 16
+    assert set(np.unique(g3["seq"])) == {128, 256, 512, 1024, 2048, 4096}
+    dptp = g3[g3["method"] == 3]
+    assert len(dptp) > 0
+    assert ((dptp["gpu_n"] % dptp["tp_n"]) == 0).all() and (dptp["tp_n"] >= 2).all()
+    assert (2 * dptp["tp_n"].astype(int) <= dptp["gpu_n"]).all()
+    assert set(np.unique(g3["method"])) == {0, 1, 2, 3}
+    g4 = grids.g4_search_grid(0, 2)
+    assert len(g4) == 2 * 64
+    g4s = grids.g4_select_grid(0, 2)
+    assert len(g4s) == 2 * 16 and g4s["tp_n"][:16].tolist() == [0, 0, 0, 2, 0, 2, 0, 2, 3, 2, 0, 2, 0, 2, 3, 2]
+    g5 = grids.g5_stress(0, 1000)
+    assert g5["layers"].min() >= 64 and g5["hidden"].min() >= 8192 and (g5["chunk_elems"] == 1 << 23).all()
+    assert grids.g4_capacities().tolist() == [g << 30 for g in (16, 24, 40, 48, 80, 96, 141, 180, 192)]
+
+
+def test_shard_bounds_balance_weights():
+    w = np.array([5, 1, 1, 1, 1, 1, 5, 5], dtype=np.int64)
+    b = grids.shard_bounds(w, 2)
+    assert b[0] == 0 and b[-1] == len(w) and (np.diff(b) >= 0).all()
+    left = w[b[0]:b[1]].sum()
+    assert abs(left - w.sum() / 2) <= w.max()
+    assert grids.shard_bounds(w, 1).tolist() == [0, 8]
+    assert grids.shard_bounds(np.ones(3), 8)[-1] == 3

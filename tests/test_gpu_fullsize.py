@@ -1,0 +1,139 @@
+"""Parity at the full sizes of the five configuration grids, in the launch
+configuration the benchmark times.  Where the level-1 oracle (explicit event list)
+would take too long for every element, all elements are compared with the oracle's
+level-2 evaluation (shown equal to level 1 by the CPU pins) and a seeded sample is
+compared with level 1, including event-list slices and peak positions."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2404_10933_b200 import grids
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+THREADS = 16
+
+
+@pytest.fixture(scope="module")
+def llmem():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    import paper_2404_10933_b200 as m
+    m.lib()
+    return m
+
+
+def sample_indices(n, k, seed):
+    return np.sort(np.random.default_rng(seed).choice(n, size=min(k, n), replace=False))
+
+
+def test_g2_shape_grid_full(llmem):
+    cfgs = grids.g2_shape_grid()
+    assert len(cfgs) == 4096 * 32 * 29
+    got = llmem.estimate_batch(cfgs)
+    want2 = oracle.estimate(cfgs, level=2, threads=THREADS)
+    assert np.array_equal(got["status"].cpu().numpy(), want2["status"])
+    peak = got["peak"].cpu().numpy()
+    assert np.array_equal(peak, want2["peak"])
+    idx = sample_indices(len(cfgs), 1500, 2)
+    want1 = oracle.estimate(cfgs[idx], level=1, threads=THREADS)
+    assert np.array_equal(peak[idx], want1["peak"])
+    assert np.array_equal(got["index"].cpu().numpy()[idx], want1["index"])
+
+
+def test_g3_large_sweep_full(llmem):
+    cfgs = grids.g3_sweep()
+    assert len(cfgs) == 1 << 20
+    got = llmem.estimate_batch(cfgs)
+    want2 = oracle.estimate(cfgs, level=2, threads=THREADS)
+    peak = got["peak"].cpu().numpy()
+    assert (want2["status"] == 0).all()
+    assert np.array_equal(got["status"].cpu().numpy(), want2["status"])
+    assert np.array_equal(peak, want2["peak"])
+    idx = sample_indices(len(cfgs), 3000, 3)
+    want1 = oracle.estimate(cfgs[idx], level=1, threads=THREADS)
+    assert np.array_equal(peak[idx], want1["peak"])
+    assert np.array_equal(got["index"].cpu().numpy()[idx], want1["index"])
+    # event counts of the whole sweep
+    offsets, _ = llmem.event_counts(cfgs)
+    counts = np.diff(offsets.cpu().numpy())
+    assert np.array_equal(counts[idx], want1["count"])
+
+
+def test_g4_max_batch_and_selection_full(llmem):
+    caps = grids.g4_capacities()
+    bmax = grids.G4_BMAX
+    search = grids.g4_search_grid()
+    assert len(search) == (1 << 17) * 64
+    dev = llmem.to_device(search)
+    bs, st = llmem.max_batch(dev, caps, bmax)
+    bs = bs.cpu().numpy()
+    st = st.cpu().numpy()
+    del dev
+    # every 16th shape in full against the bisecting oracle
+    sub = np.arange(0, 1 << 17, 16)
+    rows = (sub[:, None] * 64 + np.arange(64)[None, :]).reshape(-1)
+    want_bs, want_st = oracle.max_batch(search[rows], caps, bmax, level=2, threads=THREADS)
+    assert np.array_equal(st[rows], want_st)
+    assert np.array_equal(bs[rows], want_bs)
+    # the defining property with the level-1 estimate on a sample of the rest
+    ok = np.flatnonzero(st == 0)
+    for i in sample_indices(len(ok), 120, 4):
+        r = ok[i]
+        for m in (0, 5, 8):
+            b = int(bs[r, m])
+            c = search[r:r + 1].copy()
+            if b >= 1:
+                c["batch"] = b
+                e = oracle.estimate(c)
+                assert e["status"][0] == 0 and e["peak"][0] <= caps[m]
+            if b < bmax:
+                c["batch"] = b + 1
+                e = oracle.estimate(c)
+                assert e["status"][0] != 0 or e["peak"][0] > caps[m]
+    assert (st[search["method"] != 3] == 0).all()
+    sel_cfg = grids.g4_select_grid()
+    assert len(sel_cfg) == (1 << 17) * 16
+    got = llmem.select_method(sel_cfg, caps, bmax)
+    rows = (sub[:, None] * 16 + np.arange(16)[None, :]).reshape(-1)
+    want = oracle.select_method(sel_cfg[rows], caps, bmax, level=2, threads=THREADS)
+    for k in ("method", "batch", "bs_list", "status"):
+        assert np.array_equal(got[k].cpu().numpy()[rows], want[k]), k
+    # selection is consistent with the search results of the same shapes everywhere
+    bl = got["bs_list"].cpu().numpy()
+    bs4 = np.maximum(bs.reshape(1 << 17, 4, 16, len(caps)), 0).transpose(0, 2, 3, 1).reshape(-1, len(caps), 4)
+    assert np.array_equal(bl, bs4)
+    assert len(np.unique(got["method"].cpu().numpy())) >= 4
+
+
+def test_g5_stress_materialized_full(llmem):
+    cfgs = grids.g5_stress()
+    assert len(cfgs) == 1 << 16
+    dev = llmem.to_device(cfgs)
+    offsets, status = llmem.event_counts(dev)
+    total = int(offsets[-1].item())
+    free, _ = torch.cuda.mem_get_info()
+    if free < total * 8 + (2 << 30):
+        pytest.skip(f"needs {total * 8 / 2**30:.0f} GiB of free device memory")
+    assert 4_000_000_000 < total < 8_000_000_000
+    delta = llmem.expand_events(dev, offsets, total, fuse_round=True)
+    r = llmem.scan_peak(delta, offsets, dev, check_status=True)
+    fused = llmem.estimate_batch(dev)
+    peak = r["peak"].cpu().numpy()
+    index = r["index"].cpu().numpy()
+    assert np.array_equal(peak, fused["peak"].cpu().numpy())
+    assert np.array_equal(index, fused["index"].cpu().numpy())
+    want2 = oracle.estimate(cfgs, level=2, threads=THREADS)
+    assert (want2["status"] == 0).all() and (status.cpu().numpy() == 0).all()
+    assert np.array_equal(peak, want2["peak"])
+    idx = sample_indices(len(cfgs), 96, 5)
+    want1 = oracle.estimate(cfgs[idx], level=1, threads=THREADS)
+    assert np.array_equal(peak[idx], want1["peak"])
+    assert np.array_equal(index[idx], want1["index"])
+    off = offsets.cpu().numpy()
+    assert np.array_equal(np.diff(off)[idx], want1["count"])
+    # whole event lists of a few configurations, bit for bit
+    for i in idx[:6]:
+        ev = oracle.round_events(oracle.expand_events(cfgs[i:i + 1]))
+        assert np.array_equal(delta[off[i]:off[i + 1]].cpu().numpy(), ev)

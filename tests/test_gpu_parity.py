@@ -1,0 +1,249 @@
+"""Parity of the CUDA library with the CPU oracle, element by element, on the same
+seeded inputs.  All quantities are integers: the bar is bit-exact equality.
+Sizes here are ones the level-1 oracle finishes in seconds; they still span many
+tiles of the expansion and scan kernels (4608 events each) with ragged tails."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2404_10933_b200 import grids
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+G = 2 * 1024 * 1024
+
+
+@pytest.fixture(scope="module")
+def llmem():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    import paper_2404_10933_b200 as m
+    m.lib()
+    return m
+
+
+def oracle_lists(cfgs, rounded):
+    """Concatenated oracle event lists and offsets (status != 0 contributes nothing)."""
+    parts, counts = [], []
+    for i in range(len(cfgs)):
+        st, n = oracle.event_count(cfgs[i:i + 1])
+        if st == 0:
+            ev = oracle.expand_events(cfgs[i:i + 1])
+            parts.append(oracle.round_events(ev) if rounded else ev)
+            counts.append(n)
+        else:
+            counts.append(0)
+    offsets = np.concatenate([[0], np.cumsum(counts)]).astype(np.int64)
+    delta = np.concatenate(parts) if parts else np.zeros(0, dtype=np.int64)
+    return delta, offsets
+
+
+def mixed_small_grid():
+    """All methods and degrees on small shapes, plus inadmissible records."""
+    c = grids.g2_shape_grid(40, 3)           # 3 shapes x 32 batches x 29 combos
+    c = c[::7].copy()                        # 398 configs, every method / degree appears
+    c["chunk_elems"] = np.where(np.arange(len(c)) % 3 == 0, 1 << 22, c["chunk_elems"])
+    c["iters"] = 1 + (np.arange(len(c)) % 3)
+    bad = grids.g2_shape_grid(41, 1)[:12].copy()
+    bad["layers"][0] = 0
+    bad["heads"][1] = 7
+    bad["method"][2] = 9
+    bad["method"][3], bad["gpu_n"][3], bad["tp_n"][3] = 3, 4, 3      # inadmissible DP+TP
+    bad["method"][4], bad["gpu_n"][4], bad["tp_n"][4] = 3, 2, 2
+    bad["batch"][5], bad["seq"][5], bad["vocab"][5] = 1 << 26, 1 << 26, 1 << 26   # >= 2^62 bytes
+    bad["layers"][6], bad["hidden"][6], bad["heads"][6], bad["ffn"][6] = 48, 8192, 64, 32768
+    bad["chunk_elems"][6] = 1                                         # >= 2^31 events
+    bad["reserved"][7, 8] = 1
+    bad["lm_bytes"][8] = 3
+    bad["seq"][9] = 1                                                 # valid: zero-byte shifted logits
+    bad["method"][10], bad["gpu_n"][10] = 2, 1                        # valid: zero-byte TP buffers
+    bad["method"][11], bad["gpu_n"][11] = 1, 1                        # valid: zero-byte gathers
+    out = np.concatenate([c[:150], bad, c[150:]])
+    return out
+
+
+def check_estimate(llmem, cfgs, threads=8):
+    want = oracle.estimate(cfgs, threads=threads)
+    got = llmem.estimate_batch(cfgs)
+    torch.cuda.synchronize()
+    assert np.array_equal(got["status"].cpu().numpy(), want["status"])
+    assert np.array_equal(got["peak"].cpu().numpy(), want["peak"])
+    assert np.array_equal(got["index"].cpu().numpy(), want["index"])
+    return want
+
+
+def check_materialized(llmem, cfgs, want):
+    dev = llmem.to_device(cfgs)
+    offsets, status = llmem.event_counts(dev)
+    raw_want, off_want = oracle_lists(cfgs, rounded=False)
+    assert np.array_equal(offsets.cpu().numpy(), off_want)
+    assert np.array_equal(status.cpu().numpy(), want["status"])
+    total = int(off_want[-1])
+    raw = llmem.expand_events(dev, offsets, total)
+    assert np.array_equal(raw.cpu().numpy(), raw_want)
+    rounded_want = oracle.round_events(raw_want)
+    fused = llmem.expand_events(dev, offsets, total, fuse_round=True)
+    assert np.array_equal(fused.cpu().numpy(), rounded_want)
+    # scan of raw deltas with rounding fused into the read
+    r1 = llmem.scan_peak(raw, offsets, dev, fuse_round=True, check_status=True)
+    # separate rounding kernel, then plain scan
+    rounded = llmem.round_events(raw.clone())
+    assert np.array_equal(rounded.cpu().numpy(), rounded_want)
+    r2 = llmem.scan_peak(rounded, offsets, dev, check_status=True)
+    r3 = llmem.scan_peak(fused, offsets, dev, check_status=True)
+    for r in (r1, r2, r3):
+        assert np.array_equal(r["peak"].cpu().numpy(), want["peak"])
+        assert np.array_equal(r["index"].cpu().numpy(), want["index"])
+    return total
+
+
+def test_g1_small_grid_all_entry_points(llmem):
+    cfgs = grids.g1_small()
+    want = check_estimate(llmem, cfgs)
+    assert (want["count"] == 308).all()
+    total = check_materialized(llmem, cfgs, want)
+    assert total == 64 * 308
+    pipe = llmem.estimate_materialized(cfgs)
+    assert np.array_equal(pipe["peak"].cpu().numpy(), want["peak"])
+
+
+def test_mixed_methods_and_inadmissible_records(llmem):
+    cfgs = mixed_small_grid()
+    want = check_estimate(llmem, cfgs)
+    assert set(np.unique(want["status"])) == {0, 1, 2, 3}
+    total = check_materialized(llmem, cfgs, want)
+    assert total > 50 * 4608          # spans many tiles
+
+
+def test_tiny_segments_many_per_tile(llmem):
+    # 21 .. ~100 events per configuration: dozens of segments inside every tile
+    c = grids.g2_shape_grid(7, 1)
+    c["layers"] = 1 + (np.arange(len(c)) % 3)
+    c["hidden"], c["heads"], c["ffn"] = 256, 4, 1024
+    c["chunk_elems"] = 1 << 22
+    want = check_estimate(llmem, c)
+    assert want["count"][want["status"] == 0].max() < 200
+    total = check_materialized(llmem, c, want)
+    assert total > 3 * 4608
+
+
+def test_empty_and_degenerate_calls(llmem):
+    z = grids.empty(0)
+    r = llmem.estimate_batch(z)
+    assert r["peak"].numel() == 0
+    offsets, _ = llmem.event_counts(z)
+    assert offsets.cpu().tolist() == [0]
+    # every record inadmissible: no events at all, scan must still define the outputs
+    c = grids.g1_small()[:5].copy()
+    c["layers"] = 0
+    want = oracle.estimate(c)
+    pipe = llmem.estimate_materialized(c)
+    assert pipe["total_events"] == 0
+    assert np.array_equal(pipe["peak"].cpu().numpy(), want["peak"])
+    assert np.array_equal(pipe["index"].cpu().numpy(), want["index"])
+    assert (want["peak"] == -1).all()
+    # a single configuration
+    one = grids.g1_small()[3:4]
+    check_materialized(llmem, one, check_estimate(llmem, one))
+
+
+def test_scan_of_arbitrary_lists_and_alignments(llmem):
+    """llmem_scan_peak on lists it did not produce: random signed values, segment
+    lengths from 0 to several tiles (including exact tile multiples), and a delta
+    pointer that is only 8-byte aligned."""
+    rng = np.random.default_rng(2404)
+    lens = [0, 1, 2, 4607, 4608, 4609, 0, 0, 9216, 13824, 5, 70000, 3, 0, 4608 * 3 - 1, 1, 18, 17, 19,
+            250000, 0]
+    lens += rng.integers(0, 300, size=400).tolist()
+    lens += [0]
+    offsets = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    total = int(offsets[-1])
+    delta = rng.integers(-(1 << 40), 1 << 40, size=total, dtype=np.int64)
+    delta[rng.integers(0, total, size=total // 10)] = 0
+    want_peak = np.zeros(len(lens), dtype=np.int64)
+    want_idx = np.zeros(len(lens), dtype=np.int64)
+    want_peak_r = np.zeros(len(lens), dtype=np.int64)
+    want_idx_r = np.zeros(len(lens), dtype=np.int64)
+    for i in range(len(lens)):
+        seg = delta[offsets[i]:offsets[i + 1]]
+        want_peak[i], want_idx[i] = oracle.scan_peak(seg)
+        want_peak_r[i], want_idx_r[i] = oracle.scan_peak(oracle.round_events(seg))
+    off_dev = torch.from_numpy(offsets).cuda()
+    for shift in (0, 1):
+        buf = torch.zeros(total + 3, dtype=torch.int64, device="cuda")
+        view = buf[shift:shift + total]
+        assert view.data_ptr() % 16 == 8 * shift
+        view.copy_(torch.from_numpy(delta))
+        r = llmem.scan_peak(view, off_dev, None, check_status=True)
+        assert np.array_equal(r["peak"].cpu().numpy(), want_peak)
+        assert np.array_equal(r["index"].cpu().numpy(), want_idx)
+        r = llmem.scan_peak(view, off_dev, None, fuse_round=True, check_status=True)
+        assert np.array_equal(r["peak"].cpu().numpy(), want_peak_r)
+        assert np.array_equal(r["index"].cpu().numpy(), want_idx_r)
+        # in-place rounding on the same (mis)aligned view
+        llmem.round_events(view)
+        assert np.array_equal(view.cpu().numpy(), oracle.round_events(delta))
+        assert int(buf[shift + total:].abs().sum()) == 0 and (shift == 0 or int(buf[0]) == 0)
+
+
+def test_expand_into_unaligned_output(llmem):
+    cfgs = mixed_small_grid()[:60]
+    dev = llmem.to_device(cfgs)
+    offsets, _ = llmem.event_counts(dev)
+    want, off_want = oracle_lists(cfgs, rounded=True)
+    total = int(off_want[-1])
+    buf = torch.full((total + 4,), -7, dtype=torch.int64, device="cuda")
+    out = llmem.expand_events(dev, offsets, total, fuse_round=True, out=buf[1:1 + total])
+    assert out.data_ptr() % 16 == 8
+    assert np.array_equal(out.cpu().numpy(), want)
+    assert buf[0].item() == -7 and (buf[1 + total:] == -7).all()
+
+
+def test_max_batch_and_select_small(llmem):
+    shapes = grids.g4_search_grid(0, 8)              # 8 shapes x 4 methods x 16 degrees
+    shapes["chunk_elems"] = 1 << 25                  # keeps the literal (level-1) oracle quick
+    caps = grids.g4_capacities()
+    bmax = 40
+    want_bs, want_st = oracle.max_batch(shapes, caps, bmax, level=1, threads=8)
+    got_bs, got_st = llmem.max_batch(shapes, caps, bmax)
+    assert np.array_equal(got_st.cpu().numpy(), want_st)
+    assert np.array_equal(got_bs.cpu().numpy(), want_bs)
+    assert (want_bs == 0).any() and (want_bs == bmax).any() and ((want_bs > 0) & (want_bs < bmax)).any()
+    sel_shapes = grids.g4_select_grid(0, 8)
+    sel_shapes["chunk_elems"] = 1 << 25
+    for allzero in (False, True):
+        want = oracle.select_method(sel_shapes, caps, bmax, flags=1 if allzero else 0, level=1, threads=8)
+        got = llmem.select_method(sel_shapes, caps, bmax, allzero=allzero)
+        for k in ("method", "batch", "bs_list", "status"):
+            assert np.array_equal(got[k].cpu().numpy(), want[k]), k
+    # inadmissible shapes and the full batch range against the bisecting oracle
+    bad = shapes[:6].copy()
+    bad["hidden"][0] = 0
+    bad["method"][1] = 7
+    bad["layers"][2], bad["hidden"][2], bad["heads"][2], bad["ffn"][2] = 48, 8192, 64, 32768
+    bad["chunk_elems"][2] = 1            # >= 2^31 events
+    bad["batch"][3] = -5                 # ignored by the search
+    want_bs, want_st = oracle.max_batch(bad, caps, 4096, level=2)
+    got_bs, got_st = llmem.max_batch(bad, caps, 4096)
+    assert np.array_equal(got_st.cpu().numpy(), want_st) and want_st.tolist()[:3] == [1, 1, 3]
+    assert np.array_equal(got_bs.cpu().numpy(), want_bs)
+    want = oracle.select_method(bad, caps, 4096, level=2)
+    got = llmem.select_method(bad, caps, 4096)
+    for k in ("method", "batch", "bs_list", "status"):
+        assert np.array_equal(got[k].cpu().numpy(), want[k]), k
+
+
+def test_aligned_family_on_device(llmem):
+    # the page-aligned family of the oracle pins, straight through the CUDA path
+    c = grids.empty(4)
+    for k, v in dict(layers=4, hidden=2048, heads=16, ffn=8192, vocab=65536, pos_len=0, seq=1024, batch=32,
+                     chunk_elems=1 << 24, base_bytes=123456789, lm_bytes=2, iters=2).items():
+        c[k] = v
+    c["method"] = [0, 1, 2, 3]
+    c["gpu_n"] = [1, 4, 4, 4]
+    c["tp_n"] = [0, 0, 0, 2]
+    want = oracle.estimate(c)
+    got = llmem.estimate_batch(c)
+    assert np.array_equal(got["peak"].cpu().numpy(), want["peak"])
+    assert ((want["peak"] - 123456789 - 65536 * 2048 * 2) % G == 0).all()
