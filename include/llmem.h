@@ -116,6 +116,42 @@ llmem_status llmem_event_counts(const llmem_config* DEV cfg, int64_t n, int64_t*
                                 uint8_t* DEV status_out, void* DEV scratch, size_t scratch_bytes,
                                 uint32_t flags, void* cuda_stream);
 
+/* Largest n accepted by llmem_event_counts_static. */
+#define LLMEM_STATIC_MAX_CONFIGS 4194304
+
+/* No counterpart in the paper: a convenience of this library.  Same results as
+ * llmem_event_counts, bit for bit, for callers that are not in a position to
+ * provide scratch because they cannot allocate device memory at the point of
+ * the call: code running under a framework whose allocator they may not re-enter
+ * (a callback, a custom-op hook), services that pre-size all device memory at
+ * start-up and forbid cudaMalloc afterwards, and callers preparing a sequence of
+ * work in which an allocation would force a device-wide synchronisation.  They
+ * still pass the input and output buffers; only the scratch is supplied by the
+ * library.
+ *
+ * The scratch (one partial sum per 1024 configurations) is a fixed array of about
+ * 32 KiB in the library's device image; every GPU on which the library is used
+ * holds it until the process exits.  Hence the limit: n <= LLMEM_STATIC_MAX_CONFIGS,
+ * larger n returns LLMEM_ERR_ARG with an explanatory llmem_last_error() and does no
+ * work.  The call itself performs no cudaMalloc, cudaFree or other allocation.
+ *
+ * The first call on each device looks up the array's device address (a query, not
+ * an allocation) and caches it; make that first call in ordinary stream execution,
+ * before any stream capture is begun on that device.
+ *
+ * All calls on one device share the one array, and it keeps what the previous call
+ * left there.  That is harmless for calls that follow one another in one stream
+ * (each call writes every entry before reading it), but two calls that may run on the
+ * GPU at the same time -- different streams, different host threads -- race on it and
+ * yield undefined offsets.  Serialise them, or use llmem_event_counts with separate
+ * scratch buffers.
+ *   cfg         DEV [n]
+ *   offsets_out DEV [n+1]
+ *   status_out  DEV [n], nullable */
+llmem_status llmem_event_counts_static(const llmem_config* DEV cfg, int64_t n,
+                                       int64_t* DEV offsets_out, uint8_t* DEV status_out,
+                                       uint32_t flags, void* cuda_stream);
+
 /* Sections 4.1 and 5: the signed byte count of every event, allocations
  * positive and frees negative, configuration i occupying
  * delta_out[offsets[i] .. offsets[i+1]).  Order: initialisation (embedding unit,

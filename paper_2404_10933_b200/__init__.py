@@ -32,8 +32,9 @@ METHOD_OFFLOAD = 4
 EXPORTS = (
     "llmem_scratch_bytes", "llmem_estimate_batch", "llmem_event_counts", "llmem_expand_events",
     "llmem_round_events", "llmem_scan_peak", "llmem_max_batch", "llmem_select_method",
-    "llmem_scratch_status", "llmem_last_error", "llmem_version",
+    "llmem_scratch_status", "llmem_last_error", "llmem_version", "llmem_event_counts_static",
 )
+STATIC_MAX_CONFIGS = 4194304
 
 
 class LlmemError(RuntimeError):
@@ -60,6 +61,7 @@ def lib() -> ctypes.CDLL:
         L.llmem_scratch_bytes.argtypes = [ctypes.c_int, i64, i64]
         L.llmem_estimate_batch.argtypes = [vp, i64, vp, vp, vp, vp, sz, u32, vp]
         L.llmem_event_counts.argtypes = [vp, i64, vp, vp, vp, sz, u32, vp]
+        L.llmem_event_counts_static.argtypes = [vp, i64, vp, vp, u32, vp]
         L.llmem_expand_events.argtypes = [vp, i64, vp, i64, vp, vp, sz, u32, vp]
         L.llmem_round_events.argtypes = [vp, i64, vp, sz, u32, vp]
         L.llmem_scan_peak.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, sz, u32, vp]
@@ -149,6 +151,29 @@ def event_counts(cfg, *, want_status: bool = True, stream=None):
     _check(lib().llmem_event_counts(_ptr(cfg), n, _ptr(offsets), _ptr(status), _ptr(scratch), nbytes, 0,
                                     _stream_ptr(stream)))
     return offsets, status
+
+
+def event_counts_static(cfg, offsets_out, status_out=None, *, stream=None):
+    """``event_counts`` for callers that must not allocate device memory at the point of
+    the call (for instance code running inside a framework callback that may not re-enter
+    the allocator, or a service whose device memory is fixed at start-up).  The caller
+    passes every tensor, ``offsets_out`` ([n+1] int64) and optionally ``status_out`` ([n]
+    uint8); the library's own fixed device array serves as scratch, so neither this
+    function nor the library allocates anything.  ``n`` may not exceed
+    ``STATIC_MAX_CONFIGS``.  Calls that can overlap on the GPU share that array and race:
+    keep them in one stream."""
+    torch = _torch()
+    if cfg.dtype != torch.uint8 or cfg.dim() != 2 or cfg.shape[1] != 64 or not cfg.is_cuda \
+            or not cfg.is_contiguous():
+        raise ValueError("cfg must be a contiguous CUDA uint8 tensor of shape [n, 64]")
+    n = cfg.shape[0]
+    if offsets_out.dtype != torch.int64 or offsets_out.numel() < n + 1 or not offsets_out.is_contiguous():
+        raise ValueError("offsets_out must be a contiguous int64 tensor with n + 1 elements")
+    if status_out is not None and (status_out.dtype != torch.uint8 or status_out.numel() < n):
+        raise ValueError("status_out must be a uint8 tensor with n elements")
+    _check(lib().llmem_event_counts_static(_ptr(cfg), n, _ptr(offsets_out), _ptr(status_out), 0,
+                                           _stream_ptr(stream)))
+    return offsets_out
 
 
 def expand_events(cfg, offsets, total_events: Optional[int] = None, *, fuse_round: bool = False,

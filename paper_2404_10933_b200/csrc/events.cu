@@ -3,6 +3,8 @@
 // rounding.  The expansion is bound by HBM writes (8 bytes per event): each CTA
 // builds a tile of deltas in shared memory and hands it to the TMA engine as one
 // bulk store, double-buffered so that filling the next tile overlaps the store.
+#include <mutex>
+
 #include "llmem_host.h"
 #include "llmem_model.cuh"
 
@@ -445,6 +447,81 @@ extern "C" llmem_status llmem_event_counts(const llmem_config* cfg, int64_t n, i
   if (blocks3 > cap3) blocks3 = cap3;
   add_block_base_kernel<<<(unsigned)blocks3, 256, 0, s>>>(reinterpret_cast<i64*>(offsets_out), n, block_sums, nblocks);
   return check_launch("llmem_event_counts");
+}
+
+// ---------------------------------------------------------------------------
+// llmem_event_counts_static: the same three kernels, with the per-CTA partial sums
+// kept in a file-scope device array instead of caller-provided scratch.
+// ---------------------------------------------------------------------------
+namespace llmem {
+
+constexpr i64 kStaticMaxConfigs = LLMEM_STATIC_MAX_CONFIGS;
+constexpr i64 kStaticSums = kStaticMaxConfigs / kCountBlock + 1;  // 4096 CTA totals + the grand total
+static_assert(kStaticMaxConfigs % kCountBlock == 0, "limit is a whole number of CTAs");
+
+// Lives in the module image of every device that loads the library (about 32 KiB)
+// until the process exits.  Shared by all calls of the entry point below.
+static __device__ __align__(256) unsigned long long g_static_block_sums[kStaticSums];
+
+constexpr int kMaxDevices = 64;
+static u64* g_static_ptr[kMaxDevices];  // device address of the array, per device ordinal
+static std::mutex g_static_mutex;
+
+// In host code `g_static_block_sums` names a host-side shadow of the symbol, not
+// device memory; the address a kernel may dereference has to be asked for, with the
+// device in question current.
+static llmem_status static_sums_address(u64** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) { set_error("llmem_event_counts_static: cudaGetDevice: %s", cudaGetErrorString(e)); return LLMEM_ERR_CUDA; }
+  if (dev < 0 || dev >= kMaxDevices) { set_error("llmem_event_counts_static: device ordinal %d beyond %d", dev, kMaxDevices - 1); return LLMEM_ERR_ARG; }
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (!g_static_ptr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_block_sums);
+    if (e != cudaSuccess || !p) {
+      set_error("llmem_event_counts_static: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+      return LLMEM_ERR_CUDA;
+    }
+    g_static_ptr[dev] = static_cast<u64*>(p);
+  }
+  *out = g_static_ptr[dev];
+  return LLMEM_OK;
+}
+
+}  // namespace llmem
+
+extern "C" llmem_status llmem_event_counts_static(const llmem_config* cfg, int64_t n, int64_t* offsets_out,
+                                                  uint8_t* status_out, uint32_t flags, void* cuda_stream) {
+  (void)flags;
+  clear_error();
+  if (n < 0) { set_error("llmem_event_counts_static: n < 0"); return LLMEM_ERR_ARG; }
+  if (n > kStaticMaxConfigs) {
+    set_error("llmem_event_counts_static: n = %lld exceeds LLMEM_STATIC_MAX_CONFIGS = %lld; split the batch or "
+              "use llmem_event_counts with caller-provided scratch", (long long)n, (long long)kStaticMaxConfigs);
+    return LLMEM_ERR_ARG;
+  }
+  if (!offsets_out || !aligned_to(offsets_out, 8)) { set_error("llmem_event_counts_static: offsets_out is required"); return LLMEM_ERR_ARG; }
+  if (n > 0 && (!cfg || !aligned_to(cfg, 16))) { set_error("llmem_event_counts_static: cfg must be a 16-byte aligned device pointer"); return LLMEM_ERR_ARG; }
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (n == 0) {
+    if (cudaMemsetAsync(offsets_out, 0, sizeof(int64_t), s) != cudaSuccess) return check_launch("llmem_event_counts_static");
+    return LLMEM_OK;
+  }
+  u64* block_sums = nullptr;
+  llmem_status st = static_sums_address(&block_sums);
+  if (st != LLMEM_OK) return st;
+  // Nothing in the array has to start at zero: pass 1 writes entries [0, nblocks), pass 2
+  // rewrites them and writes entry [nblocks], and no pass reads an entry this call has not
+  // written.  What an earlier call left beyond nblocks is never looked at.
+  const i64 nblocks = (n + kCountBlock - 1) / kCountBlock;
+  count_kernel<<<(unsigned)nblocks, kCountThreads, 0, s>>>(cfg, n, reinterpret_cast<i64*>(offsets_out), status_out, block_sums);
+  scan_block_sums_kernel<<<1, kCountThreads, 0, s>>>(block_sums, nblocks);
+  i64 blocks3 = (n + 1 + 255) / 256;
+  const i64 cap3 = (i64)sm_count() * 8;
+  if (blocks3 > cap3) blocks3 = cap3;
+  add_block_base_kernel<<<(unsigned)blocks3, 256, 0, s>>>(reinterpret_cast<i64*>(offsets_out), n, block_sums, nblocks);
+  return check_launch("llmem_event_counts_static");
 }
 
 extern "C" llmem_status llmem_expand_events(const llmem_config* cfg, int64_t n, const int64_t* offsets,
