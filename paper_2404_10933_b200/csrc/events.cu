@@ -1,8 +1,9 @@
 // Materialised event lists: per-configuration event counts and their exclusive
 // scan, the expansion kernel that writes every signed delta, and in-place page
-// rounding.  The expansion is bound by HBM writes (8 bytes per event): each CTA
-// builds a tile of deltas in shared memory and hands it to the TMA engine as one
-// bulk store, double-buffered so that filling the next tile overlaps the store.
+// rounding.  The expansion is bound by HBM writes (8 bytes per event): each warp
+// builds 576-event chunks of deltas in its own shared memory and hands each to the
+// TMA engine as one bulk store, double-buffered so that filling the next chunk
+// overlaps the store.
 #include <mutex>
 
 #include "llmem_host.h"
@@ -119,11 +120,12 @@ add_block_base_kernel(i64* __restrict__ offsets, i64 n, const u64* __restrict__ 
 // expansion
 // ---------------------------------------------------------------------------
 constexpr int kExpThreads = 256;
-// 18 events = 144 bytes = nine 16-byte words per thread: an odd word count makes
-// the per-thread spans fall on distinct shared-memory banks.
-constexpr int kExpPerThread = 18;
-constexpr int kExpTile = kExpThreads * kExpPerThread;  // 4608 events, 36 KiB
-constexpr int kDescBatch = 8;
+constexpr int kExpWarps = kExpThreads / 32;
+// 18 events = 144 bytes = nine 16-byte words per lane: an odd word count makes
+// the per-lane spans fall on distinct shared-memory banks.
+constexpr int kExpPerLane = 18;
+constexpr int kExpChunk = 32 * kExpPerLane;  // 576 events, 4608 bytes: one warp's unit of work
+constexpr int kExpCtasPerSm = 2;
 constexpr int kRuns = 17;
 
 // A run of events that repeat with a short period: the first `split` events of each
@@ -285,111 +287,117 @@ __device__ i64 first_segment_after(const i64* __restrict__ offsets, i64 n, i64 p
   return lo;
 }
 
-struct ExpandSmem {
-  alignas(128) i64 tile[2][kExpTile];
-  SegDesc desc[kDescBatch];
-  i64 tag[kDescBatch];
-  i64 seg0;
+// One warp's private shared memory: two chunk buffers (filled, then handed to the
+// TMA engine while the other one is being filled) and the descriptor of the
+// segment the warp is currently inside.
+struct ExpandWarpSmem {
+  alignas(128) i64 buf[2][kExpChunk];
+  SegDesc desc;
 };
 
+// Write `cnt` events starting at segment position `pos` to dst[0 .. cnt).  Spans that
+// stay inside one run of period 1 or 2 (parameter chunks, gathers, outputs: almost
+// all of a long list) are written as constants; anything else goes through the
+// run cursor event by event.
+__device__ __forceinline__ void fill_span(i64* __restrict__ dst, const SegDesc& d, u32 pos, int cnt) {
+  Cursor c;
+  seek(c, d, pos);
+  if (c.rem >= cnt && c.period <= 2) {
+    const i64 x0 = c.phase < c.split ? c.a : c.b;
+    const i64 x1 = c.period == 1 ? x0 : (c.phase < c.split ? c.b : c.a);
+    if (cnt == kExpPerLane && (smem_addr(dst) & 15u) == 0) {
+      longlong2* v = reinterpret_cast<longlong2*>(dst);
+#pragma unroll
+      for (int j = 0; j < kExpPerLane / 2; ++j) v[j] = make_longlong2(x0, x1);
+    } else {
+      for (int j = 0; j < cnt; ++j) dst[j] = (j & 1) ? x1 : x0;
+    }
+    return;
+  }
+  for (int j = 0; j < cnt; ++j) dst[j] = emit(c, d);
+}
+
+// Every warp streams its own contiguous range of 576-event chunks: no CTA-wide
+// barrier anywhere, so the warps of an SM drift apart and cover each other's
+// latencies.  Lane l owns events [18 l, 18 l + 18) of a chunk.
 __global__ void __launch_bounds__(kExpThreads)
 expand_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict__ offsets, i64 total,
-              i64* __restrict__ out, i64 tiles_per_cta, int round, int bulk_ok) {
+              i64* __restrict__ out, i64 chunks_per_warp, int round, int bulk_ok) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  ExpandSmem& sm = *reinterpret_cast<ExpandSmem*>(smem_raw);
-  const int tid = threadIdx.x;
-  const i64 ntiles = (total + kExpTile - 1) / kExpTile;
-  const i64 tile_lo = (i64)blockIdx.x * tiles_per_cta;
-  const i64 tile_hi = tile_lo + tiles_per_cta < ntiles ? tile_lo + tiles_per_cta : ntiles;
-  if (tile_lo >= tile_hi) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  ExpandWarpSmem& ws = reinterpret_cast<ExpandWarpSmem*>(smem_raw)[warp];
+  const i64 gw = (i64)blockIdx.x * kExpWarps + warp;
+  const i64 nchunks = (total + kExpChunk - 1) / kExpChunk;
+  const i64 c_lo = gw * chunks_per_warp;
+  const i64 c_hi = c_lo + chunks_per_warp < nchunks ? c_lo + chunks_per_warp : nchunks;
+  if (c_lo >= c_hi) return;
 
-  if (tid < kDescBatch) sm.tag[tid] = -1;
-  if (tid == 0) sm.seg0 = first_segment_after(offsets, n, tile_lo * kExpTile);
-  __syncthreads();
-  i64 seg = sm.seg0;  // smallest segment index whose end lies beyond the current position
+  // seg: smallest segment whose end lies beyond the current position; gs/ge its range
+  i64 seg = first_segment_after(offsets, n, c_lo * kExpChunk);
+  i64 gs = seg < n ? __ldg(offsets + seg) : total;
+  i64 ge = seg < n ? __ldg(offsets + seg + 1) : total;
+  i64 desc_seg = -1;  // segment described by ws.desc
 
   int parity = 0;
-  for (i64 tile = tile_lo; tile < tile_hi; ++tile, parity ^= 1) {
-    const i64 tb = tile * kExpTile;
-    const i64 te = tb + kExpTile < total ? tb + kExpTile : total;
-    i64* buf = sm.tile[parity];
-    // the bulk store issued from this buffer two tiles ago must have read it
-    if (tid == 0) bulk_wait_read<1>();
-    __syncthreads();
-    const i64 span_lo = tb + (i64)tid * kExpPerThread;
-    const i64 span_hi = span_lo + kExpPerThread < te ? span_lo + kExpPerThread : te;
+  for (i64 c = c_lo; c < c_hi; ++c, parity ^= 1) {
+    const i64 tb = c * kExpChunk;
+    const i64 te = tb + kExpChunk < total ? tb + kExpChunk : total;
+    i64* buf = ws.buf[parity];
+    // the bulk store issued from this buffer two chunks ago must have read it
+    if (lane == 0) bulk_wait_read<1>();
+    __syncwarp();
+    const i64 span_lo = tb + (i64)lane * kExpPerLane;
+    const i64 span_hi = span_lo + kExpPerLane < te ? span_lo + kExpPerLane : te;
     i64 pos = tb;
     while (pos < te) {
-      // descriptors of the next kDescBatch segments that begin before the tile ends
-      if (tid < kDescBatch) {
-        const i64 s = seg + tid;
-        i64 gs = INT64_MAX, ge = INT64_MAX;
-        if (s < n) {
-          gs = __ldg(offsets + s);
-          ge = __ldg(offsets + s + 1);
-        }
-        if (s < n && gs < te) {
-          if (sm.tag[tid] != s) {
-            build_desc(sm.desc[tid], cfg + s, gs, ge, round != 0);
-            sm.tag[tid] = s;
-          }
-        } else {
-          sm.desc[tid].gstart = INT64_MAX;
-          sm.desc[tid].gend = INT64_MAX;
-          sm.tag[tid] = -1;
-        }
-      }
-      __syncthreads();
-      int nb = 0;
-      while (nb < kDescBatch && sm.desc[nb].gstart != INT64_MAX) ++nb;
-      if (nb == 0) {
-        // offsets do not cover the rest of the tile: define it as zeros
+      if (seg >= n) {
+        // offsets do not cover the rest of the chunk: define it as zeros
         for (i64 e = (span_lo > pos ? span_lo : pos); e < span_hi; ++e) buf[e - tb] = 0;
-        pos = te;
-        __syncthreads();
         break;
       }
-      const i64 last_end = sm.desc[nb - 1].gend;
-      const i64 batch_end = last_end < te ? last_end : te;
-      i64 e = span_lo > pos ? span_lo : pos;
-      const i64 e_end = span_hi < batch_end ? span_hi : batch_end;
+      if (desc_seg != seg) {
+        __syncwarp();  // every lane is done with the previous descriptor
+        if (lane == 0) build_desc(ws.desc, cfg + seg, gs, ge, round != 0);
+        __syncwarp();
+        desc_seg = seg;
+      }
+      const i64 piece_end = ge < te ? ge : te;
+      const i64 e = span_lo > pos ? span_lo : pos;
+      const i64 e_end = span_hi < piece_end ? span_hi : piece_end;
       if (e < e_end) {
-        int di = 0;
-        while (di + 1 < nb && sm.desc[di + 1].gstart <= e) ++di;
-        while (di + 1 < nb && sm.desc[di].gend <= e) ++di;
-        Cursor c;
-        bool inval = sm.desc[di].invalid != 0;
-        if (!inval) seek(c, sm.desc[di], (u32)(e - sm.desc[di].gstart));
-        for (; e < e_end; ++e) {
-          if (e >= sm.desc[di].gend) {
-            do { ++di; } while (di + 1 < nb && sm.desc[di].gend <= e);
-            inval = sm.desc[di].invalid != 0;
-            if (!inval) seek(c, sm.desc[di], (u32)(e - sm.desc[di].gstart));
-          }
-          buf[e - tb] = inval ? 0 : emit(c, sm.desc[di]);
+        if (ws.desc.invalid) {
+          for (i64 j = e; j < e_end; ++j) buf[j - tb] = 0;
+        } else {
+          fill_span(buf + (e - tb), ws.desc, (u32)(e - gs), (int)(e_end - e));
         }
       }
-      pos = batch_end;
-      seg += (last_end <= te) ? nb : nb - 1;
-      __syncthreads();  // descriptors are rebuilt by the next round
+      pos = piece_end;
+      if (ge <= te) {
+        // the segment ends inside this chunk: move to the next non-empty one
+        do {
+          ++seg;
+          gs = seg < n ? __ldg(offsets + seg) : total;
+          ge = seg < n ? __ldg(offsets + seg + 1) : total;
+        } while (seg < n && ge <= pos);
+      }
     }
-    // hand the tile to the TMA engine (generic-proxy writes -> async-proxy read)
+    // hand the chunk to the TMA engine (generic-proxy writes -> async-proxy read)
     const u32 cnt = (u32)(te - tb);
     if (bulk_ok) {
       fence_async_shared();
-      __syncthreads();
-      if (tid == 0) {
+      __syncwarp();
+      if (lane == 0) {
         const u32 even = cnt & ~1u;
         if (even) bulk_store(out + tb, buf, even * 8u);
         bulk_commit();
         if (cnt & 1u) out[tb + cnt - 1] = buf[cnt - 1];
       }
     } else {
-      __syncthreads();
-      for (u32 i = tid; i < cnt; i += kExpThreads) out[tb + i] = buf[i];
+      __syncwarp();
+      for (u32 i = lane; i < cnt; i += 32) out[tb + i] = buf[i];
     }
   }
-  if (tid == 0) bulk_wait_read<0>();
+  if (lane == 0) bulk_wait_read<0>();
 }
 
 // ---------------------------------------------------------------------------
@@ -536,22 +544,25 @@ extern "C" llmem_status llmem_expand_events(const llmem_config* cfg, int64_t n, 
     set_error("llmem_expand_events: misaligned pointer");
     return LLMEM_ERR_ARG;
   }
+  const size_t smem = sizeof(ExpandWarpSmem) * kExpWarps;
   static thread_local int configured_dev = -1;
   int dev = 0;
   cudaGetDevice(&dev);
   if (configured_dev != dev) {
-    if (cudaFuncSetAttribute(expand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ExpandSmem)) != cudaSuccess)
+    if (cudaFuncSetAttribute(expand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return check_launch("llmem_expand_events (shared memory opt-in)");
     configured_dev = dev;
   }
-  const i64 ntiles = (total_events + kExpTile - 1) / kExpTile;
-  i64 grid = (i64)sm_count() * 2;
-  if (grid > ntiles) grid = ntiles;
-  const i64 tiles_per_cta = (ntiles + grid - 1) / grid;
-  grid = (ntiles + tiles_per_cta - 1) / tiles_per_cta;
-  expand_kernel<<<(unsigned)grid, kExpThreads, sizeof(ExpandSmem), static_cast<cudaStream_t>(cuda_stream)>>>(
+  const i64 nchunks = (total_events + kExpChunk - 1) / kExpChunk;
+  i64 grid = (i64)sm_count() * kExpCtasPerSm;
+  i64 warps = grid * kExpWarps;
+  if (warps > nchunks) warps = nchunks;
+  const i64 chunks_per_warp = (nchunks + warps - 1) / warps;
+  warps = (nchunks + chunks_per_warp - 1) / chunks_per_warp;
+  grid = (warps + kExpWarps - 1) / kExpWarps;
+  expand_kernel<<<(unsigned)grid, kExpThreads, smem, static_cast<cudaStream_t>(cuda_stream)>>>(
       cfg, n, reinterpret_cast<const i64*>(offsets), total_events, reinterpret_cast<i64*>(delta_out),
-      tiles_per_cta, (flags & LLMEM_FUSE_ROUND) ? 1 : 0, aligned_to(delta_out, 16) ? 1 : 0);
+      chunks_per_warp, (flags & LLMEM_FUSE_ROUND) ? 1 : 0, aligned_to(delta_out, 16) ? 1 : 0);
   return check_launch("llmem_expand_events");
 }
 

@@ -1,31 +1,33 @@
 // Segmented prefix-sum + max over materialised event lists (llmem_scan_peak).
 //
-// Bound by HBM reads (8 bytes per event).  The event array is cut into flat tiles
-// regardless of segment boundaries, so long and short segments load every SM
-// equally.  Each persistent CTA owns a contiguous range of tiles.  A producer lane
-// streams tiles into a ring of shared-memory stages with 1-D TMA bulk copies
-// completing on mbarriers; 256 consumer threads each read 18 consecutive events
-// from the stage (nine 16-byte words, an odd count, hence conflict-free), fold them
-// in order, and combine across the warp with shuffles and across warps through
-// shared memory.  The fold is the associative, non-commutative operator on
-// (sum, max prefix, arg max):  (s1,m1) + (s2,m2) = (s1+s2, max(m1, s1+m2)).
+// Bound by HBM reads (8 bytes per event).  The event array is cut into flat
+// 576-event chunks regardless of segment boundaries, so long and short segments
+// load every SM equally.  Every warp of the persistent grid owns a contiguous range
+// of chunks and streams it on its own: lane 0 keeps four 1-D TMA bulk copies in
+// flight into the warp's private ring of shared-memory stages, each completing on
+// an mbarrier; each lane reads 18 consecutive events from a landed stage (nine
+// 16-byte words, an odd count, hence conflict-free), folds them in order, and the
+// warp combines with shuffles.  The fold is the associative, non-commutative
+// operator on (sum, max prefix, arg max):  (s1,m1) + (s2,m2) = (s1+s2, max(m1, s1+m2)).
+// There is no CTA-wide barrier: the warps of an SM drift apart and cover each
+// other's latencies.
 //
-// Segments that end inside a CTA's range are finished by that CTA.  A segment that
-// crosses CTA ranges leaves one partial per CTA in scratch; a second, tiny kernel
-// folds those in order.  No CTA ever waits on another CTA.  The only waits are on
-// the CTA's own mbarriers, and they are bounded: on expiry the kernel records
-// LLMEM_ERR_TIMEOUT in the scratch status word, drains its own copies and returns.
+// Segments that end inside a warp's range are finished by that warp.  A segment
+// that crosses warp ranges leaves one partial per warp in scratch; a second, tiny
+// kernel folds those in order.  No warp ever waits on another warp.  The only waits
+// are on the warp's own mbarriers, and they are bounded: on expiry the kernel
+// records LLMEM_ERR_TIMEOUT in the scratch status word, drains its own copies and
+// returns.
 #include "llmem_host.h"
 #include "llmem_model.cuh"
 
 namespace llmem {
 
-constexpr int kScanConsumers = 256;
-constexpr int kScanWarps = kScanConsumers / 32;
-constexpr int kScanThreads = kScanConsumers + 32;  // + one producer warp
-constexpr int kScanPerThread = 18;
-constexpr int kScanTile = kScanConsumers * kScanPerThread;  // 4608 events = 36 KiB
-constexpr int kScanStages = 4;
+constexpr int kScanThreads = 256;
+constexpr int kScanWarps = kScanThreads / 32;
+constexpr int kScanPerLane = 18;
+constexpr int kScanChunk = 32 * kScanPerLane;  // 576 events = 4608 bytes: one warp's unit of work
+constexpr int kScanStages = 4;                 // chunks in flight per warp
 
 struct Agg {
   i64 sum, mx, idx;  // idx: virtual (alignment-shifted) global index of the first arg max
@@ -96,16 +98,17 @@ __device__ __forceinline__ u64 global_timer_ns() {
 
 constexpr u64 kWaitLimitNs = 2000000000ull;  // 2 s
 
-// Wait for a phase of an mbarrier, giving up after kWaitLimitNs or when another
-// thread of the CTA has given up.  Returns false on give-up.
+// Wait for a phase of an mbarrier, giving up after kWaitLimitNs, or at once when
+// `abort_flag` (optional) shows that another lane of the warp has given up.  Returns
+// false on give-up and raises the flag.
 __device__ __forceinline__ bool mbar_wait_bounded(u64* bar, u32 parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
   const u64 t0 = global_timer_ns();
   for (u32 spin = 0;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
+    if (abort_flag && *abort_flag) return false;
     if ((spin & 63u) == 63u && global_timer_ns() - t0 > kWaitLimitNs) {
-      *abort_flag = 1;
+      if (abort_flag) *abort_flag = 1;
       return false;
     }
   }
@@ -118,18 +121,10 @@ __device__ __forceinline__ void bulk_load(void* sdst, const void* gsrc, u32 byte
       : "memory");
 }
 
-__device__ __forceinline__ void consumer_barrier() {
-  asm volatile("bar.sync 1, %0;\n" ::"n"(kScanConsumers) : "memory");
-}
-
-struct ScanSmem {
-  alignas(128) i64 stage[kScanStages][kScanTile];
+// One warp's private shared memory.
+struct ScanWarpSmem {
+  alignas(128) i64 stage[kScanStages][kScanChunk];
   u64 full[kScanStages];
-  u64 empty[kScanStages];
-  Agg warp_agg[2][kScanWarps];
-  Agg head, tail;     // slow path: partial of a segment entering / leaving the tile
-  i64 next_seg;       // slow path: broadcast of the segment that contains the next tile
-  int abort_flag;
 };
 
 // Per-configuration additive offset m_base + lm_p and admissibility.
@@ -177,79 +172,84 @@ __device__ __forceinline__ Agg warp_fold_range(const i64* __restrict__ tile, int
   return warp_fold(g, lane);
 }
 
-// Scratch payload: per CTA a head partial (segment that began in an earlier CTA's
-// range) and a tail partial (segment that continues into a later CTA's range).
-struct CtaPartials {
+// Scratch payload: per warp a head partial (segment that began in an earlier warp's
+// range) and a tail partial (segment that continues into a later warp's range).
+struct WarpPartials {
   Agg head, tail;
 };
+
+// Result of the fast path before it is widened to an Agg: chunk-local arg max.
+struct Fold3 {
+  i64 sum, mx;
+  int ix;
+};
+
+__device__ __forceinline__ Fold3 fold3(const Fold3& a, const Fold3& b) {
+  Fold3 r;
+  r.sum = a.sum + b.sum;
+  const i64 cand = a.sum + b.mx;
+  const bool take = cand > a.mx;
+  r.mx = take ? cand : a.mx;
+  r.ix = take ? b.ix : a.ix;
+  return r;
+}
 
 template <bool kRound>
 __global__ void __launch_bounds__(kScanThreads, 1)
 scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, int shift /* 0 or 1 */,
             const i64* __restrict__ offsets, i64 n, i64 total,
-            i64* __restrict__ peak_out, i64* __restrict__ index_out, i64 tiles_per_cta,
-            CtaPartials* __restrict__ partials, u32* __restrict__ status_word) {
+            i64* __restrict__ peak_out, i64* __restrict__ index_out, i64 chunks_per_warp,
+            WarpPartials* __restrict__ partials, u32* __restrict__ status_word) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  ScanSmem& sm = *reinterpret_cast<ScanSmem*>(smem_raw);
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  ScanWarpSmem& ws = reinterpret_cast<ScanWarpSmem*>(smem_raw)[warp];
+  __shared__ int abort_flags[kScanWarps];
+  const i64 gw = (i64)blockIdx.x * kScanWarps + warp;
   // virtual indices: event e lives at v = e + shift, so that v even <=> 16-byte aligned
   const i64 v_begin = shift, v_end = (i64)shift + total;
-  const i64 ntiles = (v_end + kScanTile - 1) / kScanTile;
-  const i64 tile_lo = (i64)blockIdx.x * tiles_per_cta;
-  const i64 tile_hi = tile_lo + tiles_per_cta < ntiles ? tile_lo + tiles_per_cta : ntiles;
+  const i64 nchunks = (v_end + kScanChunk - 1) / kScanChunk;
+  const i64 c_lo = gw * chunks_per_warp;
+  const i64 c_hi = c_lo + chunks_per_warp < nchunks ? c_lo + chunks_per_warp : nchunks;
 
-  if (tid == 0) {
-    partials[blockIdx.x].head = agg_identity();
-    partials[blockIdx.x].tail = agg_identity();
-    for (int s = 0; s < kScanStages; ++s) {
-      mbar_init(&sm.full[s], 1);
-      mbar_init(&sm.empty[s], kScanWarps);
-    }
-    sm.abort_flag = 0;
+  if (lane == 0) {
+    partials[gw].head = agg_identity();
+    partials[gw].tail = agg_identity();
+  }
+  if (c_lo >= c_hi) return;
+  if (lane == 0) {
+    for (int s = 0; s < kScanStages; ++s) mbar_init(&ws.full[s], 1);
+    abort_flags[warp] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
-  __syncthreads();
-  if (tile_lo >= tile_hi) return;
-  volatile int* abort_flag = &sm.abort_flag;
+  __syncwarp();
+  volatile int* abort_flag = &abort_flags[warp];
 
-  if (warp == kScanWarps) {
-    // ---------------- producer ----------------
-    if (lane == 0) {
-      i64 issued = 0;
-      for (i64 t = tile_lo; t < tile_hi; ++t, ++issued) {
-        const int s = (int)(issued % kScanStages);
-        const u32 par = (u32)((issued / kScanStages) & 1);
-        if (!mbar_wait_bounded(&sm.empty[s], par ^ 1u, abort_flag)) break;
-        const i64 t0 = t * kScanTile;
-        const i64 v_lo = t0 > v_begin ? t0 : v_begin;
-        const i64 v_hi = t0 + kScanTile < v_end ? t0 + kScanTile : v_end;
-        const i64 a_lo = v_lo + (v_lo & 1), a_hi = v_hi - (v_hi & 1);
-        i64* dst = sm.stage[s];
-        // ragged first / last element (at most one each): plain loads
-        if (a_lo > v_lo) dst[v_lo - t0] = delta_aligned[v_lo];
-        if (a_hi < v_hi && v_hi - 1 >= a_lo) dst[v_hi - 1 - t0] = delta_aligned[v_hi - 1];
-        if (a_hi > a_lo) {
-          const u32 bytes = (u32)((a_hi - a_lo) * 8);
-          mbar_arrive_expect_tx(&sm.full[s], bytes);
-          bulk_load(dst + (a_lo - t0), delta_aligned + a_lo, bytes, &sm.full[s]);
-        } else {
-          mbar_arrive(&sm.full[s]);
-        }
-      }
-      // drain: every copy that was issued must have landed before the CTA exits
-      const i64 first = issued > kScanStages ? issued - kScanStages : 0;
-      for (i64 k = first; k < issued; ++k)
-        mbar_wait_bounded(&sm.full[k % kScanStages], (u32)((k / kScanStages) & 1), abort_flag);
-      if (*abort_flag) atomicExch(status_word, (u32)LLMEM_ERR_TIMEOUT);
+  // lane 0: start the copy of chunk c into stage (c - c_lo) % kScanStages
+  auto issue = [&](i64 c) {
+    const int s = (int)((c - c_lo) % kScanStages);
+    const i64 t0 = c * kScanChunk;
+    const i64 v_lo = t0 > v_begin ? t0 : v_begin;
+    const i64 v_hi = t0 + kScanChunk < v_end ? t0 + kScanChunk : v_end;
+    const i64 a_lo = v_lo + (v_lo & 1), a_hi = v_hi - (v_hi & 1);
+    i64* dst = ws.stage[s];
+    // ragged first / last element (at most one each): plain loads
+    if (a_lo > v_lo) dst[v_lo - t0] = delta_aligned[v_lo];
+    if (a_hi < v_hi && v_hi - 1 >= a_lo) dst[v_hi - 1 - t0] = delta_aligned[v_hi - 1];
+    if (a_hi > a_lo) {
+      const u32 bytes = (u32)((a_hi - a_lo) * 8);
+      mbar_arrive_expect_tx(&ws.full[s], bytes);
+      bulk_load(dst + (a_lo - t0), delta_aligned + a_lo, bytes, &ws.full[s]);
+    } else {
+      mbar_arrive(&ws.full[s]);
     }
-    return;
-  }
+  };
+  if (lane == 0)
+    for (i64 c = c_lo; c < c_hi && c < c_lo + kScanStages; ++c) issue(c);
 
-  // ---------------- consumers ----------------
-  // seg: the segment that contains the first event of the current tile
+  // seg: the segment that contains the first event of the current chunk
   i64 seg, seg_vstart, seg_vend;
   {
-    const i64 first_v = tile_lo * kScanTile > v_begin ? tile_lo * kScanTile : v_begin;
+    const i64 first_v = c_lo * kScanChunk > v_begin ? c_lo * kScanChunk : v_begin;
     i64 lo = 0, hi = n;  // smallest s with offsets[s+1] + shift > first_v
     while (lo < hi) {
       const i64 mid = lo + (hi - lo) / 2;
@@ -260,137 +260,130 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
     seg_vstart = seg < n ? __ldg(offsets + seg) + shift : v_end;
     seg_vend = seg < n ? __ldg(offsets + seg + 1) + shift : v_end;
   }
-  const i64 cta_vlo = tile_lo * kScanTile;  // segments that start at or after this started in this CTA
-  Agg run = agg_identity();                 // thread 0: fold of the current segment so far
-  int fast_parity = 0;
+  const i64 warp_vlo = c_lo * kScanChunk;  // segments that start at or after this started in this warp's range
+  Agg run = agg_identity();                // lane 0: fold of the current segment so far
+  i64 consumed = 0;
   bool aborted = false;
 
-  i64 it = 0;
-  for (i64 t = tile_lo; t < tile_hi; ++t, ++it) {
-    const int s = (int)(it % kScanStages);
-    const u32 par = (u32)((it / kScanStages) & 1);
-    const i64 t0 = t * kScanTile;
-    const i64 v_lo = t0 > v_begin ? t0 : v_begin;
-    const i64 v_hi = t0 + kScanTile < v_end ? t0 + kScanTile : v_end;
-    // On expiry the wait raises the CTA's abort flag; control still runs to the next
-    // consumer barrier, after which every consumer sees the flag and leaves together.
-    mbar_wait_bounded(&sm.full[s], par, abort_flag);
-    const i64* tile = sm.stage[s];
+  // the segment `seg` ends: store its result, or leave a partial if it began earlier
+  auto finish_segment = [&]() {
+    if (lane == 0) {
+      if (seg_vstart >= warp_vlo) write_raw(seg, run, seg_vstart, peak_out, index_out);
+      else partials[gw].head = run;
+      run = agg_identity();
+    }
+  };
+  auto next_segment = [&](i64 pos) {
+    do {
+      ++seg;
+      seg_vstart = seg < n ? __ldg(offsets + seg) + shift : v_end;
+      seg_vend = seg < n ? __ldg(offsets + seg + 1) + shift : v_end;
+    } while (seg < n && seg_vend <= pos);
+  };
 
-    if (v_lo == t0 && v_hi == t0 + kScanTile && seg < n && seg_vend >= v_hi) {
-      // ---------- fast path: the whole tile lies inside one segment ----------
-      const longlong2* src = reinterpret_cast<const longlong2*>(tile + tid * kScanPerThread);
-      longlong2 x[kScanPerThread / 2];
+  for (i64 c = c_lo; c < c_hi; ++c, ++consumed) {
+    const int s = (int)(consumed % kScanStages);
+    const u32 par = (u32)((consumed / kScanStages) & 1);
+    const i64 t0 = c * kScanChunk;
+    const i64 v_lo = t0 > v_begin ? t0 : v_begin;
+    const i64 v_hi = t0 + kScanChunk < v_end ? t0 + kScanChunk : v_end;
+    const bool ok = mbar_wait_bounded(&ws.full[s], par, abort_flag);
+    if (!__all_sync(0xffffffffu, ok)) { aborted = true; break; }
+    const i64* tile = ws.stage[s];
+
+    if (v_lo == t0 && v_hi == t0 + kScanChunk && seg < n && seg_vend >= v_hi) {
+      // ---------- fast path: the whole chunk lies inside one segment ----------
+      const longlong2* src = reinterpret_cast<const longlong2*>(tile + lane * kScanPerLane);
+      longlong2 x[kScanPerLane / 2];
 #pragma unroll
-      for (int j = 0; j < kScanPerThread / 2; ++j) x[j] = src[j];
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sm.empty[s]);  // the stage may be refilled
-      i64 sum = ev<kRound>(x[0].x), mx = sum;
-      int ix = 0;
-      {
-        sum += ev<kRound>(x[0].y);
-        if (sum > mx) { mx = sum; ix = 1; }
-      }
+      for (int j = 0; j < kScanPerLane / 2; ++j) x[j] = src[j];
+      // two independent in-order folds (events 0..9 and 10..17), then joined
+      Fold3 fa, fb;
+      fa.sum = ev<kRound>(x[0].x); fa.mx = fa.sum; fa.ix = 0;
+      fb.sum = ev<kRound>(x[5].x); fb.mx = fb.sum; fb.ix = 10;
 #pragma unroll
-      for (int j = 1; j < kScanPerThread / 2; ++j) {
-        sum += ev<kRound>(x[j].x);
-        if (sum > mx) { mx = sum; ix = 2 * j; }
-        sum += ev<kRound>(x[j].y);
-        if (sum > mx) { mx = sum; ix = 2 * j + 1; }
-      }
-      Agg g{sum, mx, t0 + (i64)tid * kScanPerThread + ix, 1};
-      g = warp_fold(g, lane);
-      if (lane == 0) sm.warp_agg[fast_parity][warp] = g;
-      consumer_barrier();
-      if (*abort_flag) { aborted = true; break; }
-      if (tid == 0) {
-#pragma unroll
-        for (int w = 0; w < kScanWarps; ++w) run = agg_fold(run, sm.warp_agg[fast_parity][w]);
-      }
-      fast_parity ^= 1;
-      if (seg_vend == v_hi) {
-        // the segment ends exactly with the tile
-        if (tid == 0) {
-          if (seg_vstart >= cta_vlo) write_raw(seg, run, seg_vstart, peak_out, index_out);
-          else partials[blockIdx.x].head = run;
-          run = agg_identity();
+      for (int j = 0; j < 5; ++j) {
+        if (j > 0) {
+          fa.sum += ev<kRound>(x[j].x);
+          if (fa.sum > fa.mx) { fa.mx = fa.sum; fa.ix = 2 * j; }
         }
-        do {
-          ++seg;
-          seg_vstart = seg < n ? __ldg(offsets + seg) + shift : v_end;
-          seg_vend = seg < n ? __ldg(offsets + seg + 1) + shift : v_end;
-        } while (seg < n && seg_vend <= v_hi);
+        fa.sum += ev<kRound>(x[j].y);
+        if (fa.sum > fa.mx) { fa.mx = fa.sum; fa.ix = 2 * j + 1; }
+      }
+#pragma unroll
+      for (int j = 5; j < 9; ++j) {
+        if (j > 5) {
+          fb.sum += ev<kRound>(x[j].x);
+          if (fb.sum > fb.mx) { fb.mx = fb.sum; fb.ix = 2 * j; }
+        }
+        fb.sum += ev<kRound>(x[j].y);
+        if (fb.sum > fb.mx) { fb.mx = fb.sum; fb.ix = 2 * j + 1; }
+      }
+      Fold3 f = fold3(fa, fb);
+      f.ix += lane * kScanPerLane;
+      // every lane has consumed its part of the stage: refill it
+      __syncwarp();
+      if (lane == 0 && c + kScanStages < c_hi) issue(c + kScanStages);
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        Fold3 o;
+        o.sum = __shfl_down_sync(0xffffffffu, f.sum, d);
+        o.mx = __shfl_down_sync(0xffffffffu, f.mx, d);
+        o.ix = __shfl_down_sync(0xffffffffu, f.ix, d);
+        if (lane + d < 32) f = fold3(f, o);
+      }
+      if (lane == 0) run = agg_fold(run, Agg{f.sum, f.mx, t0 + f.ix, 1});
+      if (seg_vend == v_hi) {
+        finish_segment();
+        next_segment(v_hi);
       }
       continue;
     }
 
-    // ---------- slow path: segment boundaries inside the tile, or a ragged tile ----------
-    if (tid == 0) {
-      sm.head = agg_identity();
-      sm.tail = agg_identity();
-    }
-    consumer_barrier();
-    // pieces: segments seg, seg+1, ... that begin before v_hi; warps take them round-robin
-    for (i64 sg = seg + warp; sg < n; sg += kScanWarps) {
-      const i64 a = __ldg(offsets + sg) + shift, b = __ldg(offsets + sg + 1) + shift;
-      if (a >= v_hi) break;
-      if (b <= a || b <= v_lo) continue;  // empty, or (only with inconsistent offsets) already past
-      const i64 pa = a > v_lo ? a : v_lo, pb = b < v_hi ? b : v_hi;
-      Agg g = warp_fold_range<kRound>(tile, (int)(pa - t0), (int)(pb - t0), lane, t0);
-      if (lane == 0) {
-        const bool starts_here = a >= v_lo, ends_here = b <= v_hi;
-        if (starts_here && ends_here) write_raw(sg, g, a, peak_out, index_out);
-        else if (!starts_here) sm.head = g;
-        else sm.tail = g;
+    // ---------- slow path: segment boundaries inside the chunk, or a ragged chunk ----------
+    i64 pos = v_lo;
+    while (pos < v_hi && seg < n) {
+      const i64 pb = seg_vend < v_hi ? seg_vend : v_hi;
+      Agg g = warp_fold_range<kRound>(tile, (int)(pos - t0), (int)(pb - t0), lane, t0);
+      if (lane == 0) run = agg_fold(run, g);
+      pos = pb;
+      if (seg_vend <= v_hi) {
+        finish_segment();
+        next_segment(pos);
       }
-    }
-    consumer_barrier();
-    if (tid == 0) {
-      // the segment that entered the tile
-      if (seg < n && seg_vstart < v_lo) {
-        run = agg_fold(run, sm.head);
-        if (seg_vend <= v_hi) {
-          if (seg_vstart >= cta_vlo) write_raw(seg, run, seg_vstart, peak_out, index_out);
-          else partials[blockIdx.x].head = run;
-          run = agg_identity();
-        }
-      }
-      // the segment that leaves the tile (it began inside it)
-      if (sm.tail.valid) run = sm.tail;
-      // which segment contains the first event of the next tile
-      i64 sg = seg;
-      while (sg < n && __ldg(offsets + sg + 1) + shift <= v_hi) ++sg;
-      sm.next_seg = sg;
     }
     __syncwarp();
-    if (lane == 0) mbar_arrive(&sm.empty[s]);
-    consumer_barrier();
-    if (*abort_flag) { aborted = true; break; }
-    seg = sm.next_seg;
-    seg_vstart = seg < n ? __ldg(offsets + seg) + shift : v_end;
-    seg_vend = seg < n ? __ldg(offsets + seg + 1) + shift : v_end;
+    if (lane == 0 && c + kScanStages < c_hi) issue(c + kScanStages);
   }
 
-  if (tid == 0 && !aborted && run.valid) {
-    // the current segment continues into the next CTA's range
-    if (seg_vstart >= cta_vlo) partials[blockIdx.x].tail = run;
-    else partials[blockIdx.x].head = run;
+  if (lane == 0) {
+    if (!aborted && run.valid) {
+      // the current segment continues into the next warp's range
+      if (seg_vstart >= warp_vlo) partials[gw].tail = run;
+      else partials[gw].head = run;
+    }
+    // drain: every copy that was issued must have landed before the warp exits
+    i64 issued = c_hi - c_lo;
+    if (issued > consumed + kScanStages) issued = consumed + kScanStages;
+    for (i64 k = consumed; k < issued; ++k)
+      mbar_wait_bounded(&ws.full[k % kScanStages], (u32)((k / kScanStages) & 1), nullptr);
+    if (aborted || *abort_flag) atomicExch(status_word, (u32)LLMEM_ERR_TIMEOUT);
   }
 }
 
-// Finish, one thread per segment: fold the partials of segments that cross CTA
+// Finish, one thread per segment: fold the partials of segments that cross warp
 // ranges, define empty segments, add m_base + lm_p, and mark inadmissible
 // configurations.
 __global__ void __launch_bounds__(256)
 scan_finish_kernel(const i64* __restrict__ offsets, i64 n, int shift, const llmem_config* __restrict__ cfg,
-                   i64* __restrict__ peak_out, i64* __restrict__ index_out, i64 tiles_per_cta,
-                   const CtaPartials* __restrict__ partials) {
+                   i64* __restrict__ peak_out, i64* __restrict__ index_out, i64 chunks_per_warp,
+                   const WarpPartials* __restrict__ partials) {
   for (i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (i64)gridDim.x * blockDim.x) {
     const i64 a = offsets[i] + shift, b = offsets[i + 1] + shift;
     i64 mx = 0, idx = -1;
     if (b > a) {
-      const i64 ca = (a / kScanTile) / tiles_per_cta, cb = ((b - 1) / kScanTile) / tiles_per_cta;
-      if (ca == cb) {  // finished by the CTA that owns it
+      const i64 ca = (a / kScanChunk) / chunks_per_warp, cb = ((b - 1) / kScanChunk) / chunks_per_warp;
+      if (ca == cb) {  // finished by the warp that owns it
         mx = peak_out[i];
         if (index_out) idx = index_out[i];
       } else {
@@ -434,37 +427,39 @@ extern "C" llmem_status llmem_scan_peak(const int64_t* delta, const int64_t* off
   }
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   u32* status_word = static_cast<u32*>(scratch);
-  CtaPartials* partials = reinterpret_cast<CtaPartials*>(static_cast<unsigned char*>(scratch) + kScratchHeader);
+  WarpPartials* partials = reinterpret_cast<WarpPartials*>(static_cast<unsigned char*>(scratch) + kScratchHeader);
   if (cudaMemsetAsync(status_word, 0, kScratchHeader, s) != cudaSuccess) return check_launch("llmem_scan_peak (memset)");
 
   const int shift = aligned_to(delta, 16) ? 0 : 1;
   const i64* delta_aligned = reinterpret_cast<const i64*>(delta) - shift;
   const bool round = (flags & LLMEM_FUSE_ROUND) != 0;
-  i64 tiles_per_cta = 1;
+  i64 chunks_per_warp = 1;
   if (total_events > 0) {
+    const size_t smem = sizeof(ScanWarpSmem) * kScanWarps;
     static thread_local int configured_dev = -1;
     int dev = 0;
     cudaGetDevice(&dev);
     if (configured_dev != dev) {
-      cudaError_t e1 = cudaFuncSetAttribute(scan_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ScanSmem));
-      cudaError_t e2 = cudaFuncSetAttribute(scan_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ScanSmem));
+      cudaError_t e1 = cudaFuncSetAttribute(scan_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      cudaError_t e2 = cudaFuncSetAttribute(scan_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e1 != cudaSuccess || e2 != cudaSuccess) return check_launch("llmem_scan_peak (shared memory opt-in)");
       configured_dev = dev;
     }
-    const i64 ntiles = (total_events + shift + kScanTile - 1) / kScanTile;
-    i64 grid = sm_count();
-    if (grid > kMaxScanCtas) grid = kMaxScanCtas;
-    if (grid > ntiles) grid = ntiles;
-    tiles_per_cta = (ntiles + grid - 1) / grid;
-    grid = (ntiles + tiles_per_cta - 1) / tiles_per_cta;
+    const i64 nchunks = (total_events + shift + kScanChunk - 1) / kScanChunk;
+    i64 warps = (i64)sm_count() * kScanWarps;
+    if (warps > kMaxScanWarps) warps = kMaxScanWarps;
+    if (warps > nchunks) warps = nchunks;
+    chunks_per_warp = (nchunks + warps - 1) / warps;
+    warps = (nchunks + chunks_per_warp - 1) / chunks_per_warp;
+    const i64 grid = (warps + kScanWarps - 1) / kScanWarps;
     if (round)
-      scan_kernel<true><<<(unsigned)grid, kScanThreads, sizeof(ScanSmem), s>>>(
+      scan_kernel<true><<<(unsigned)grid, kScanThreads, smem, s>>>(
           delta_aligned, shift, reinterpret_cast<const i64*>(offsets), n, total_events,
-          reinterpret_cast<i64*>(peak_out), reinterpret_cast<i64*>(peak_index_out), tiles_per_cta, partials, status_word);
+          reinterpret_cast<i64*>(peak_out), reinterpret_cast<i64*>(peak_index_out), chunks_per_warp, partials, status_word);
     else
-      scan_kernel<false><<<(unsigned)grid, kScanThreads, sizeof(ScanSmem), s>>>(
+      scan_kernel<false><<<(unsigned)grid, kScanThreads, smem, s>>>(
           delta_aligned, shift, reinterpret_cast<const i64*>(offsets), n, total_events,
-          reinterpret_cast<i64*>(peak_out), reinterpret_cast<i64*>(peak_index_out), tiles_per_cta, partials, status_word);
+          reinterpret_cast<i64*>(peak_out), reinterpret_cast<i64*>(peak_index_out), chunks_per_warp, partials, status_word);
     llmem_status st = check_launch("llmem_scan_peak");
     if (st != LLMEM_OK) return st;
   }
@@ -473,6 +468,6 @@ extern "C" llmem_status llmem_scan_peak(const int64_t* delta, const int64_t* off
   if (blocks > cap) blocks = cap;
   scan_finish_kernel<<<(unsigned)blocks, 256, 0, s>>>(
       reinterpret_cast<const i64*>(offsets), n, shift, cfg, reinterpret_cast<i64*>(peak_out),
-      reinterpret_cast<i64*>(peak_index_out), tiles_per_cta, partials);
+      reinterpret_cast<i64*>(peak_index_out), chunks_per_warp, partials);
   return check_launch("llmem_scan_peak (finish)");
 }
