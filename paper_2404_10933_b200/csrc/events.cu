@@ -119,13 +119,24 @@ add_block_base_kernel(i64* __restrict__ offsets, i64 n, const u64* __restrict__ 
 // ---------------------------------------------------------------------------
 // expansion
 // ---------------------------------------------------------------------------
-constexpr int kExpThreads = 256;
+// Launch shape (overridable at compile time for tuning sweeps).
+#ifndef LLMEM_EXP_THREADS
+#define LLMEM_EXP_THREADS 256
+#endif
+#ifndef LLMEM_EXP_PER_LANE
+#define LLMEM_EXP_PER_LANE 18
+#endif
+#ifndef LLMEM_EXP_CTAS_PER_SM
+#define LLMEM_EXP_CTAS_PER_SM 1
+#endif
+constexpr int kExpThreads = LLMEM_EXP_THREADS;
 constexpr int kExpWarps = kExpThreads / 32;
 // 18 events = 144 bytes = nine 16-byte words per lane: an odd word count makes
 // the per-lane spans fall on distinct shared-memory banks.
-constexpr int kExpPerLane = 18;
+constexpr int kExpPerLane = LLMEM_EXP_PER_LANE;
 constexpr int kExpChunk = 32 * kExpPerLane;  // 576 events, 4608 bytes: one warp's unit of work
-constexpr int kExpCtasPerSm = 2;
+constexpr int kExpCtasPerSm = LLMEM_EXP_CTAS_PER_SM;
+static_assert(kExpPerLane % 2 == 0 && (kExpPerLane / 2) % 2 == 1, "per-lane span: odd number of 16-byte words");
 constexpr int kRuns = 17;
 
 // A run of events that repeat with a short period: the first `split` events of each

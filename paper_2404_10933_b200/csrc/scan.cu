@@ -1,11 +1,11 @@
 // Segmented prefix-sum + max over materialised event lists (llmem_scan_peak).
 //
 // Bound by HBM reads (8 bytes per event).  The event array is cut into flat
-// 576-event chunks regardless of segment boundaries, so long and short segments
+// 832-event chunks regardless of segment boundaries, so long and short segments
 // load every SM equally.  Every warp of the persistent grid owns a contiguous range
-// of chunks and streams it on its own: lane 0 keeps four 1-D TMA bulk copies in
+// of chunks and streams it on its own: lane 0 keeps two 1-D TMA bulk copies in
 // flight into the warp's private ring of shared-memory stages, each completing on
-// an mbarrier; each lane reads 18 consecutive events from a landed stage (nine
+// an mbarrier; each lane reads 26 consecutive events from a landed stage (thirteen
 // 16-byte words, an odd count, hence conflict-free), folds them in order, and the
 // warp combines with shuffles.  The fold is the associative, non-commutative
 // operator on (sum, max prefix, arg max):  (s1,m1) + (s2,m2) = (s1+s2, max(m1, s1+m2)).
@@ -23,11 +23,24 @@
 
 namespace llmem {
 
-constexpr int kScanThreads = 256;
+// Launch shape (overridable at compile time for tuning sweeps).
+#ifndef LLMEM_SCAN_THREADS
+#define LLMEM_SCAN_THREADS 512
+#endif
+#ifndef LLMEM_SCAN_PER_LANE
+#define LLMEM_SCAN_PER_LANE 26
+#endif
+#ifndef LLMEM_SCAN_STAGES
+#define LLMEM_SCAN_STAGES 2
+#endif
+constexpr int kScanThreads = LLMEM_SCAN_THREADS;
 constexpr int kScanWarps = kScanThreads / 32;
-constexpr int kScanPerLane = 18;
-constexpr int kScanChunk = 32 * kScanPerLane;  // 576 events = 4608 bytes: one warp's unit of work
-constexpr int kScanStages = 4;                 // chunks in flight per warp
+// events per lane: twice an odd number, so that a lane's span is an odd number of
+// 16-byte words and the spans of a quarter-warp fall on distinct banks
+constexpr int kScanPerLane = LLMEM_SCAN_PER_LANE;
+constexpr int kScanChunk = 32 * kScanPerLane;  // 832 events = 6656 bytes: one warp's unit of work
+constexpr int kScanStages = LLMEM_SCAN_STAGES;  // chunks in flight per warp
+static_assert(kScanPerLane % 2 == 0 && (kScanPerLane / 2) % 2 == 1, "per-lane span: odd number of 16-byte words");
 
 struct Agg {
   i64 sum, mx, idx;  // idx: virtual (alignment-shifted) global index of the first arg max
@@ -297,12 +310,13 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
       longlong2 x[kScanPerLane / 2];
 #pragma unroll
       for (int j = 0; j < kScanPerLane / 2; ++j) x[j] = src[j];
-      // two independent in-order folds (events 0..9 and 10..17), then joined
+      // two independent in-order folds (first and second half of the span), then joined
+      constexpr int kVec = kScanPerLane / 2, kHalf = (kVec + 1) / 2;
       Fold3 fa, fb;
       fa.sum = ev<kRound>(x[0].x); fa.mx = fa.sum; fa.ix = 0;
-      fb.sum = ev<kRound>(x[5].x); fb.mx = fb.sum; fb.ix = 10;
+      fb.sum = ev<kRound>(x[kHalf].x); fb.mx = fb.sum; fb.ix = 2 * kHalf;
 #pragma unroll
-      for (int j = 0; j < 5; ++j) {
+      for (int j = 0; j < kHalf; ++j) {
         if (j > 0) {
           fa.sum += ev<kRound>(x[j].x);
           if (fa.sum > fa.mx) { fa.mx = fa.sum; fa.ix = 2 * j; }
@@ -311,8 +325,8 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
         if (fa.sum > fa.mx) { fa.mx = fa.sum; fa.ix = 2 * j + 1; }
       }
 #pragma unroll
-      for (int j = 5; j < 9; ++j) {
-        if (j > 5) {
+      for (int j = kHalf; j < kVec; ++j) {
+        if (j > kHalf) {
           fb.sum += ev<kRound>(x[j].x);
           if (fb.sum > fb.mx) { fb.mx = fb.sum; fb.ix = 2 * j; }
         }
