@@ -266,19 +266,13 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    from paper_2404_10933_b200 import multi
+
     def max_over_ranks(x: float) -> float:
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return multi.reduce_scalar(x, "max", device="cuda")
 
     def sum_over_ranks(x: float) -> float:
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.SUM)
-        return float(t.item())
+        return multi.reduce_scalar(x, "sum", device="cuda")
 
     n_cfg = args.configs
     cfgs = grids.g5_stress(0, n_cfg, seed_offset=rank)     # weak scaling: one full grid per rank
