@@ -37,11 +37,12 @@ __device__ __forceinline__ u64 sat_mul(u64 a, u64 b) {
 // ceil(x / cu_p) * cu_p; x <= 2^62 keeps the result <= 2^62
 __host__ __device__ __forceinline__ u64 page_round(u64 x) { return (x + (kPage - 1)) & ~(kPage - 1); }
 
-// signed variant: the magnitude is rounded, the sign kept
+// signed variant: the magnitude is rounded, the sign kept.  For d < 0 the result
+// -ceil(|d| / cu_p) * cu_p equals floor(d / cu_p) * cu_p, i.e. clearing the low bits of
+// the two's-complement value; for d >= 0 it is the usual add-and-mask.
 __host__ __device__ __forceinline__ i64 page_round_signed(i64 d) {
-  u64 mag = d < 0 ? (u64)0 - (u64)d : (u64)d;
-  u64 r = (mag + (kPage - 1)) & ~(kPage - 1);
-  return d < 0 ? (i64)((u64)0 - r) : (i64)r;
+  const i64 addend = ~(d >> 63) & (i64)(kPage - 1);
+  return (i64)(((u64)d + (u64)addend) & ~(kPage - 1));
 }
 
 __device__ __forceinline__ u64 ceil_div(u64 a, u64 b) { return (a + b - 1) / b; }

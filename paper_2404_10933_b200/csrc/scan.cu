@@ -25,7 +25,7 @@ namespace llmem {
 
 // Launch shape (overridable at compile time for tuning sweeps).
 #ifndef LLMEM_SCAN_THREADS
-#define LLMEM_SCAN_THREADS 512
+#define LLMEM_SCAN_THREADS 256
 #endif
 #ifndef LLMEM_SCAN_PER_LANE
 #define LLMEM_SCAN_PER_LANE 26
@@ -115,7 +115,12 @@ constexpr u64 kWaitLimitNs = 2000000000ull;  // 2 s
 // `abort_flag` (optional) shows that another lane of the warp has given up.  Returns
 // false on give-up and raises the flag.
 __device__ __forceinline__ bool mbar_wait_bounded(u64* bar, u32 parity, volatile int* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
+  // common case: the data has landed, or lands within a few polls (each try_wait
+  // already suspends the thread for a hardware-defined interval)
+#pragma unroll 1
+  for (int i = 0; i < 64; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  // rare case: keep polling against a wall-clock limit
   const u64 t0 = global_timer_ns();
   for (u32 spin = 0;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -207,6 +212,25 @@ __device__ __forceinline__ Fold3 fold3(const Fold3& a, const Fold3& b) {
   return r;
 }
 
+// In-order fold of the 16-byte words [V0, V1) of a lane's span (compile-time bounds).
+template <bool kRound, int V0, int V1>
+__device__ __forceinline__ Fold3 fold_words(const longlong2* x) {
+  Fold3 f;
+  f.sum = ev<kRound>(x[V0].x);
+  f.mx = f.sum;
+  f.ix = 2 * V0;
+#pragma unroll
+  for (int j = V0; j < V1; ++j) {
+    if (j > V0) {
+      f.sum += ev<kRound>(x[j].x);
+      if (f.sum > f.mx) { f.mx = f.sum; f.ix = 2 * j; }
+    }
+    f.sum += ev<kRound>(x[j].y);
+    if (f.sum > f.mx) { f.mx = f.sum; f.ix = 2 * j + 1; }
+  }
+  return f;
+}
+
 template <bool kRound>
 __global__ void __launch_bounds__(kScanThreads, 1)
 scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, int shift /* 0 or 1 */,
@@ -274,16 +298,41 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
     seg_vend = seg < n ? __ldg(offsets + seg + 1) + shift : v_end;
   }
   const i64 warp_vlo = c_lo * kScanChunk;  // segments that start at or after this started in this warp's range
-  Agg run = agg_identity();                // lane 0: fold of the current segment so far
+  // Fold of the current segment so far, kept distributed over the warp: `base` (the same
+  // in every lane) is the sum of all events folded; each lane remembers the best prefix
+  // value it has seen among its own events and where.  Because every lane only ever
+  // replaces its candidate by a strictly larger, later one, and the final reduction
+  // prefers the smaller index among equals, the result is the first arg max.
+  i64 base = 0, best_v = 0, best_i = 0;
+  bool lane_has = false, seg_has = false;
   i64 consumed = 0;
   bool aborted = false;
 
+  // all lanes: reduce the distributed state to one Agg (valid in every lane) and reset it
+  auto take_state = [&]() -> Agg {
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+      const i64 ov = __shfl_xor_sync(0xffffffffu, best_v, d);
+      const i64 oi = __shfl_xor_sync(0xffffffffu, best_i, d);
+      const bool oh = __shfl_xor_sync(0xffffffffu, (int)lane_has, d) != 0;
+      if (oh && (!lane_has || ov > best_v || (ov == best_v && oi < best_i))) {
+        best_v = ov;
+        best_i = oi;
+        lane_has = true;
+      }
+    }
+    Agg a{base, best_v, best_i, seg_has ? 1 : 0};
+    base = 0;
+    lane_has = false;
+    seg_has = false;
+    return a;
+  };
   // the segment `seg` ends: store its result, or leave a partial if it began earlier
   auto finish_segment = [&]() {
+    const Agg run = take_state();
     if (lane == 0) {
       if (seg_vstart >= warp_vlo) write_raw(seg, run, seg_vstart, peak_out, index_out);
       else partials[gw].head = run;
-      run = agg_identity();
     }
   };
   auto next_segment = [&](i64 pos) {
@@ -310,43 +359,30 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
       longlong2 x[kScanPerLane / 2];
 #pragma unroll
       for (int j = 0; j < kScanPerLane / 2; ++j) x[j] = src[j];
-      // two independent in-order folds (first and second half of the span), then joined
-      constexpr int kVec = kScanPerLane / 2, kHalf = (kVec + 1) / 2;
-      Fold3 fa, fb;
-      fa.sum = ev<kRound>(x[0].x); fa.mx = fa.sum; fa.ix = 0;
-      fb.sum = ev<kRound>(x[kHalf].x); fb.mx = fb.sum; fb.ix = 2 * kHalf;
-#pragma unroll
-      for (int j = 0; j < kHalf; ++j) {
-        if (j > 0) {
-          fa.sum += ev<kRound>(x[j].x);
-          if (fa.sum > fa.mx) { fa.mx = fa.sum; fa.ix = 2 * j; }
-        }
-        fa.sum += ev<kRound>(x[j].y);
-        if (fa.sum > fa.mx) { fa.mx = fa.sum; fa.ix = 2 * j + 1; }
-      }
-#pragma unroll
-      for (int j = kHalf; j < kVec; ++j) {
-        if (j > kHalf) {
-          fb.sum += ev<kRound>(x[j].x);
-          if (fb.sum > fb.mx) { fb.mx = fb.sum; fb.ix = 2 * j; }
-        }
-        fb.sum += ev<kRound>(x[j].y);
-        if (fb.sum > fb.mx) { fb.mx = fb.sum; fb.ix = 2 * j + 1; }
-      }
-      Fold3 f = fold3(fa, fb);
-      f.ix += lane * kScanPerLane;
+      // four independent in-order folds over quarters of the span, then joined
+      constexpr int kVec = kScanPerLane / 2;
+      constexpr int q1 = kVec / 4, q2 = kVec / 2, q3 = (3 * kVec) / 4;
+      const Fold3 f0 = fold_words<kRound, 0, q1>(x), f1 = fold_words<kRound, q1, q2>(x);
+      const Fold3 f2 = fold_words<kRound, q2, q3>(x), f3 = fold_words<kRound, q3, kVec>(x);
+      const Fold3 f = fold3(fold3(f0, f1), fold3(f2, f3));
       // every lane has consumed its part of the stage: refill it
       __syncwarp();
       if (lane == 0 && c + kScanStages < c_hi) issue(c + kScanStages);
+      // prefix of the lane sums across the warp
+      i64 inc = f.sum;
 #pragma unroll
       for (int d = 1; d < 32; d <<= 1) {
-        Fold3 o;
-        o.sum = __shfl_down_sync(0xffffffffu, f.sum, d);
-        o.mx = __shfl_down_sync(0xffffffffu, f.mx, d);
-        o.ix = __shfl_down_sync(0xffffffffu, f.ix, d);
-        if (lane + d < 32) f = fold3(f, o);
+        const i64 o = __shfl_up_sync(0xffffffffu, inc, d);
+        if (lane >= d) inc += o;
       }
-      if (lane == 0) run = agg_fold(run, Agg{f.sum, f.mx, t0 + f.ix, 1});
+      const i64 cand = base + (inc - f.sum) + f.mx;
+      if (!lane_has || cand > best_v) {
+        best_v = cand;
+        best_i = t0 + lane * kScanPerLane + f.ix;
+        lane_has = true;
+      }
+      base += __shfl_sync(0xffffffffu, inc, 31);
+      seg_has = true;
       if (seg_vend == v_hi) {
         finish_segment();
         next_segment(v_hi);
@@ -359,7 +395,21 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
     while (pos < v_hi && seg < n) {
       const i64 pb = seg_vend < v_hi ? seg_vend : v_hi;
       Agg g = warp_fold_range<kRound>(tile, (int)(pos - t0), (int)(pb - t0), lane, t0);
-      if (lane == 0) run = agg_fold(run, g);
+      // the piece's fold (lane 0) joins the distributed state through lane 0's candidate
+      const i64 g_sum = __shfl_sync(0xffffffffu, g.sum, 0);
+      const bool g_valid = __shfl_sync(0xffffffffu, (int)g.valid, 0) != 0;
+      if (g_valid) {
+        if (lane == 0) {
+          const i64 cand = base + g.mx;
+          if (!lane_has || cand > best_v) {
+            best_v = cand;
+            best_i = g.idx;
+            lane_has = true;
+          }
+        }
+        base += g_sum;
+        seg_has = true;
+      }
       pos = pb;
       if (seg_vend <= v_hi) {
         finish_segment();
@@ -370,6 +420,7 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
     if (lane == 0 && c + kScanStages < c_hi) issue(c + kScanStages);
   }
 
+  const Agg run = take_state();
   if (lane == 0) {
     if (!aborted && run.valid) {
       // the current segment continues into the next warp's range
