@@ -508,6 +508,20 @@ def test_max_batch_definition_and_bisect():
     assert seen_zero and seen_mid and seen_cap
 
 
+def test_capacity_equal_to_peak_fits():
+    # Algorithm 1 leaves its loop only when the peak *exceeds* m_total: a batch whose
+    # peak equals the capacity exactly still fits, the next one does not.
+    for meth in (dict(method=0), dict(method=1, gpu_n=4), dict(method=2, gpu_n=4),
+                 dict(method=3, gpu_n=8, tp_n=2)):
+        for b in (1, 5, 12):
+            c = mk(**meth, batch=b)
+            cap = oracle_peak(c)
+            for level in (1, 2):
+                bs, st = oracle.max_batch(c, [cap, cap - 1, cap + 1], 64, level=level)
+                assert st[0] == 0
+                assert bs[0].tolist() == [b, b - 1, b], (meth, b, level)
+
+
 def test_max_batch_full_range_bisect_sampled():
     cfgs = grids.g4_search_grid(7, 2)
     caps = grids.g4_capacities()
