@@ -38,6 +38,11 @@ from paper_2404_10933_b200 import grids  # noqa: E402
 METRIC = "alloc-events/sec (configs/sec in configs_per_sec, % of HBM roofline in roofline)"
 UNIT = "events/s"
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes per event (dram__bytes_read.sum + dram__bytes_write.sum over events) of the two
+# HBM-bound kernels, from the ncu capture summarised in profiles/expand_scan_g5_4096cfg_ncu.md
+# (4096 configurations; traffic grows in proportion to the number of events).  Set an entry
+# to None when its kernel changes after the capture.
+NCU_TRAFFIC_BYTES_PER_EVENT = {"expand": 7.8206, "scan": 8.0145}
 
 
 def measured_peaks():
@@ -357,7 +362,11 @@ def run_ours(args):
         "bound": "hbm", "kernel": {"expand": "expand_kernel (8 B written / event)",
                                    "scan": "scan_kernel (8 B read / event)"}[dom],
         "achieved": achieved, "peak": peak_gbs, "unit": "GB/s", "frac": achieved / peak_gbs,
-        "peak_source": peak_src, "traffic": None,
+        "peak_source": peak_src,
+        "traffic": (NCU_TRAFFIC_BYTES_PER_EVENT[dom] * hp.total
+                    if NCU_TRAFFIC_BYTES_PER_EVENT.get(dom) is not None else None),
+        "traffic_note": "ncu dram bytes per event on a 4096-configuration capture, scaled by events",
+        "algorithmic_bytes": bytes_per_launch,
         "per_kernel": {k: {"ms": kernel_ms[k], "gbs": bytes_per_launch / (kernel_ms[k] * 1e-3) / 1e9,
                            "frac": bytes_per_launch / (kernel_ms[k] * 1e-3) / 1e9 / peak_gbs}
                        for k in kernel_ms},
