@@ -39,8 +39,8 @@ METRIC = "alloc-events/sec (configs/sec in configs_per_sec, % of HBM roofline in
 UNIT = "events/s"
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per event (dram__bytes_read.sum + dram__bytes_write.sum over events) of the two
-# HBM-bound kernels, from the ncu capture summarised in profiles/expand_scan_g5_4096cfg_ncu.md
-# (4096 configurations; traffic grows in proportion to the number of events).  Set an entry
+# HBM-bound kernels, from an ncu capture of a 4096-configuration run (summary kept under
+# profiles/; traffic grows in proportion to the number of events).  Set an entry
 # to None when its kernel changes after the capture.
 NCU_TRAFFIC_BYTES_PER_EVENT = {"expand": 7.8206, "scan": 8.0145}
 

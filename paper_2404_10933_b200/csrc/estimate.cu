@@ -20,19 +20,75 @@ struct Search {
     u64 rel = relative_peak(p, s, sat_add(s.gather, dyn_sum(p, d)), first_wins);
     return sat_add(p.offset, rel);
   }
+};
+
+// The batch search of Section 6 in units of pages.  Every rounded event is a multiple
+// of cu_p = 2^21, so  peak(b) <= capacity  <=>  pages(b) <= (capacity - m_base - lm_p) >> 21.
+// Batches whose raw sizes would reach 2^62 bytes are excluded up front (they cannot fit
+// any capacity), which leaves plain, unchecked 64-bit arithmetic inside the probes; the
+// one division a probe would need, floor(out / tp) for the TP backward buffer, is done
+// with a per-configuration reciprocal.
+struct PageSearch {
+  u64 out1, logit1, shift1;  // bytes per sample of a layer output / the logits / a shifted copy
+  u64 q1, recip;             // floor(out1 / tp), ceil(2^64 / tp)
+  u64 fixed_a, fixed_b;      // pages that do not depend on the batch (see pages())
+  u64 offset;                // m_base + lm_p
+  u32 r1;                    // out1 mod tp
+  u32 n_out, n_back;         // outputs kept per iteration; TP backward buffers (0 if none or tp = 1)
+  int b_safe;                // probes stay within 1..b_safe; 0: nothing can fit
+  bool single_iter;
+
+  __device__ __forceinline__ void init(const Plan& p, const StaticSums& s, int bmax) {
+    out1 = p.out1; logit1 = p.logit1; shift1 = p.shift1;
+    offset = p.offset;
+    n_out = (u32)(p.e_n + p.L);
+    n_back = (p.tpback && p.tp > 1) ? (u32)p.L : 0u;
+    q1 = 0; r1 = 0; recip = 0;
+    if (n_back) {
+      q1 = out1 / p.tp;
+      r1 = (u32)(out1 - q1 * p.tp);
+      recip = ~0ull / p.tp + 1;  // ceil(2^64 / tp), tp >= 2
+    }
+    single_iter = p.iters < 2;
+    if (s.init >= kSat || s.os >= kSat || s.gather >= kSat) {
+      b_safe = 0;
+      fixed_a = fixed_b = 0;
+      return;
+    }
+    const u64 init_p = s.init >> 21, os_p = s.os >> 21, gat_p = s.gather >> 21;
+    // one iteration: max(init + gather + dyn, init + os); otherwise init + os + gather + dyn
+    fixed_a = single_iter ? init_p + gat_p : init_p + os_p + gat_p;
+    fixed_b = init_p + os_p;
+    const u64 big = out1 > logit1 ? out1 : logit1;  // >= 2
+    const u64 lim = (kSat - 1) / big;                // largest b with b * big < 2^62
+    b_safe = lim < (u64)bmax ? (int)lim : bmax;
+  }
+
+  __device__ __forceinline__ u64 pages(u32 b) const {
+    const u64 out = (u64)b * out1, logit = (u64)b * logit1, shift = (u64)b * shift1;
+    u64 dyn = (u64)n_out * ((out + (kPage - 1)) >> 21) + ((logit + (kPage - 1)) >> 21) +
+              2 * ((shift + (kPage - 1)) >> 21);
+    if (n_back) {
+      // floor(out / tp) = b q1 + floor(b r1 / tp); b r1 < 2^34, exact with the 64-bit reciprocal
+      const u64 back = out - ((u64)b * q1 + __umul64hi((u64)b * r1, recip));
+      dyn += (u64)n_back * ((back + (kPage - 1)) >> 21);
+    }
+    const u64 t = fixed_a + dyn;
+    return single_iter ? (t > fixed_b ? t : fixed_b) : t;
+  }
+
   // Section 6: the largest b in 1..bmax with peak(b) <= capacity.  Algorithm 1
   // increments b until the peak exceeds m_total; the peak never decreases with b,
   // so bisection finds the same b.
-  __device__ __forceinline__ int largest_batch(i64 capacity, int bmax) const {
-    int lo = 0, hi = bmax;
+  __device__ __forceinline__ int largest_batch(i64 capacity) const {
+    const u64 cap = capacity >= (i64)kSat ? kSat - 1 : (u64)(capacity < 0 ? 0 : capacity);
+    if (capacity < 0 || cap < offset) return 0;
+    const u64 budget = (cap - offset) >> 21;
+    int lo = 0, hi = b_safe;
     while (lo < hi) {
-      int mid = lo + (hi - lo + 1) / 2;
-      bool fw;
-      u64 pk = peak((u64)mid, nullptr, &fw);
-      if (pk < kSat && (i64)pk <= capacity)
-        lo = mid;
-      else
-        hi = mid - 1;
+      const int mid = lo + (hi - lo + 1) / 2;
+      if (pages((u32)mid) <= budget) lo = mid;
+      else hi = mid - 1;
     }
     return lo;
   }
@@ -92,17 +148,17 @@ max_batch_kernel(const llmem_config* __restrict__ shape, i64 n, const i64* __res
   for (i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (i64)gridDim.x * blockDim.x) {
     Cfg f = load_cfg(shape + i);
     int st = check_fields(f, false, true);
-    Search q;
+    PageSearch q;
     if (st == LLMEM_CFG_OK) {
-      q.p = make_plan(f, f.method);
-      st = q.p.status;
+      const Plan p = make_plan(f, f.method);
+      st = p.status;
+      if (st == LLMEM_CFG_OK) q.init(p, make_static_sums(p, f.pos_len > 0), bmax);
     }
     int* out = bs_out + i * n_cap;
     if (st != LLMEM_CFG_OK) {
       for (int m = 0; m < n_cap; ++m) out[m] = -1;
     } else {
-      q.s = make_static_sums(q.p, f.pos_len > 0);
-      for (int m = 0; m < n_cap; ++m) out[m] = q.largest_batch(__ldg(caps + m), bmax);
+      for (int m = 0; m < n_cap; ++m) out[m] = q.largest_batch(__ldg(caps + m));
     }
     if (status_out) status_out[i] = (uint8_t)st;
   }
@@ -124,7 +180,7 @@ select_kernel(const llmem_config* __restrict__ shape, i64 n, const i64* __restri
   for (i64 i = ((i64)blockIdx.x * blockDim.x + threadIdx.x) >> 2; i < n_warp_rounded; i += quads_per_grid) {
     const bool live = i < n;
     int st = LLMEM_CFG_FIELD;
-    Search q;
+    PageSearch q;
     bool usable = false;
     u32 gpu_n = 1, tp_n = 1;
     if (live) {
@@ -133,14 +189,14 @@ select_kernel(const llmem_config* __restrict__ shape, i64 n, const i64* __restri
       gpu_n = f.gpu_n;
       tp_n = f.tp_n;
       if (st == LLMEM_CFG_OK) {
-        q.p = make_plan(f, k);
-        usable = q.p.status == LLMEM_CFG_OK;  // a method that cannot be configured scores 0
-        if (usable) q.s = make_static_sums(q.p, f.pos_len > 0);
+        const Plan p = make_plan(f, k);
+        usable = p.status == LLMEM_CFG_OK;  // a method that cannot be configured scores 0
+        if (usable) q.init(p, make_static_sums(p, f.pos_len > 0), bmax);
       }
     }
     for (int m = 0; m < n_cap; ++m) {
       int bs = 0;
-      if (usable) bs = q.largest_batch(__ldg(caps + m), bmax);
+      if (usable) bs = q.largest_batch(__ldg(caps + m));
       int b0 = __shfl_sync(0xffffffffu, bs, quad_base + 0);
       int b1 = __shfl_sync(0xffffffffu, bs, quad_base + 1);
       int b2 = __shfl_sync(0xffffffffu, bs, quad_base + 2);

@@ -247,3 +247,43 @@ def test_aligned_family_on_device(llmem):
     got = llmem.estimate_batch(c)
     assert np.array_equal(got["peak"].cpu().numpy(), want["peak"])
     assert ((want["peak"] - 123456789 - 65536 * 2048 * 2) % G == 0).all()
+
+
+def test_search_edge_capacities_and_ranges(llmem):
+    """Capacities below the fixed part, equal to a peak, one byte less, negative, at and
+    beyond 2^62; one-iteration lists; TP on a single device; the largest admissible bmax."""
+    base = grids.g4_search_grid(3, 2)                       # 2 shapes x 4 methods x 16 degrees
+    one_iter = base.copy(); one_iter["iters"] = 1
+    tiny = base[:32].copy()
+    tiny["layers"], tiny["hidden"], tiny["heads"], tiny["ffn"], tiny["vocab"] = 1, 64, 1, 256, 1000
+    tiny["seq"], tiny["chunk_elems"], tiny["base_bytes"] = 1, 1 << 20, 0   # zero-byte shifted copies
+    shapes = np.concatenate([base, one_iter, tiny])
+    probe = shapes.copy(); probe["batch"] = 3
+    est = oracle.estimate(probe, level=2)
+    exact = est["peak"][est["status"] == 0]
+    caps = np.array([-5, 0, 1, int(exact.min()), int(exact.min()) - 1, int(np.median(exact)),
+                     int(exact.max()), int(exact.max()) - 1, (1 << 62) - 1, 1 << 62, (1 << 63) - 1,
+                     16 << 30, 80 << 30], dtype=np.int64)
+    for bmax in (1, 7, 1 << 26):
+        want_bs, want_st = oracle.max_batch(shapes, caps, bmax, level=2, threads=8)
+        got_bs, got_st = llmem.max_batch(shapes, caps, bmax)
+        assert np.array_equal(got_st.cpu().numpy(), want_st)
+        assert np.array_equal(got_bs.cpu().numpy(), want_bs), bmax
+    want_bs, _ = oracle.max_batch(shapes, caps, 9, level=1, threads=8)
+    got_bs, _ = llmem.max_batch(shapes, caps, 9)
+    assert np.array_equal(got_bs.cpu().numpy(), want_bs)
+    # a capacity equal to the peak at batch 3 admits exactly batch 3 (strict exit test)
+    ok = np.flatnonzero(est["status"] == 0)[::7]
+    for i in ok:
+        cap = np.array([int(est["peak"][i])], dtype=np.int64)
+        got, _ = llmem.max_batch(shapes[i:i + 1], cap, 64)
+        want, _ = oracle.max_batch(shapes[i:i + 1], cap, 64, level=1)
+        assert got.cpu().numpy().tolist() == want.tolist()
+        assert want[0, 0] >= 3
+    sel_shapes = np.concatenate([grids.g4_select_grid(3, 2), grids.g4_select_grid(5, 1)])
+    sel_shapes["iters"][::3] = 1
+    for allzero in (False, True):
+        want = oracle.select_method(sel_shapes, caps, 1 << 26, flags=1 if allzero else 0, level=2, threads=8)
+        got = llmem.select_method(sel_shapes, caps, 1 << 26, allzero=allzero)
+        for k in ("method", "batch", "bs_list", "status"):
+            assert np.array_equal(got[k].cpu().numpy(), want[k]), k
