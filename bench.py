@@ -399,6 +399,99 @@ def run_ours(args):
     return 0 if agree else 4
 
 
+# ---------------------------------------------------------------------------
+# secondary workloads: the kernels that generate events in registers (integer-ALU bound)
+# ---------------------------------------------------------------------------
+# Warp instructions executed per unit of work (smsp__inst_executed.sum / units) from ncu
+# captures of these kernels on reduced grids; None once a kernel changes after the capture.
+NCU_WARP_INSTR_PER_UNIT = {"estimate_kernel": 44.81, "max_batch_kernel": 24.70, "select_kernel": 127.83}
+
+
+def run_register_paths(args):
+    """--workload g3: fused estimate over the 2^20-configuration sweep.
+    --workload g4: largest-batch search (2^17 shapes x 4 methods x 16 degrees x 9 capacities)
+    and Algorithm 1 selection (2^17 shapes x 16 degrees x 9 capacities).
+    Inputs are resident in HBM; L2 is flushed between timed steps (the g3 input is smaller
+    than L2).  Reports units/s and the issue-rate (integer ALU) roofline."""
+    import torch
+    import paper_2404_10933_b200 as llmem
+    llmem.lib()
+    torch.cuda.set_device(0)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    caps_np = grids.g4_capacities()
+    caps = torch.from_numpy(caps_np).cuda()
+    if args.workload == "g3":
+        n = min(args.configs, grids.G3_CONFIGS) if args.configs != grids.G5_CONFIGS else grids.G3_CONFIGS
+        host = [grids.g3_sweep(0, n)]
+        dev = [llmem.to_device(host[0])]
+        events = int(torch.diff(llmem.event_counts(dev[0])[0]).sum().item())
+        units = {"estimate_kernel": n}
+
+        def step():
+            return llmem.estimate_batch(dev[0])
+        unit_name, n_units, extra = "configs/s", n, {"virtual_events_per_config": events / n}
+        workload = "G3 large sweep: fused estimate, event runs summed in registers (no list materialised)"
+        launches = 1
+    else:
+        shapes = min(args.configs, grids.G4_SHAPES) if args.configs != grids.G5_CONFIGS else grids.G4_SHAPES
+        host = [grids.g4_search_grid(0, shapes), grids.g4_select_grid(0, shapes)]
+        dev = [llmem.to_device(h) for h in host]
+        units = {"max_batch_kernel": len(host[0]) * len(caps_np), "select_kernel": len(host[1]) * len(caps_np)}
+
+        def step():
+            a = llmem.max_batch(dev[0], caps, grids.G4_BMAX, want_status=False)
+            b = llmem.select_method(dev[1], caps, grids.G4_BMAX, want_bs_list=False, want_status=False)
+            return a, b
+        unit_name, n_units, extra = "searches/s", units["max_batch_kernel"] + 4 * units["select_kernel"], {
+            "selections": units["select_kernel"]}
+        workload = "G4 max-batch search + Algorithm 1 selection, bisection on batch 1..4096 in registers"
+        launches = 2
+    for _ in range(max(args.warmup, 3)):
+        step()
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(0).uuid)
+    except Exception:
+        gpu_id = "0"
+    sampler = ClockSampler(gpu_id)
+    sampler.start()
+    time.sleep(0.3)
+    torch.cuda.synchronize()
+    wall0 = time.time()
+    total_ms = 0.0
+    for _ in range(args.steps):
+        flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        step()
+        e1.record()
+        torch.cuda.synchronize()
+        total_ms += e0.elapsed_time(e1)
+    wall1 = time.time()
+    clocks = sampler.stop(wall0, wall1)
+    ms = total_ms / args.steps
+    # issue-rate roofline: 4 schedulers per SM, one warp instruction per cycle each
+    sm = torch.cuda.get_device_properties(0).multi_processor_count
+    mhz = clocks.get("sm_mhz") or 1965.0
+    peak = sm * 4 * mhz * 1e6
+    instr = None
+    if all(NCU_WARP_INSTR_PER_UNIT.get(k) is not None for k in units):
+        instr = sum(NCU_WARP_INSTR_PER_UNIT[k] * u for k, u in units.items())
+    line = {
+        "metric": f"{unit_name.split('/')[0]} per second ({args.workload})", "value": n_units / (ms * 1e-3),
+        "unit": unit_name, "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+        "config": {"workload": workload, "l2": "256 MB write between timed steps flushes L2", **extra},
+        "roofline": {"bound": "alu", "unit": "warp-instr/s", "peak": peak,
+                     "achieved": (instr / (ms * 1e-3)) if instr else None,
+                     "frac": (instr / (ms * 1e-3) / peak) if instr else None,
+                     "peak_source": "148 SMs x 4 schedulers x sampled SM clock (one warp instruction per cycle each)",
+                     "traffic": None},
+        "gpu_launches": launches * args.steps, "clocks": clocks,
+    }
+    print(json.dumps(line))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -408,9 +501,13 @@ def main():
     ap.add_argument("--configs", type=int, default=grids.G5_CONFIGS,
                     help="configurations of the stress grid per GPU (default: the full grid)")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--workload", choices=("g5", "g3", "g4"), default="g5",
+                    help="g5 (default): the full hot path on the stress grid; g3 / g4: the in-register kernels")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.workload != "g5":
+        return run_register_paths(args)
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if world == 1 and args.gpus > 1:
         # launched without torchrun: re-launch one rank per GPU
