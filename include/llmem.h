@@ -210,6 +210,29 @@ llmem_status llmem_select_method(const llmem_config* DEV shape, int64_t n,
                                  void* DEV scratch, size_t scratch_bytes, uint32_t flags,
                                  void* cuda_stream);
 
+/* Section 6 (scores and tie order of Algorithm 1) applied to candidate lists of any
+ * length; Section 7.4 notes that DP+TP admits several splits once more devices are at
+ * hand.  A group is a run of consecutive candidates, each a (method, gpu_n, tp_n) with its
+ * largest batch per capacity as written by llmem_max_batch: for instance every method,
+ * every degree up to the devices available and every admissible DP+TP split of one
+ * decoder shape.  Scores as in Algorithm 1 (CDP 1.5 bs gpu_n, ADP bs gpu_n, TP bs, DP+TP
+ * bs gpu_n/tp_n); a candidate with bs <= 0 scores 0; the first candidate with the largest
+ * score wins; if all scores are 0 (or the group is empty) the result is CPU offloading.
+ * The candidates are not checked for out-of-bounds group_offsets: these must be
+ * non-decreasing and end at n_items.
+ *   item_cfg      DEV [n_items]      method, gpu_n, tp_n read
+ *   bs            DEV [n_items][n_cap]
+ *   group_offsets DEV [n_groups+1]
+ *   item_out      DEV [n_groups][n_cap]  index of the winning candidate, -1 = offloading
+ *   method_out    DEV [n_groups][n_cap]  nullable; its method, LLMEM_METHOD_OFFLOAD if none
+ *   batch_out     DEV [n_groups][n_cap]  nullable; its batch, 0 if none */
+llmem_status llmem_select_segmented(const llmem_config* DEV item_cfg, const int32_t* DEV bs,
+                                    const int64_t* DEV group_offsets, int64_t n_groups,
+                                    int64_t n_items, int32_t n_cap, int64_t* DEV item_out,
+                                    int32_t* DEV method_out, int32_t* DEV batch_out,
+                                    void* DEV scratch, size_t scratch_bytes, uint32_t flags,
+                                    void* cuda_stream);
+
 /* Synchronises cuda_stream and returns the device status word that
  * llmem_scan_peak keeps at the start of its scratch: LLMEM_OK, or
  * LLMEM_ERR_TIMEOUT if a bounded wait inside a kernel gave up (outputs are then

@@ -170,3 +170,19 @@ def decide(bs_list, gpu_n: int, tp_n: int, flags: int = 0) -> tuple[int, int]:
     lib().oracle_decide(_p(bl), ctypes.c_int32(gpu_n), ctypes.c_int32(tp_n),
                         ctypes.c_uint32(flags), ctypes.byref(m), ctypes.byref(b))
     return int(m.value), int(b.value)
+
+
+def select_segmented(item_cfg: np.ndarray, bs: np.ndarray, group_offsets):
+    """Decision of Algorithm 1 over arbitrary candidate groups.
+    Returns dict(item[n_groups, n_cap] int64, method, batch int32)."""
+    item_cfg = _cfgs(item_cfg)
+    bs = np.ascontiguousarray(bs, dtype=np.int32)
+    assert bs.ndim == 2 and bs.shape[0] == item_cfg.size
+    offs = np.ascontiguousarray(group_offsets, dtype=np.int64)
+    n_groups, n_cap = offs.size - 1, bs.shape[1]
+    item = np.full((n_groups, n_cap), -2, dtype=np.int64)
+    method = np.full((n_groups, n_cap), -2, dtype=np.int32)
+    batch = np.full((n_groups, n_cap), -2, dtype=np.int32)
+    lib().oracle_select_segmented(_p(item_cfg), _p(bs), _p(offs), ctypes.c_int64(n_groups),
+                                  ctypes.c_int32(n_cap), _p(item), _p(method), _p(batch))
+    return {"item": item, "method": method, "batch": batch}

@@ -749,3 +749,48 @@ void oracle_select_many(const oracle_config *cfg, int64_t n, const int64_t *caps
   j.status = status;
   run_job(&j, nthreads);
 }
+
+/* ------------------------------------------------------------------------ */
+/* extension: the decision of Algorithm 1 over an arbitrary candidate list  */
+/* ------------------------------------------------------------------------ */
+/* Section 6 scores a fixed list of four candidates.  Here a group holds any number
+ * of candidates (method, gpu_n, tp_n), each with its largest batch per capacity, e.g.
+ * every DP+TP split of every degree up to the number of devices at hand (Section 7.4
+ * remarks that DP+TP admits several combinations).  Score of a candidate, as in
+ * Algorithm 1: CDP 1.5 bs gpu_n, ADP bs gpu_n, TP bs, DP+TP bs gpu_n / tp_n; a
+ * candidate with bs <= 0 (does not fit, or not admissible) scores 0.  The first
+ * candidate with the largest score wins; if every score is 0 the answer is CPU
+ * offloading: item -1, method 4, batch 0.
+ *   item_cfg[n_items]        method, gpu_n, tp_n read
+ *   bs[n_items][n_cap]
+ *   group_offsets[n_groups+1] items of group g are [group_offsets[g], group_offsets[g+1])
+ *   outputs [n_groups][n_cap] */
+void oracle_select_segmented(const oracle_config *item_cfg, const int32_t *bs,
+                             const int64_t *group_offsets, int64_t n_groups, int32_t n_cap,
+                             int64_t *item_out, int32_t *method_out, int32_t *batch_out) {
+  for (int64_t g = 0; g < n_groups; ++g) {
+    for (int32_t m = 0; m < n_cap; ++m) {
+      int64_t best_item = -1;
+      i128 best_score = 0; /* doubled */
+      for (int64_t i = group_offsets[g]; i < group_offsets[g + 1]; ++i) {
+        const oracle_config *c = item_cfg + i;
+        int64_t b = bs[i * n_cap + m];
+        i128 score2 = 0;
+        if (b > 0) {
+          if (c->method == M_CDP) score2 = (i128)3 * b * c->gpu_n;
+          else if (c->method == M_ADP) score2 = (i128)2 * b * c->gpu_n;
+          else if (c->method == M_TP) score2 = (i128)2 * b;
+          else if (c->method == M_DPTP && c->tp_n > 0) score2 = (i128)2 * b * (c->gpu_n / c->tp_n);
+        }
+        if (score2 > best_score) { /* strict: the first of equals stays */
+          best_score = score2;
+          best_item = i;
+        }
+      }
+      int64_t o = g * n_cap + m;
+      item_out[o] = best_item;
+      method_out[o] = best_item >= 0 ? item_cfg[best_item].method : 4;
+      batch_out[o] = best_item >= 0 ? bs[best_item * n_cap + m] : 0;
+    }
+  }
+}

@@ -33,6 +33,7 @@ EXPORTS = (
     "llmem_scratch_bytes", "llmem_estimate_batch", "llmem_event_counts", "llmem_expand_events",
     "llmem_round_events", "llmem_scan_peak", "llmem_max_batch", "llmem_select_method",
     "llmem_scratch_status", "llmem_last_error", "llmem_version", "llmem_event_counts_static",
+    "llmem_select_segmented",
 )
 STATIC_MAX_CONFIGS = 4194304
 
@@ -67,6 +68,7 @@ def lib() -> ctypes.CDLL:
         L.llmem_scan_peak.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, sz, u32, vp]
         L.llmem_max_batch.argtypes = [vp, i64, vp, i32, i32, vp, vp, vp, sz, u32, vp]
         L.llmem_select_method.argtypes = [vp, i64, vp, i32, i32, vp, vp, vp, vp, vp, sz, u32, vp]
+        L.llmem_select_segmented.argtypes = [vp, vp, vp, i64, i64, i32, vp, vp, vp, vp, sz, u32, vp]
         L.llmem_scratch_status.argtypes = [vp, vp]
         L.llmem_last_error.restype = ctypes.c_char_p
         L.llmem_version.restype = ctypes.c_int
@@ -252,6 +254,26 @@ def select_method(shape, capacities, bmax: int, *, allzero: bool = False, want_b
                                      _ptr(bs_list), _ptr(status), None, 0,
                                      SELECT_ALLZERO if allzero else 0, _stream_ptr(stream)))
     return {"method": method, "batch": batch, "bs_list": bs_list, "status": status}
+
+
+def select_segmented(item_cfg, bs, group_offsets, *, stream=None):
+    """Algorithm 1's decision over arbitrary candidate groups.  ``bs`` is the [n_items, n_cap]
+    matrix written by ``max_batch`` for ``item_cfg``; ``group_offsets`` ([n_groups+1] int64)
+    delimits the groups.  Returns dict(item[n_groups, n_cap] int64, method, batch int32)."""
+    torch = _torch()
+    item_cfg = _as_cfg(item_cfg)
+    n_items, n_cap = bs.shape
+    if not isinstance(group_offsets, torch.Tensor):
+        group_offsets = torch.as_tensor(np.asarray(group_offsets, dtype=np.int64))
+    group_offsets = group_offsets.to(device=item_cfg.device, dtype=torch.int64).contiguous()
+    n_groups = group_offsets.numel() - 1
+    item = torch.empty((n_groups, n_cap), dtype=torch.int64, device=item_cfg.device)
+    method = torch.empty((n_groups, n_cap), dtype=torch.int32, device=item_cfg.device)
+    batch = torch.empty((n_groups, n_cap), dtype=torch.int32, device=item_cfg.device)
+    _check(lib().llmem_select_segmented(_ptr(item_cfg), _ptr(bs.contiguous()), _ptr(group_offsets), n_groups,
+                                        n_items, n_cap, _ptr(item), _ptr(method), _ptr(batch), None, 0, 0,
+                                        _stream_ptr(stream)))
+    return {"item": item, "method": method, "batch": batch}
 
 
 def _caps(capacities, device):

@@ -228,6 +228,47 @@ select_kernel(const llmem_config* __restrict__ shape, i64 n, const i64* __restri
   }
 }
 
+// ---------------------------------------------------------------------------
+// llmem_select_segmented: the decision of Algorithm 1 over arbitrary candidate groups.
+// One thread per (group, capacity); capacities vary fastest so that a warp reads
+// contiguous rows of the batch matrix.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+select_segmented_kernel(const llmem_config* __restrict__ item_cfg, const int* __restrict__ bs,
+                        const i64* __restrict__ group_offsets, i64 n_groups, int n_cap,
+                        i64* __restrict__ item_out, int* __restrict__ method_out, int* __restrict__ batch_out) {
+  const i64 total = n_groups * n_cap;
+  for (i64 o = (i64)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (i64)gridDim.x * blockDim.x) {
+    const i64 g = o / n_cap;
+    const int m = (int)(o - g * n_cap);
+    const i64 lo = __ldg(group_offsets + g), hi = __ldg(group_offsets + g + 1);
+    i64 best_item = -1;
+    u64 best_score = 0;  // doubled, so that CDP's factor 1.5 stays integral
+    int best_method = LLMEM_METHOD_OFFLOAD, best_batch = 0;
+    for (i64 i = lo; i < hi; ++i) {
+      const int b = __ldg(bs + i * n_cap + m);
+      if (b <= 0) continue;  // does not fit, or not admissible: score 0
+      // bytes 48..51 of the record: method, gpu_n, tp_n, lm_bytes
+      const u32 w = __ldg(reinterpret_cast<const u32*>(item_cfg + i) + 12);
+      const u32 method = w & 0xff, n = (w >> 8) & 0xff, t = (w >> 16) & 0xff;
+      u64 score = 0;
+      if (method == LLMEM_METHOD_CDP) score = 3ull * (u64)b * n;
+      else if (method == LLMEM_METHOD_ADP) score = 2ull * (u64)b * n;
+      else if (method == LLMEM_METHOD_TP) score = 2ull * (u64)b;
+      else if (method == LLMEM_METHOD_DPTP && t > 0) score = 2ull * (u64)b * (n / t);
+      if (score > best_score) {  // strict: the first of equals stays
+        best_score = score;
+        best_item = i;
+        best_method = (int)method;
+        best_batch = b;
+      }
+    }
+    item_out[o] = best_item;
+    if (method_out) method_out[o] = best_method;
+    if (batch_out) batch_out[o] = best_batch;
+  }
+}
+
 static int grid_for(i64 threads_needed, int block, int ctas_per_sm) {
   i64 blocks = (threads_needed + block - 1) / block;
   i64 cap = (i64)sm_count() * ctas_per_sm;
@@ -296,4 +337,27 @@ extern "C" llmem_status llmem_select_method(const llmem_config* shape, int64_t n
       shape, n, reinterpret_cast<const i64*>(capacity_bytes), n_cap, bmax, flags, method_out,
       batch_out, bs_list_out, status_out);
   return check_launch("llmem_select_method");
+}
+
+extern "C" llmem_status llmem_select_segmented(const llmem_config* item_cfg, const int32_t* bs,
+                                               const int64_t* group_offsets, int64_t n_groups,
+                                               int64_t n_items, int32_t n_cap, int64_t* item_out,
+                                               int32_t* method_out, int32_t* batch_out, void* scratch,
+                                               size_t scratch_bytes, uint32_t flags, void* cuda_stream) {
+  (void)scratch; (void)scratch_bytes; (void)flags;
+  clear_error();
+  if (n_groups < 0 || n_items < 0 || n_cap < 0) { set_error("llmem_select_segmented: negative size"); return LLMEM_ERR_ARG; }
+  if (n_groups == 0 || n_cap == 0) return LLMEM_OK;
+  if (!group_offsets || !item_out || (n_items > 0 && (!item_cfg || !bs))) {
+    set_error("llmem_select_segmented: item_cfg, bs, group_offsets and item_out are required");
+    return LLMEM_ERR_ARG;
+  }
+  if (!aligned_to(item_cfg, 16) || !aligned_to(bs, 4) || !aligned_to(group_offsets, 8) || !aligned_to(item_out, 8)) {
+    set_error("llmem_select_segmented: misaligned pointer");
+    return LLMEM_ERR_ARG;
+  }
+  select_segmented_kernel<<<grid_for(n_groups * n_cap, 256, 8), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      item_cfg, bs, reinterpret_cast<const i64*>(group_offsets), n_groups, n_cap,
+      reinterpret_cast<i64*>(item_out), method_out, batch_out);
+  return check_launch("llmem_select_segmented");
 }

@@ -263,6 +263,28 @@ def g4_select_grid(first: int = 0, count: int = G4_SHAPES) -> np.ndarray:
     return c
 
 
+def all_split_candidates(n_max: int = G4_DEGREES) -> list[tuple[int, int, int]]:
+    """Every (method, gpu_n, tp_n) candidate on up to n_max devices, ordered by degree,
+    then CDP, ADP, TP, then the DP+TP splits by increasing tp_n (67 candidates for 16)."""
+    out = []
+    for n in range(1, n_max + 1):
+        out += [(METHOD_CDP, n, 0), (METHOD_ADP, n, 0), (METHOD_TP, n, 0)]
+        out += [(METHOD_DPTP, n, t) for t in valid_tp_degrees(n)]
+    return out
+
+
+def g4_all_splits_grid(first: int = 0, count: int = G4_SHAPES, n_max: int = G4_DEGREES):
+    """Configs ordered [shape][candidate] and the group offsets (one group per shape)."""
+    shapes = g4_shapes(first, count)
+    cand = np.asarray(all_split_candidates(n_max), dtype=np.int64)
+    k = len(cand)
+    c = np.repeat(shapes, k)
+    c["method"] = np.tile(cand[:, 0], count)
+    c["gpu_n"] = np.tile(cand[:, 1], count)
+    c["tp_n"] = np.tile(cand[:, 2], count)
+    return c, np.arange(count + 1, dtype=np.int64) * k
+
+
 # --------------------------------------------------------------------------
 # G5: deep/wide stress grid with long event lists
 # --------------------------------------------------------------------------

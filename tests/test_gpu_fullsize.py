@@ -137,3 +137,29 @@ def test_g5_stress_materialized_full(llmem):
     for i in idx[:6]:
         ev = oracle.round_events(oracle.expand_events(cfgs[i:i + 1]))
         assert np.array_equal(delta[off[i]:off[i + 1]].cpu().numpy(), ev)
+
+
+def test_g4_selection_over_all_degrees_and_splits(llmem):
+    """Per shape and capacity, the best of 67 candidates: CDP / ADP / TP on 1..16 devices and
+    every admissible DP+TP split.  The CUDA pipeline (max_batch on all 8.8 M candidates, then
+    the segmented decision) runs at full size; every fourth shape is compared with the oracle
+    end to end (its own batches, its own decision)."""
+    caps = grids.g4_capacities()
+    cand, offsets = grids.g4_all_splits_grid()
+    k = len(grids.all_split_candidates())
+    assert k == 67 and len(cand) == (1 << 17) * k
+    dev = llmem.to_device(cand)
+    bs, st = llmem.max_batch(dev, caps, grids.G4_BMAX)
+    got = llmem.select_segmented(dev, bs, offsets)
+    assert int(st.max()) == 0
+    sub = np.arange(0, 1 << 17, 4)
+    rows = (sub[:, None] * k + np.arange(k)[None, :]).reshape(-1)
+    want_bs, _ = oracle.max_batch(cand[rows], caps, grids.G4_BMAX, level=2, threads=THREADS)
+    assert np.array_equal(bs.cpu().numpy()[rows], want_bs)
+    want = oracle.select_segmented(cand[rows], want_bs, np.arange(len(sub) + 1, dtype=np.int64) * k)
+    item = got["item"].cpu().numpy()[sub]
+    local = np.where(item >= 0, item - (sub * k)[:, None], -1)
+    assert np.array_equal(local, np.where(want["item"] >= 0, want["item"] - (np.arange(len(sub)) * k)[:, None], -1))
+    assert np.array_equal(got["method"].cpu().numpy()[sub], want["method"])
+    assert np.array_equal(got["batch"].cpu().numpy()[sub], want["batch"])
+    assert set(np.unique(want["method"]).tolist()) >= {0, 1, 4}

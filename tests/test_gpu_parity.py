@@ -287,3 +287,22 @@ def test_search_edge_capacities_and_ranges(llmem):
         got = llmem.select_method(sel_shapes, caps, 1 << 26, allzero=allzero)
         for k in ("method", "batch", "bs_list", "status"):
             assert np.array_equal(got[k].cpu().numpy(), want[k]), k
+
+
+def test_segmented_selection_random_groups(llmem):
+    rng = np.random.default_rng(10933)
+    sizes = rng.integers(0, 40, size=300)
+    sizes[[0, 17, 299]] = 0                              # empty groups, first and last included
+    offsets = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    n_items, n_cap = int(offsets[-1]), 7
+    items = grids.empty(n_items)
+    items["method"] = rng.integers(0, 6, size=n_items)   # 4 and 5 are not methods: score 0
+    items["gpu_n"] = rng.integers(1, 64, size=n_items)
+    items["tp_n"] = rng.integers(0, 9, size=n_items)     # 0 with DP+TP: score 0
+    bs = rng.integers(-1, 6, size=(n_items, n_cap)).astype(np.int32)   # many ties
+    bs[rng.random((n_items, n_cap)) < 0.05] = 1 << 26
+    want = oracle.select_segmented(items, bs, offsets)
+    got = llmem.select_segmented(items, torch.from_numpy(bs).cuda(), offsets)
+    for k in ("item", "method", "batch"):
+        assert np.array_equal(got[k].cpu().numpy(), want[k]), k
+    assert (want["item"] == -1).any() and (want["method"] == 3).any()

@@ -52,6 +52,10 @@ MUTANTS = [
     ("collapsed_os_count", "(u128)z->L * (4 * page_round(z->os_hh) + (u128)(z->K - 4) * page_round(z->os_hf));",
      "(u128)z->L * (4 * page_round(z->os_hh) + (u128)(z->K - 5) * page_round(z->os_hf));", 1),
     ("tp_without_backward_buffers", "z->tpback = (c->method == M_TP || c->method == M_DPTP);", "z->tpback = (c->method == M_DPTP);", 1),
+    ("segmented_tie_prefers_later", "if (score2 > best_score) { /* strict: the first of equals stays */",
+     "if (score2 >= best_score && score2 > 0) {", 1),
+    ("segmented_dp_degree", "score2 = (i128)2 * b * (c->gpu_n / c->tp_n);", "score2 = (i128)2 * b * c->tp_n;", 1),
+    ("segmented_cdp_factor", "score2 = (i128)3 * b * c->gpu_n;", "score2 = (i128)2 * b * c->gpu_n;", 1),
     ("frees_forgotten_gather", "      for (int64_t j = 0; j < C; ++j) emit(s, -1, z->gat_chunk);\n", "", 1),
 ]
 

@@ -592,3 +592,57 @@ def test_llama7b_on_four_16gib_devices_offloads(golden_dir):
                 sel = oracle.select_method(c, [16384 << 20], 8, flags=flags, level=2)
                 assert (int(sel["method"][0, 0]), int(sel["batch"][0, 0])) == (4, 0)
                 assert sel["bs_list"][0, 0].tolist() == [0, 0, 0, 0]
+
+
+# --------------------------------------------------------------------------
+# extension: Algorithm 1's decision over arbitrary candidate groups
+# --------------------------------------------------------------------------
+def _items(triples):
+    c = grids.empty(len(triples))
+    c["layers"] = c["hidden"] = c["heads"] = c["ffn"] = c["vocab"] = c["seq"] = 1
+    for i, (m, n, t) in enumerate(triples):
+        c["method"][i], c["gpu_n"][i], c["tp_n"][i] = m, n, t
+    return c
+
+
+def test_segmented_selection_reduces_to_algorithm1(golden_dir):
+    """With the four candidates of Algorithm 1 in its order, the segmented decision is the
+    hand-worked decision (cases where both offload rules agree, or the prose rule)."""
+    used = 0
+    for line in open(f"{golden_dir}/algorithm1_decisions.txt"):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        lhs, rhs = line.split("->")
+        b0, b1, b2, b3, n, t, flags = (int(x) for x in lhs.split())
+        if flags == 0 and b2 == 0:
+            continue                      # literal rule offloads although something fits
+        want_method, want_batch = (int(x) for x in rhs.split())
+        items = _items([(0, n, 0), (1, n, 0), (2, n, 0), (3, n, t)])
+        bs = np.array([[b0], [b1], [b2], [b3]], dtype=np.int32)
+        r = oracle.select_segmented(items, bs, [0, 4])
+        assert (int(r["method"][0, 0]), int(r["batch"][0, 0])) == (want_method, want_batch), line
+        assert int(r["item"][0, 0]) == (want_method if want_method < 4 else -1)
+        used += 1
+    assert used >= 12
+
+
+def test_segmented_selection_hand_cases():
+    # candidates on 8 devices: CDP, ADP, TP, DP+TP with tp 2 (dp 4) and tp 4 (dp 2)
+    items = _items([(0, 8, 0), (1, 8, 0), (2, 8, 0), (3, 8, 2), (3, 8, 4)])
+    cases = [
+        ([0, 0, 9, 3, 4], (3, 3, 3)),     # scores x2: 0 0 18 24 16 -> the tp-2 split
+        ([0, 0, 0, 2, 4], (3, 3, 2)),     # 16 = 16: the earlier split wins
+        ([0, 0, 13, 3, 4], (2, 2, 13)),   # TP 26 beats 24
+        ([2, 1, 13, 3, 5], (0, 0, 2)),    # CDP 1.5*2*8 = 24, doubled 48, beats ADP 16, TP 26, DP+TP 24 / 20
+        ([-1, -1, -1, -1, -1], (-1, 4, 0)),
+        ([0, 0, 0, 0, 0], (-1, 4, 0)),
+    ]
+    bs = np.array([c[0] for c in cases], dtype=np.int32).T.copy()   # [items][cases as capacities]
+    r = oracle.select_segmented(items, bs, [0, 5])
+    for k, (_, (item, method, batch)) in enumerate(cases):
+        assert (int(r["item"][0, k]), int(r["method"][0, k]), int(r["batch"][0, k])) == (item, method, batch), k
+    # several groups, one of them empty; item indices are global
+    r = oracle.select_segmented(items, bs[:, :2], [0, 0, 3, 5])
+    assert r["item"][:, 0].tolist() == [-1, 2, 3] and r["method"][:, 0].tolist() == [4, 2, 3]
+    assert r["item"][:, 1].tolist() == [-1, -1, 3]
