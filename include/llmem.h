@@ -86,7 +86,7 @@ enum { LLMEM_CFG_OK = 0, LLMEM_CFG_FIELD = 1 /* a field outside its range */,
 
 /* operations, for llmem_scratch_bytes */
 enum { LLMEM_OP_ESTIMATE = 0, LLMEM_OP_EVENT_COUNTS = 1, LLMEM_OP_EXPAND = 2, LLMEM_OP_ROUND = 3,
-       LLMEM_OP_SCAN_PEAK = 4, LLMEM_OP_MAX_BATCH = 5, LLMEM_OP_SELECT = 6 };
+       LLMEM_OP_SCAN_PEAK = 4, LLMEM_OP_MAX_BATCH = 5, LLMEM_OP_SELECT = 6, LLMEM_OP_EXPAND_SCAN = 7 };
 
 /* call flags */
 #define LLMEM_SELECT_ALLZERO 1u /* llmem_select_method: offload only if every score is 0 */
@@ -182,6 +182,24 @@ llmem_status llmem_scan_peak(const int64_t* DEV delta, const int64_t* DEV offset
                              int64_t total_events, const llmem_config* DEV cfg,
                              int64_t* DEV peak_out, int64_t* DEV peak_index_out, void* DEV scratch,
                              size_t scratch_bytes, uint32_t flags, void* cuda_stream);
+
+/* llmem_expand_events and llmem_scan_peak in one pass (Sections 4.1, 4.2 and 5): the list
+ * is written exactly as llmem_expand_events writes it (raw sizes, or page-rounded with
+ * LLMEM_FUSE_ROUND) and, while each piece of it is still in shared memory, folded into the
+ * per-configuration peak of the page-rounded list.  Outputs are those of
+ * llmem_scan_peak(..., cfg, ...) on the rounded list: m_base + lm_p + largest prefix sum,
+ * first index attaining it, -1 / -1 for an inadmissible cfg[i].  The list is written to
+ * device memory once and not read back.
+ *   offsets        DEV [n+1]  as written by llmem_event_counts for the same cfg
+ *   total_events   HOST value of offsets[n]
+ *   delta_out      DEV [total_events]
+ *   peak_out       DEV [n]
+ *   peak_index_out DEV [n], nullable
+ *   scratch        required, llmem_scratch_bytes(LLMEM_OP_EXPAND_SCAN, n, total_events) */
+llmem_status llmem_expand_scan(const llmem_config* DEV cfg, int64_t n, const int64_t* DEV offsets,
+                               int64_t total_events, int64_t* DEV delta_out, int64_t* DEV peak_out,
+                               int64_t* DEV peak_index_out, void* DEV scratch, size_t scratch_bytes,
+                               uint32_t flags, void* cuda_stream);
 
 /* Algorithm 1, the inner loop of every method: the largest batch b in 1..bmax
  * whose peak does not exceed the capacity (0 if even b = 1 does not fit, -1 on

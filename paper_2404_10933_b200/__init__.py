@@ -24,7 +24,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "csrc", "libllmem.so")
 
 OK, ERR_ARG, ERR_SCRATCH, ERR_CUDA, ERR_TIMEOUT = 0, 1, 2, 3, 4
-OP_ESTIMATE, OP_EVENT_COUNTS, OP_EXPAND, OP_ROUND, OP_SCAN_PEAK, OP_MAX_BATCH, OP_SELECT = range(7)
+OP_ESTIMATE, OP_EVENT_COUNTS, OP_EXPAND, OP_ROUND, OP_SCAN_PEAK, OP_MAX_BATCH, OP_SELECT, OP_EXPAND_SCAN = range(8)
 SELECT_ALLZERO = 1
 FUSE_ROUND = 2
 METHOD_OFFLOAD = 4
@@ -33,7 +33,7 @@ EXPORTS = (
     "llmem_scratch_bytes", "llmem_estimate_batch", "llmem_event_counts", "llmem_expand_events",
     "llmem_round_events", "llmem_scan_peak", "llmem_max_batch", "llmem_select_method",
     "llmem_scratch_status", "llmem_last_error", "llmem_version", "llmem_event_counts_static",
-    "llmem_select_segmented",
+    "llmem_select_segmented", "llmem_expand_scan",
 )
 STATIC_MAX_CONFIGS = 4194304
 
@@ -68,6 +68,7 @@ def lib() -> ctypes.CDLL:
         L.llmem_scan_peak.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, sz, u32, vp]
         L.llmem_max_batch.argtypes = [vp, i64, vp, i32, i32, vp, vp, vp, sz, u32, vp]
         L.llmem_select_method.argtypes = [vp, i64, vp, i32, i32, vp, vp, vp, vp, vp, sz, u32, vp]
+        L.llmem_expand_scan.argtypes = [vp, i64, vp, i64, vp, vp, vp, vp, sz, u32, vp]
         L.llmem_select_segmented.argtypes = [vp, vp, vp, i64, i64, i32, vp, vp, vp, vp, sz, u32, vp]
         L.llmem_scratch_status.argtypes = [vp, vp]
         L.llmem_last_error.restype = ctypes.c_char_p
@@ -222,6 +223,31 @@ def scan_peak(delta, offsets, cfg=None, *, fuse_round: bool = False, want_index:
     if check_status:
         _check(lib().llmem_scratch_status(_ptr(scratch), _stream_ptr(stream)))
     return {"peak": peak, "index": index, "scratch": scratch}
+
+
+def expand_scan(cfg, offsets, total_events: Optional[int] = None, *, fuse_round: bool = True, out=None,
+                want_index: bool = True, scratch=None, stream=None):
+    """Materialise the event list and compute the peaks in one pass (the list is written
+    once and not read back).  Returns dict(delta, peak[n], index[n] | None, scratch)."""
+    torch = _torch()
+    cfg = _as_cfg(cfg)
+    n = cfg.shape[0]
+    if total_events is None:
+        total_events = int(offsets[-1].item())
+    if out is None:
+        out = torch.empty(total_events, dtype=torch.int64, device=cfg.device)
+    elif out.numel() < total_events or out.dtype != torch.int64:
+        raise ValueError("out must be an int64 tensor with at least total_events elements")
+    peak = torch.empty(n, dtype=torch.int64, device=cfg.device)
+    index = torch.empty(n, dtype=torch.int64, device=cfg.device) if want_index else None
+    if scratch is None:
+        scratch, nbytes = _scratch(OP_EXPAND_SCAN, n, total_events, cfg.device)
+    else:
+        nbytes = scratch.numel()
+    _check(lib().llmem_expand_scan(_ptr(cfg), n, _ptr(offsets), total_events, _ptr(out), _ptr(peak), _ptr(index),
+                                   _ptr(scratch), nbytes, FUSE_ROUND if fuse_round else 0, _stream_ptr(stream)))
+    delta = out[:total_events] if out.numel() != total_events else out
+    return {"delta": delta, "peak": peak, "index": index, "scratch": scratch}
 
 
 def max_batch(shape, capacities, bmax: int, *, want_status: bool = True, stream=None):

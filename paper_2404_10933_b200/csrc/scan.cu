@@ -19,7 +19,7 @@
 // records LLMEM_ERR_TIMEOUT in the scratch status word, drains its own copies and
 // returns.
 #include "llmem_host.h"
-#include "llmem_model.cuh"
+#include "fold.cuh"
 
 namespace llmem {
 
@@ -41,46 +41,6 @@ constexpr int kScanPerLane = LLMEM_SCAN_PER_LANE;
 constexpr int kScanChunk = 32 * kScanPerLane;  // 832 events = 6656 bytes: one warp's unit of work
 constexpr int kScanStages = LLMEM_SCAN_STAGES;  // chunks in flight per warp
 static_assert(kScanPerLane % 2 == 0 && (kScanPerLane / 2) % 2 == 1, "per-lane span: odd number of 16-byte words");
-
-struct Agg {
-  i64 sum, mx, idx;  // idx: virtual (alignment-shifted) global index of the first arg max
-  i64 valid;         // 0: identity
-};
-
-__device__ __forceinline__ Agg agg_identity() { return Agg{0, 0, -1, 0}; }
-
-// ordered fold: a covers earlier events than b
-__device__ __forceinline__ Agg agg_fold(const Agg& a, const Agg& b) {
-  if (!a.valid) return b;
-  if (!b.valid) return a;
-  Agg r;
-  r.sum = a.sum + b.sum;
-  const i64 cand = a.sum + b.mx;
-  const bool take = cand > a.mx;  // ties keep the earlier index
-  r.mx = take ? cand : a.mx;
-  r.idx = take ? b.idx : a.idx;
-  r.valid = 1;
-  return r;
-}
-
-__device__ __forceinline__ Agg agg_shfl_down(const Agg& a, int delta) {
-  Agg r;
-  r.sum = __shfl_down_sync(0xffffffffu, a.sum, delta);
-  r.mx = __shfl_down_sync(0xffffffffu, a.mx, delta);
-  r.idx = __shfl_down_sync(0xffffffffu, a.idx, delta);
-  r.valid = __shfl_down_sync(0xffffffffu, (int)a.valid, delta);
-  return r;
-}
-
-// lane 0 receives the in-order fold of all 32 lanes
-__device__ __forceinline__ Agg warp_fold(Agg a, int lane) {
-#pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {
-    Agg o = agg_shfl_down(a, d);
-    if (lane + d < 32) a = agg_fold(a, o);
-  }
-  return a;
-}
 
 // ---- mbarrier / TMA primitives ---------------------------------------------
 __device__ __forceinline__ u32 saddr(const void* p) { return (u32)__cvta_generic_to_shared(p); }
@@ -157,80 +117,6 @@ __device__ __forceinline__ bool segment_offset(const llmem_config* __restrict__ 
   return true;
 }
 
-// The scan kernel stores the bare result of a finished segment: its largest prefix
-// sum and the segment-relative index of the first event attaining it.  The finish
-// kernel adds the per-configuration offset.
-__device__ __forceinline__ void write_raw(i64 seg, const Agg& a, i64 seg_vstart, i64* __restrict__ peak_out,
-                                          i64* __restrict__ index_out) {
-  peak_out[seg] = a.valid ? a.mx : 0;
-  if (index_out) index_out[seg] = a.valid ? a.idx - seg_vstart : -1;
-}
-
-template <bool kRound>
-__device__ __forceinline__ i64 ev(i64 d) { return kRound ? page_round_signed(d) : d; }
-
-// In-order fold of tile-local events [lo, hi) by one warp; lanes take contiguous
-// chunks of odd length (distinct banks).  `vbase` is the virtual index of tile slot 0.
-template <bool kRound>
-__device__ __forceinline__ Agg warp_fold_range(const i64* __restrict__ tile, int lo, int hi, int lane, i64 vbase) {
-  const int len = hi - lo;
-  const int ch = ((len + 31) / 32) | 1;
-  const int a = lo + lane * ch;
-  const int b = a + ch < hi ? a + ch : hi;
-  Agg g = agg_identity();
-  if (a < b) {
-    i64 s = ev<kRound>(tile[a]), m = s;
-    int ix = a;
-    for (int j = a + 1; j < b; ++j) {
-      s += ev<kRound>(tile[j]);
-      if (s > m) { m = s; ix = j; }
-    }
-    g = Agg{s, m, vbase + ix, 1};
-  }
-  return warp_fold(g, lane);
-}
-
-// Scratch payload: per warp a head partial (segment that began in an earlier warp's
-// range) and a tail partial (segment that continues into a later warp's range).
-struct WarpPartials {
-  Agg head, tail;
-};
-
-// Result of the fast path before it is widened to an Agg: chunk-local arg max.
-struct Fold3 {
-  i64 sum, mx;
-  int ix;
-};
-
-__device__ __forceinline__ Fold3 fold3(const Fold3& a, const Fold3& b) {
-  Fold3 r;
-  r.sum = a.sum + b.sum;
-  const i64 cand = a.sum + b.mx;
-  const bool take = cand > a.mx;
-  r.mx = take ? cand : a.mx;
-  r.ix = take ? b.ix : a.ix;
-  return r;
-}
-
-// In-order fold of the 16-byte words [V0, V1) of a lane's span (compile-time bounds).
-template <bool kRound, int V0, int V1>
-__device__ __forceinline__ Fold3 fold_words(const longlong2* x) {
-  Fold3 f;
-  f.sum = ev<kRound>(x[V0].x);
-  f.mx = f.sum;
-  f.ix = 2 * V0;
-#pragma unroll
-  for (int j = V0; j < V1; ++j) {
-    if (j > V0) {
-      f.sum += ev<kRound>(x[j].x);
-      if (f.sum > f.mx) { f.mx = f.sum; f.ix = 2 * j; }
-    }
-    f.sum += ev<kRound>(x[j].y);
-    if (f.sum > f.mx) { f.mx = f.sum; f.ix = 2 * j + 1; }
-  }
-  return f;
-}
-
 template <bool kRound>
 __global__ void __launch_bounds__(kScanThreads, 1)
 scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, int shift /* 0 or 1 */,
@@ -298,43 +184,10 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
     seg_vend = seg < n ? __ldg(offsets + seg + 1) + shift : v_end;
   }
   const i64 warp_vlo = c_lo * kScanChunk;  // segments that start at or after this started in this warp's range
-  // Fold of the current segment so far, kept distributed over the warp: `base` (the same
-  // in every lane) is the sum of all events folded; each lane remembers the best prefix
-  // value it has seen among its own events and where.  Because every lane only ever
-  // replaces its candidate by a strictly larger, later one, and the final reduction
-  // prefers the smaller index among equals, the result is the first arg max.
-  i64 base = 0, best_v = 0, best_i = 0;
-  bool lane_has = false, seg_has = false;
+  SegmentFolder folder;
+  WarpPartials* my_partials = partials + gw;
   i64 consumed = 0;
   bool aborted = false;
-
-  // all lanes: reduce the distributed state to one Agg (valid in every lane) and reset it
-  auto take_state = [&]() -> Agg {
-#pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) {
-      const i64 ov = __shfl_xor_sync(0xffffffffu, best_v, d);
-      const i64 oi = __shfl_xor_sync(0xffffffffu, best_i, d);
-      const bool oh = __shfl_xor_sync(0xffffffffu, (int)lane_has, d) != 0;
-      if (oh && (!lane_has || ov > best_v || (ov == best_v && oi < best_i))) {
-        best_v = ov;
-        best_i = oi;
-        lane_has = true;
-      }
-    }
-    Agg a{base, best_v, best_i, seg_has ? 1 : 0};
-    base = 0;
-    lane_has = false;
-    seg_has = false;
-    return a;
-  };
-  // the segment `seg` ends: store its result, or leave a partial if it began earlier
-  auto finish_segment = [&]() {
-    const Agg run = take_state();
-    if (lane == 0) {
-      if (seg_vstart >= warp_vlo) write_raw(seg, run, seg_vstart, peak_out, index_out);
-      else partials[gw].head = run;
-    }
-  };
   auto next_segment = [&](i64 pos) {
     do {
       ++seg;
@@ -355,36 +208,13 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
 
     if (v_lo == t0 && v_hi == t0 + kScanChunk && seg < n && seg_vend >= v_hi) {
       // ---------- fast path: the whole chunk lies inside one segment ----------
-      const longlong2* src = reinterpret_cast<const longlong2*>(tile + lane * kScanPerLane);
-      longlong2 x[kScanPerLane / 2];
-#pragma unroll
-      for (int j = 0; j < kScanPerLane / 2; ++j) x[j] = src[j];
-      // four independent in-order folds over quarters of the span, then joined
-      constexpr int kVec = kScanPerLane / 2;
-      constexpr int q1 = kVec / 4, q2 = kVec / 2, q3 = (3 * kVec) / 4;
-      const Fold3 f0 = fold_words<kRound, 0, q1>(x), f1 = fold_words<kRound, q1, q2>(x);
-      const Fold3 f2 = fold_words<kRound, q2, q3>(x), f3 = fold_words<kRound, q3, kVec>(x);
-      const Fold3 f = fold3(fold3(f0, f1), fold3(f2, f3));
+      const Fold3 f = fold_lane_span<kRound, kScanPerLane>(tile + lane * kScanPerLane);
       // every lane has consumed its part of the stage: refill it
       __syncwarp();
       if (lane == 0 && c + kScanStages < c_hi) issue(c + kScanStages);
-      // prefix of the lane sums across the warp
-      i64 inc = f.sum;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const i64 o = __shfl_up_sync(0xffffffffu, inc, d);
-        if (lane >= d) inc += o;
-      }
-      const i64 cand = base + (inc - f.sum) + f.mx;
-      if (!lane_has || cand > best_v) {
-        best_v = cand;
-        best_i = t0 + lane * kScanPerLane + f.ix;
-        lane_has = true;
-      }
-      base += __shfl_sync(0xffffffffu, inc, 31);
-      seg_has = true;
+      folder.add_spans<kScanPerLane>(f, t0, lane);
       if (seg_vend == v_hi) {
-        finish_segment();
+        folder.finish_segment(seg, seg_vstart, warp_vlo, my_partials, peak_out, index_out, lane);
         next_segment(v_hi);
       }
       continue;
@@ -395,24 +225,10 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
     while (pos < v_hi && seg < n) {
       const i64 pb = seg_vend < v_hi ? seg_vend : v_hi;
       Agg g = warp_fold_range<kRound>(tile, (int)(pos - t0), (int)(pb - t0), lane, t0);
-      // the piece's fold (lane 0) joins the distributed state through lane 0's candidate
-      const i64 g_sum = __shfl_sync(0xffffffffu, g.sum, 0);
-      const bool g_valid = __shfl_sync(0xffffffffu, (int)g.valid, 0) != 0;
-      if (g_valid) {
-        if (lane == 0) {
-          const i64 cand = base + g.mx;
-          if (!lane_has || cand > best_v) {
-            best_v = cand;
-            best_i = g.idx;
-            lane_has = true;
-          }
-        }
-        base += g_sum;
-        seg_has = true;
-      }
+      folder.add_piece(g, lane);
       pos = pb;
       if (seg_vend <= v_hi) {
-        finish_segment();
+        folder.finish_segment(seg, seg_vstart, warp_vlo, my_partials, peak_out, index_out, lane);
         next_segment(pos);
       }
     }
@@ -420,13 +236,9 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
     if (lane == 0 && c + kScanStages < c_hi) issue(c + kScanStages);
   }
 
-  const Agg run = take_state();
+  // the current segment may continue into the next warp's range
+  if (!aborted) folder.finish_range(seg_vstart, warp_vlo, my_partials, lane);
   if (lane == 0) {
-    if (!aborted && run.valid) {
-      // the current segment continues into the next warp's range
-      if (seg_vstart >= warp_vlo) partials[gw].tail = run;
-      else partials[gw].head = run;
-    }
     // drain: every copy that was issued must have landed before the warp exits
     i64 issued = c_hi - c_lo;
     if (issued > consumed + kScanStages) issued = consumed + kScanStages;
@@ -441,13 +253,13 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
 // configurations.
 __global__ void __launch_bounds__(256)
 scan_finish_kernel(const i64* __restrict__ offsets, i64 n, int shift, const llmem_config* __restrict__ cfg,
-                   i64* __restrict__ peak_out, i64* __restrict__ index_out, i64 chunks_per_warp,
+                   i64* __restrict__ peak_out, i64* __restrict__ index_out, i64 range_events,
                    const WarpPartials* __restrict__ partials) {
   for (i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (i64)gridDim.x * blockDim.x) {
     const i64 a = offsets[i] + shift, b = offsets[i + 1] + shift;
     i64 mx = 0, idx = -1;
     if (b > a) {
-      const i64 ca = (a / kScanChunk) / chunks_per_warp, cb = ((b - 1) / kScanChunk) / chunks_per_warp;
+      const i64 ca = a / range_events, cb = (b - 1) / range_events;
       if (ca == cb) {  // finished by the warp that owns it
         mx = peak_out[i];
         if (index_out) idx = index_out[i];
@@ -463,6 +275,18 @@ scan_finish_kernel(const i64* __restrict__ offsets, i64 n, int shift, const llme
     peak_out[i] = ok ? off + mx : -1;
     if (index_out) index_out[i] = ok ? idx : -1;
   }
+}
+
+llmem_status launch_scan_finish(const i64* offsets, i64 n, int shift, const llmem_config* cfg, i64* peak_out,
+                                i64* index_out, i64 range_events, const WarpPartials* partials,
+                                cudaStream_t stream) {
+  i64 blocks = (n + 255) / 256;
+  const i64 cap = (i64)sm_count() * 8;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  scan_finish_kernel<<<(unsigned)blocks, 256, 0, stream>>>(offsets, n, shift, cfg, peak_out, index_out,
+                                                          range_events < 1 ? 1 : range_events, partials);
+  return check_launch("llmem_scan_peak (finish)");
 }
 
 }  // namespace llmem
@@ -528,11 +352,6 @@ extern "C" llmem_status llmem_scan_peak(const int64_t* delta, const int64_t* off
     llmem_status st = check_launch("llmem_scan_peak");
     if (st != LLMEM_OK) return st;
   }
-  i64 blocks = (n + 255) / 256;
-  const i64 cap = (i64)sm_count() * 8;
-  if (blocks > cap) blocks = cap;
-  scan_finish_kernel<<<(unsigned)blocks, 256, 0, s>>>(
-      reinterpret_cast<const i64*>(offsets), n, shift, cfg, reinterpret_cast<i64*>(peak_out),
-      reinterpret_cast<i64*>(peak_index_out), chunks_per_warp, partials);
-  return check_launch("llmem_scan_peak (finish)");
+  return launch_scan_finish(reinterpret_cast<const i64*>(offsets), n, shift, cfg, reinterpret_cast<i64*>(peak_out),
+                            reinterpret_cast<i64*>(peak_index_out), chunks_per_warp * kScanChunk, partials, s);
 }

@@ -133,6 +133,10 @@ def test_g5_stress_materialized_full(llmem):
     assert np.array_equal(index[idx], want1["index"])
     off = offsets.cpu().numpy()
     assert np.array_equal(np.diff(off)[idx], want1["count"])
+    # the one-pass variant at full size: same list, same peaks
+    delta.fill_(0)
+    one = llmem.expand_scan(dev, offsets, total, fuse_round=True, out=delta)
+    assert torch.equal(one["peak"], r["peak"]) and torch.equal(one["index"], r["index"])
     # whole event lists of a few configurations, bit for bit
     for i in idx[:6]:
         ev = oracle.round_events(oracle.expand_events(cfgs[i:i + 1]))

@@ -92,7 +92,12 @@ def check_materialized(llmem, cfgs, want):
     assert np.array_equal(rounded.cpu().numpy(), rounded_want)
     r2 = llmem.scan_peak(rounded, offsets, dev, check_status=True)
     r3 = llmem.scan_peak(fused, offsets, dev, check_status=True)
-    for r in (r1, r2, r3):
+    # one-pass expansion + scan, list written rounded and raw
+    r4 = llmem.expand_scan(dev, offsets, total, fuse_round=True)
+    assert np.array_equal(r4["delta"].cpu().numpy(), rounded_want)
+    r5 = llmem.expand_scan(dev, offsets, total, fuse_round=False)
+    assert np.array_equal(r5["delta"].cpu().numpy(), raw_want)
+    for r in (r1, r2, r3, r4, r5):
         assert np.array_equal(r["peak"].cpu().numpy(), want["peak"])
         assert np.array_equal(r["index"].cpu().numpy(), want["index"])
     return total
@@ -197,6 +202,14 @@ def test_expand_into_unaligned_output(llmem):
     out = llmem.expand_events(dev, offsets, total, fuse_round=True, out=buf[1:1 + total])
     assert out.data_ptr() % 16 == 8
     assert np.array_equal(out.cpu().numpy(), want)
+    assert buf[0].item() == -7 and (buf[1 + total:] == -7).all()
+    # the one-pass variant into the same unaligned view
+    buf.fill_(-7)
+    r = llmem.expand_scan(dev, offsets, total, fuse_round=True, out=buf[1:1 + total])
+    est = oracle.estimate(cfgs, threads=4)
+    assert np.array_equal(r["delta"].cpu().numpy(), want)
+    assert np.array_equal(r["peak"].cpu().numpy(), est["peak"])
+    assert np.array_equal(r["index"].cpu().numpy(), est["index"])
     assert buf[0].item() == -7 and (buf[1 + total:] == -7).all()
 
 
