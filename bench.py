@@ -7,6 +7,11 @@ decoders, about 5.8e9 allocate/free events, materialised as int64):
     event counts + offsets  ->  expansion with fused page rounding  ->  segmented
     prefix-sum + max  ->  largest batch per capacity  ->  Algorithm 1 selection
 
+By default the expansion and the scan run as one kernel (llmem_expand_scan: the list is
+written to HBM once and folded from shared memory); --two-pass times the separate
+llmem_expand_events and llmem_scan_peak kernels instead.  Either way the kernels of the
+other path are timed alone after the step and reported next to it.
+
 `value` is alloc-events per second over all ranks with the configurations already
 resident in HBM; `e2e` is the same pass through the public API starting from pinned
 host buffers, with the host<->device copies inside the timed region.  The roofline
@@ -42,7 +47,7 @@ FALLBACK_HBM_GBS = 6650.0
 # HBM-bound kernels, from an ncu capture of a 4096-configuration run (summary kept under
 # profiles/; traffic grows in proportion to the number of events).  Set an entry
 # to None when its kernel changes after the capture.
-NCU_TRAFFIC_BYTES_PER_EVENT = {"expand": 7.8206, "scan": 8.0145}
+NCU_TRAFFIC_BYTES_PER_EVENT = {"expand": 7.8206, "scan": 8.0145, "expand_scan": None}
 
 
 def measured_peaks():
@@ -173,10 +178,11 @@ def run_reference(args):
 class HotPath:
     """Holds device buffers for one grid and runs one step of the hot path."""
 
-    KERNELS_PER_STEP = 8  # counts(3) + expand(1) + scan(2) + max_batch(1) + select(1)
-
-    def __init__(self, llmem, torch, cfgs: np.ndarray, caps: np.ndarray, bmax: int):
+    def __init__(self, llmem, torch, cfgs: np.ndarray, caps: np.ndarray, bmax: int, one_pass: bool):
         self.llmem, self.torch = llmem, torch
+        self.one_pass = one_pass
+        # counts(3) + [expand_scan(1) + finish(1) | expand(1) + scan(1) + finish(1)] + max_batch(1) + select(1)
+        self.kernels_per_step = 7 if one_pass else 8
         self.n = len(cfgs)
         self.bmax = bmax
         self.host_cfg = torch.from_numpy(cfgs.view(np.uint8).reshape(-1, 64)).pin_memory()
@@ -188,7 +194,7 @@ class HotPath:
         self.delta = torch.empty(self.total, dtype=torch.int64, device="cuda")
         self.scan_scratch = torch.empty(llmem.scratch_bytes(llmem.OP_SCAN_PEAK, self.n, self.total),
                                         dtype=torch.uint8, device="cuda")
-        self.ev = {k: [] for k in ("expand", "scan")}
+        self.ev = {k: [] for k in (("expand_scan",) if one_pass else ("expand", "scan"))}
         self.side = torch.cuda.Stream()
         self.fork = torch.cuda.Event()
         self.host_out = {
@@ -197,34 +203,43 @@ class HotPath:
             "batch": torch.empty((self.n, len(caps)), dtype=torch.int32).pin_memory(),
         }
 
-    def step(self, cfg=None, caps=None, total=None, record=True):
+    def _materialise_and_search(self, cfg, caps, offsets, total, record):
+        """Rows a2-a6 for configurations and offsets already on the device."""
         llmem, torch = self.llmem, self.torch
-        cfg = self.cfg if cfg is None else cfg
-        caps = self.caps if caps is None else caps
         main = torch.cuda.current_stream()
-        offsets, status = llmem.event_counts(cfg)
-        if total is None:
-            total = self.total
         e = [torch.cuda.Event(enable_timing=True) for _ in range(3)] if record else None
         if record:
             e[0].record()
-        delta = llmem.expand_events(cfg, offsets, total, fuse_round=True, out=self.delta)
-        if record:
-            e[1].record()
-        # the searches (integer ALU, a few bytes per configuration) do not depend on the event
-        # list: they are queued on a second stream once the expansion holds its SMs, and run
-        # underneath the two HBM-bound kernels
-        self.fork.record(main)
-        self.side.wait_event(self.fork)
-        with torch.cuda.stream(self.side):
+        if self.one_pass:
+            # expansion, page rounding and segmented scan in one kernel: the list is written once
+            r = llmem.expand_scan(cfg, offsets, total, fuse_round=True, out=self.delta, scratch=self.scan_scratch)
+            if record:
+                e[1].record()
+                self.ev["expand_scan"].append((e[0], e[1]))
             bs, _ = llmem.max_batch(cfg, caps, self.bmax, want_status=False)
             sel = llmem.select_method(cfg, caps, self.bmax, want_bs_list=False, want_status=False)
-        r = llmem.scan_peak(delta, offsets, cfg, scratch=self.scan_scratch)
-        if record:
-            e[2].record()
-            self.ev["expand"].append((e[0], e[1]))
-            self.ev["scan"].append((e[1], e[2]))
-        main.wait_stream(self.side)
+        else:
+            delta = llmem.expand_events(cfg, offsets, total, fuse_round=True, out=self.delta)
+            if record:
+                e[1].record()
+            # the searches (integer ALU, a few bytes per configuration) do not depend on the event
+            # list: queued on a second stream once the expansion is done, they run underneath the scan
+            self.fork.record(main)
+            self.side.wait_event(self.fork)
+            with torch.cuda.stream(self.side):
+                bs, _ = llmem.max_batch(cfg, caps, self.bmax, want_status=False)
+                sel = llmem.select_method(cfg, caps, self.bmax, want_bs_list=False, want_status=False)
+            r = llmem.scan_peak(delta, offsets, cfg, scratch=self.scan_scratch)
+            if record:
+                e[2].record()
+                self.ev["expand"].append((e[0], e[1]))
+                self.ev["scan"].append((e[1], e[2]))
+            main.wait_stream(self.side)
+        return r, bs, sel
+
+    def step(self, record=True):
+        offsets, _ = self.llmem.event_counts(self.cfg)
+        r, bs, sel = self._materialise_and_search(self.cfg, self.caps, offsets, self.total, record)
         return {"peak": r["peak"], "index": r["index"], "bs": bs, "method": sel["method"],
                 "batch": sel["batch"], "offsets": offsets}
 
@@ -235,24 +250,36 @@ class HotPath:
         torch = self.torch
         cfg = self.host_cfg.to("cuda", non_blocking=True)
         caps = self.host_caps.to("cuda", non_blocking=True)
-        main = torch.cuda.current_stream()
         offsets, _ = self.llmem.event_counts(cfg)
         total = int(offsets[-1].item())                      # 8-byte D2H + sync
         if total > self.delta.numel():
             self.delta = torch.empty(total, dtype=torch.int64, device="cuda")
-        delta = self.llmem.expand_events(cfg, offsets, total, fuse_round=True, out=self.delta)
-        self.fork.record(main)
-        self.side.wait_event(self.fork)
-        with torch.cuda.stream(self.side):
-            self.llmem.max_batch(cfg, caps, self.bmax, want_status=False)
-            sel = self.llmem.select_method(cfg, caps, self.bmax, want_bs_list=False, want_status=False)
-        r = self.llmem.scan_peak(delta, offsets, cfg, scratch=self.scan_scratch)
-        main.wait_stream(self.side)
+        r, _, sel = self._materialise_and_search(cfg, caps, offsets, total, False)
         self.host_out["peak"].copy_(r["peak"], non_blocking=True)
         self.host_out["method"].copy_(sel["method"], non_blocking=True)
         self.host_out["batch"].copy_(sel["batch"], non_blocking=True)
         torch.cuda.current_stream().synchronize()
         return total
+
+    def time_kernel(self, what, reps=5):
+        """Mean launch time (ms) of one of the HBM-bound kernels on the resident grid."""
+        llmem, torch = self.llmem, self.torch
+        offsets, _ = llmem.event_counts(self.cfg)
+        ts = []
+        for _ in range(reps + 1):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            if what == "expand":
+                llmem.expand_events(self.cfg, offsets, self.total, fuse_round=True, out=self.delta)
+            elif what == "scan":
+                llmem.scan_peak(self.delta, offsets, self.cfg, scratch=self.scan_scratch)
+            else:
+                llmem.expand_scan(self.cfg, offsets, self.total, fuse_round=True, out=self.delta,
+                                  scratch=self.scan_scratch)
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return statistics.mean(ts[1:])
 
     @property
     def h2d_bytes(self):
@@ -297,7 +324,7 @@ def run_ours(args):
     n_cfg = args.configs
     cfgs = grids.g5_stress(0, n_cfg, seed_offset=rank)     # weak scaling: one full grid per rank
     caps = grids.g4_capacities()
-    hp = HotPath(llmem, torch, cfgs, caps, grids.G4_BMAX)
+    hp = HotPath(llmem, torch, cfgs, caps, grids.G4_BMAX, one_pass=not args.two_pass)
 
     # ---- device-resident timing ----
     for _ in range(args.warmup):
@@ -355,24 +382,34 @@ def run_ours(args):
         return 0
 
     peak_gbs, peak_src = measured_peaks()
+    bytes_per_launch = 8.0 * hp.total          # 8 algorithmic bytes per event for each of the three kernels
+    others = {k: hp.time_kernel(k) for k in ("expand", "scan", "expand_scan") if k not in kernel_ms}
     dom = max(kernel_ms, key=kernel_ms.get)
-    bytes_per_launch = 8.0 * hp.total          # 8 algorithmic bytes per event for either kernel
     achieved = bytes_per_launch / (kernel_ms[dom] * 1e-3) / 1e9
+
+    def entry(ms_):
+        g = bytes_per_launch / (ms_ * 1e-3) / 1e9
+        return {"ms": ms_, "gbs": g, "frac": g / peak_gbs}
     roofline = {
-        "bound": "hbm", "kernel": {"expand": "expand_kernel (8 B written / event)",
-                                   "scan": "scan_kernel (8 B read / event)"}[dom],
+        "bound": "hbm",
+        "kernel": {"expand": "expand_kernel (8 B written / event)", "scan": "scan_kernel (8 B read / event)",
+                   "expand_scan": "expand_scan_kernel (8 B written / event; the scan reads shared memory)"}[dom],
         "achieved": achieved, "peak": peak_gbs, "unit": "GB/s", "frac": achieved / peak_gbs,
         "peak_source": peak_src,
         "traffic": (NCU_TRAFFIC_BYTES_PER_EVENT[dom] * hp.total
                     if NCU_TRAFFIC_BYTES_PER_EVENT.get(dom) is not None else None),
         "traffic_note": "ncu dram bytes per event on a 4096-configuration capture, scaled by events",
         "algorithmic_bytes": bytes_per_launch,
-        "per_kernel": {k: {"ms": kernel_ms[k], "gbs": bytes_per_launch / (kernel_ms[k] * 1e-3) / 1e9,
-                           "frac": bytes_per_launch / (kernel_ms[k] * 1e-3) / 1e9 / peak_gbs}
-                       for k in kernel_ms},
-        "materialised_path_gbs": 2 * bytes_per_launch / ((kernel_ms["expand"] + kernel_ms["scan"]) * 1e-3) / 1e9,
+        "per_kernel": {k: entry(v) for k, v in kernel_ms.items()},
+        "other_path_kernels": {"note": "the kernels of the path not taken by the timed step, timed alone "
+                                       "after it on the same grid (5 launches each)",
+                               **{k: entry(v) for k, v in others.items()}},
         "frac_of_nominal_8000": achieved / 8000.0,
     }
+    step_text = ("event_counts + expand_scan (expansion, page rounding and segmented scan in one kernel, list "
+                 "written to HBM once) + max_batch + select_method" if hp.one_pass else
+                 "event_counts + expand(fused rounding) + scan_peak on the main stream; max_batch + "
+                 "select_method concurrently on a second stream; both joined before the step ends")
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
@@ -382,12 +419,11 @@ def run_ours(args):
                    "configs_per_gpu": hp.n, "events_per_gpu": hp.total, "capacities": len(caps),
                    "bmax": grids.G4_BMAX, "parallelism": f"replicas x{world} (independent configs, no collective)",
                    "l2": "event list (8 B/event) far larger than the 126 MB L2; no flush needed",
-                   "step": "event_counts + expand(fused rounding) + scan_peak on the main stream; max_batch + "
-                           "select_method concurrently on a second stream; both joined before the step ends"},
+                   "path": "one-pass" if hp.one_pass else "two-pass", "step": step_text},
         "roofline": roofline,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": hp.h2d_bytes,
                 "d2h_bytes_per_step": hp.d2h_bytes, "ms_per_step": e2e_ms / e2e_steps},
-        "gpu_launches": HotPath.KERNELS_PER_STEP * args.steps,
+        "gpu_launches": hp.kernels_per_step * args.steps,
         "clocks": clocks,
         "fused_equals_materialised": agree,
     }
@@ -501,6 +537,8 @@ def main():
     ap.add_argument("--configs", type=int, default=grids.G5_CONFIGS,
                     help="configurations of the stress grid per GPU (default: the full grid)")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--two-pass", action="store_true",
+                    help="time llmem_expand_events + llmem_scan_peak as separate kernels instead of llmem_expand_scan")
     ap.add_argument("--workload", choices=("g5", "g3", "g4"), default="g5",
                     help="g5 (default): the full hot path on the stress grid; g3 / g4: the in-register kernels")
     args = ap.parse_args()
