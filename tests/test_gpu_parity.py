@@ -1,7 +1,7 @@
 """Parity of the CUDA library with the CPU oracle, element by element, on the same
 seeded inputs.  All quantities are integers: the bar is bit-exact equality.
 Sizes here are ones the level-1 oracle finishes in seconds; they still span many
-tiles of the expansion and scan kernels (4608 events each) with ragged tails."""
+chunks of the expansion and scan kernels (576 and 832 events) with ragged tails."""
 import numpy as np
 import pytest
 
