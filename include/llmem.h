@@ -251,6 +251,20 @@ llmem_status llmem_select_segmented(const llmem_config* DEV item_cfg, const int3
                                     void* DEV scratch, size_t scratch_bytes, uint32_t flags,
                                     void* cuda_stream);
 
+/* Section 4.1: the chunk manager picks the chunk size that wastes the least memory for the
+ * given model.  The parameters outside the embedding occupy ceil(other_p / cs) whole chunks
+ * (Section 4.2, m_p), so a candidate cs wastes ceil(other_p / cs) * cs - other_p elements.
+ * Among the candidates cs_min, cs_min + cs_step, ..., n_candidates of them, all within
+ * 1 .. 2^40, the first with the least waste is returned.  The record's chunk_elems and
+ * batch are ignored.
+ *   chunk_out  DEV [n]  chosen cs in elements, -1 on status != 0
+ *   waste_out  DEV [n]  nullable; wasted elements of the choice
+ *   status_out DEV [n]  nullable */
+llmem_status llmem_chunk_search(const llmem_config* DEV cfg, int64_t n, int64_t cs_min,
+                                int64_t cs_step, int32_t n_candidates, int64_t* DEV chunk_out,
+                                int64_t* DEV waste_out, uint8_t* DEV status_out, void* DEV scratch,
+                                size_t scratch_bytes, uint32_t flags, void* cuda_stream);
+
 /* Synchronises cuda_stream and returns the device status word that
  * llmem_scan_peak keeps at the start of its scratch: LLMEM_OK, or
  * LLMEM_ERR_TIMEOUT if a bounded wait inside a kernel gave up (outputs are then

@@ -186,3 +186,19 @@ def select_segmented(item_cfg: np.ndarray, bs: np.ndarray, group_offsets):
     lib().oracle_select_segmented(_p(item_cfg), _p(bs), _p(offs), ctypes.c_int64(n_groups),
                                   ctypes.c_int32(n_cap), _p(item), _p(method), _p(batch))
     return {"item": item, "method": method, "batch": batch}
+
+
+def chunk_search(cfg: np.ndarray, cs_min: int, cs_step: int, n_candidates: int):
+    """Least-waste chunk size per configuration.  Returns dict(chunk, waste int64; status uint8)."""
+    cfg = _cfgs(cfg)
+    n = cfg.size
+    chunk = np.full(n, -1, dtype=np.int64)
+    waste = np.full(n, -1, dtype=np.int64)
+    status = np.zeros(n, dtype=np.uint8)
+    f = lib().oracle_chunk_search
+    for i in range(n):
+        a, b = ctypes.c_int64(0), ctypes.c_int64(0)
+        status[i] = f(_rec(cfg, i), ctypes.c_int64(cs_min), ctypes.c_int64(cs_step),
+                      ctypes.c_int32(n_candidates), ctypes.byref(a), ctypes.byref(b))
+        chunk[i], waste[i] = a.value, b.value
+    return {"chunk": chunk, "waste": waste, "status": status}

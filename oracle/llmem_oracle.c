@@ -794,3 +794,39 @@ void oracle_select_segmented(const oracle_config *item_cfg, const int32_t *bs,
     }
   }
 }
+
+/* ------------------------------------------------------------------------ */
+/* extension: chunk size search                                             */
+/* ------------------------------------------------------------------------ */
+/* Section 4.1 says only that the chunk manager picks the chunk size that wastes the least
+ * memory for the given model.  Reading: the parameters outside the embedding occupy
+ * ceil(other_p / cs) whole chunks (Section 4.2, m_p), so a candidate cs wastes
+ * ceil(other_p / cs) * cs - other_p elements; among the candidates
+ * cs_min, cs_min + cs_step, ... (n_candidates of them) the first one with the least waste
+ * is chosen.  The record's own chunk_elems is ignored.  Returns the status; on status 0
+ * *chunk_out and *waste_out (elements) are set, otherwise both are -1. */
+int oracle_chunk_search(const oracle_config *cfg, int64_t cs_min, int64_t cs_step, int32_t n_candidates,
+                        int64_t *chunk_out, int64_t *waste_out) {
+  *chunk_out = -1;
+  *waste_out = -1;
+  oracle_config c = *cfg;
+  c.chunk_elems = 1;
+  int st = validate_fields(&c, 0);
+  if (st) return st;
+  if (c.method > 3) return ST_FIELD;
+  sizes_t z;
+  compute_sizes(&c, &z);
+  u128 best_waste = 0;
+  int64_t best_cs = -1;
+  for (int32_t k = 0; k < n_candidates; ++k) {
+    u128 cs = (u128)cs_min + (u128)k * (u128)cs_step;
+    u128 waste = ceil_div(z.other_p, cs) * cs - z.other_p;
+    if (best_cs < 0 || waste < best_waste) { /* strict: the first of equals stays */
+      best_waste = waste;
+      best_cs = (int64_t)cs;
+    }
+  }
+  *chunk_out = best_cs;
+  *waste_out = (int64_t)best_waste;
+  return ST_OK;
+}

@@ -33,7 +33,7 @@ EXPORTS = (
     "llmem_scratch_bytes", "llmem_estimate_batch", "llmem_event_counts", "llmem_expand_events",
     "llmem_round_events", "llmem_scan_peak", "llmem_max_batch", "llmem_select_method",
     "llmem_scratch_status", "llmem_last_error", "llmem_version", "llmem_event_counts_static",
-    "llmem_select_segmented", "llmem_expand_scan",
+    "llmem_select_segmented", "llmem_expand_scan", "llmem_chunk_search",
 )
 STATIC_MAX_CONFIGS = 4194304
 
@@ -68,6 +68,7 @@ def lib() -> ctypes.CDLL:
         L.llmem_scan_peak.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, sz, u32, vp]
         L.llmem_max_batch.argtypes = [vp, i64, vp, i32, i32, vp, vp, vp, sz, u32, vp]
         L.llmem_select_method.argtypes = [vp, i64, vp, i32, i32, vp, vp, vp, vp, vp, sz, u32, vp]
+        L.llmem_chunk_search.argtypes = [vp, i64, i64, i64, i32, vp, vp, vp, vp, sz, u32, vp]
         L.llmem_expand_scan.argtypes = [vp, i64, vp, i64, vp, vp, vp, vp, sz, u32, vp]
         L.llmem_select_segmented.argtypes = [vp, vp, vp, i64, i64, i32, vp, vp, vp, vp, sz, u32, vp]
         L.llmem_scratch_status.argtypes = [vp, vp]
@@ -300,6 +301,20 @@ def select_segmented(item_cfg, bs, group_offsets, *, stream=None):
                                         n_items, n_cap, _ptr(item), _ptr(method), _ptr(batch), None, 0, 0,
                                         _stream_ptr(stream)))
     return {"item": item, "method": method, "batch": batch}
+
+
+def chunk_search(cfg, cs_min: int, cs_step: int, n_candidates: int, *, stream=None):
+    """Least-waste chunk size among cs_min + k cs_step.  Returns dict(chunk[n], waste[n] int64,
+    status[n] uint8)."""
+    torch = _torch()
+    cfg = _as_cfg(cfg)
+    n = cfg.shape[0]
+    chunk = torch.empty(n, dtype=torch.int64, device=cfg.device)
+    waste = torch.empty(n, dtype=torch.int64, device=cfg.device)
+    status = torch.empty(n, dtype=torch.uint8, device=cfg.device)
+    _check(lib().llmem_chunk_search(_ptr(cfg), n, cs_min, cs_step, n_candidates, _ptr(chunk), _ptr(waste),
+                                    _ptr(status), None, 0, 0, _stream_ptr(stream)))
+    return {"chunk": chunk, "waste": waste, "status": status}
 
 
 def _caps(capacities, device):

@@ -269,6 +269,51 @@ select_segmented_kernel(const llmem_config* __restrict__ item_cfg, const int* __
   }
 }
 
+// ---------------------------------------------------------------------------
+// llmem_chunk_search: least-waste chunk size.  One warp per configuration; lanes take
+// candidates cs_min + k cs_step round-robin (one 64-bit division each) and the warp
+// reduces to the smallest waste, the smaller candidate index among equals.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+chunk_search_kernel(const llmem_config* __restrict__ cfg, i64 n, i64 cs_min, i64 cs_step, int n_candidates,
+                    i64* __restrict__ chunk_out, i64* __restrict__ waste_out, uint8_t* __restrict__ status_out) {
+  const int lane = threadIdx.x & 31;
+  const i64 warps = ((i64)gridDim.x * blockDim.x) >> 5;
+  for (i64 i = ((i64)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
+    Cfg f = load_cfg(cfg + i);
+    f.chunk_elems = 1;  // the record's own chunk size plays no part here
+    const int st = check_fields(f, false, true);
+    u64 best_waste = ~0ull;
+    int best_k = 0x7fffffff;
+    if (st == LLMEM_CFG_OK) {
+      const u64 other_p = other_params(f);
+      for (int k = lane; k < n_candidates; k += 32) {
+        const u64 cs = (u64)cs_min + (u64)k * (u64)cs_step;
+        const u64 waste = ceil_div(other_p, cs) * cs - other_p;  // < cs <= 2^40
+        if (waste < best_waste) {  // k increases: the first of equals stays
+          best_waste = waste;
+          best_k = k;
+        }
+      }
+#pragma unroll
+      for (int d = 16; d >= 1; d >>= 1) {
+        const u64 ow = __shfl_xor_sync(0xffffffffu, best_waste, d);
+        const int ok = __shfl_xor_sync(0xffffffffu, best_k, d);
+        if (ow < best_waste || (ow == best_waste && ok < best_k)) {
+          best_waste = ow;
+          best_k = ok;
+        }
+      }
+    }
+    if (lane == 0) {
+      const bool ok = st == LLMEM_CFG_OK;
+      chunk_out[i] = ok ? (i64)((u64)cs_min + (u64)best_k * (u64)cs_step) : -1;
+      if (waste_out) waste_out[i] = ok ? (i64)best_waste : -1;
+      if (status_out) status_out[i] = (uint8_t)st;
+    }
+  }
+}
+
 static int grid_for(i64 threads_needed, int block, int ctas_per_sm) {
   i64 blocks = (threads_needed + block - 1) / block;
   i64 cap = (i64)sm_count() * ctas_per_sm;
@@ -360,4 +405,28 @@ extern "C" llmem_status llmem_select_segmented(const llmem_config* item_cfg, con
       item_cfg, bs, reinterpret_cast<const i64*>(group_offsets), n_groups, n_cap,
       reinterpret_cast<i64*>(item_out), method_out, batch_out);
   return check_launch("llmem_select_segmented");
+}
+
+extern "C" llmem_status llmem_chunk_search(const llmem_config* cfg, int64_t n, int64_t cs_min, int64_t cs_step,
+                                           int32_t n_candidates, int64_t* chunk_out, int64_t* waste_out,
+                                           uint8_t* status_out, void* scratch, size_t scratch_bytes,
+                                           uint32_t flags, void* cuda_stream) {
+  (void)scratch; (void)scratch_bytes; (void)flags;
+  clear_error();
+  if (n < 0) { set_error("llmem_chunk_search: n < 0"); return LLMEM_ERR_ARG; }
+  if (cs_min < 1 || cs_step < 1 || n_candidates < 1 ||
+      cs_min > (1ll << 40) || cs_step > (1ll << 40) ||
+      cs_min + (int64_t)(n_candidates - 1) * cs_step > (1ll << 40)) {
+    set_error("llmem_chunk_search: candidates must be cs_min + k cs_step in 1 .. 2^40, k < n_candidates");
+    return LLMEM_ERR_ARG;
+  }
+  if (n == 0) return LLMEM_OK;
+  if (!cfg || !chunk_out || !aligned_to(cfg, 16) || !aligned_to(chunk_out, 8) || !aligned_to(waste_out, 8)) {
+    set_error("llmem_chunk_search: cfg (16-byte aligned) and chunk_out are required");
+    return LLMEM_ERR_ARG;
+  }
+  chunk_search_kernel<<<grid_for(32 * n, 256, 8), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      cfg, n, cs_min, cs_step, n_candidates, reinterpret_cast<i64*>(chunk_out), reinterpret_cast<i64*>(waste_out),
+      status_out);
+  return check_launch("llmem_chunk_search");
 }

@@ -127,12 +127,23 @@ __device__ __forceinline__ u64 gathered_bytes(u64 x, u32 method, u32 n, u32 t) {
   return 0;
 }
 
+// Table 1, other_p: every parameter outside the input embedding and lm_head of a standard
+// decoder: per layer q, k, v, o (H x H) and 2 or 3 feed-forward matrices (H x F), their
+// biases, two norm vectors; one final norm.  `f` has passed check_fields.
+__device__ __forceinline__ u64 other_params(const Cfg& f) {
+  const u64 H = (u64)f.hidden, F = (u64)f.ffn, bias = f.has_bias;
+  const u64 nffn = f.ffn_kind ? 3 : 2;
+  const u64 bias_p = bias * (4 * H + (nffn - 1) * F + H);
+  const u64 norm_p = 2 * H * (1 + bias);
+  return (u64)f.layers * (4 * H * H + nffn * H * F + bias_p + norm_p) + H * (1 + bias);  // < 2^61
+}
+
 // a1: parameter inventory and event sizes.  `f` has passed check_fields.
 __device__ __forceinline__ Plan make_plan(const Cfg& f, u32 method) {
   Plan p;
   p.status = check_combo(method, f.gpu_n, f.tp_n);
   const u64 H = (u64)f.hidden, F = (u64)f.ffn, V = (u64)f.vocab, P = (u64)f.pos_len;
-  const u64 bias = f.has_bias, n = f.gpu_n;
+  const u64 n = f.gpu_n;
   p.e_n = 1 + (f.pos_len > 0);
   p.K = f.ffn_kind ? 7 : 6;
   p.gather = (method == LLMEM_METHOD_ADP || method == LLMEM_METHOD_DPTP);
@@ -143,10 +154,7 @@ __device__ __forceinline__ Plan make_plan(const Cfg& f, u32 method) {
   p.iters = (int)f.iters;
   const u64 tok_p = V * H, pos_p = P * H, hh_p = H * H, hf_p = H * F;
   const u64 embed_p = tok_p + pos_p;                       // <= 2^47
-  const u64 nffn = (u64)(p.K - 4);
-  const u64 bias_p = bias * (4 * H + (nffn - 1) * F + H);
-  const u64 norm_p = 2 * H * (1 + bias);
-  const u64 other_p = (u64)p.L * (4 * hh_p + nffn * hf_p + bias_p + norm_p) + H * (1 + bias);  // < 2^61
+  const u64 other_p = other_params(f);                     // < 2^61
   const u64 cs = (u64)f.chunk_elems;
   const u64 chunks = ceil_div(other_p, cs);
   p.offset = (u64)f.base_bytes + tok_p * (u64)f.lm_bytes;  // < 2^60 + 2^49

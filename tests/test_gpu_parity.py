@@ -319,3 +319,17 @@ def test_segmented_selection_random_groups(llmem):
     for k in ("item", "method", "batch"):
         assert np.array_equal(got[k].cpu().numpy(), want[k]), k
     assert (want["item"] == -1).any() and (want["method"] == 3).any()
+
+
+def test_chunk_search(llmem):
+    cfgs = np.concatenate([grids.g2_shapes(0, 300), grids.g3_sweep(0, 200), grids.g5_stress(0, 100)])
+    cfgs["layers"][5] = 0
+    cfgs["chunk_elems"][6] = -3            # ignored
+    for cs_min, step, count in ((1 << 20, 1 << 16, 257), (1 << 22, 1 << 22, 8), (12345, 1, 33), (1 << 40, 1, 1)):
+        want = oracle.chunk_search(cfgs, cs_min, step, count)
+        got = llmem.chunk_search(cfgs, cs_min, step, count)
+        for k in ("chunk", "waste", "status"):
+            assert np.array_equal(got[k].cpu().numpy(), want[k]), (k, cs_min)
+    L = llmem.lib()
+    assert L.llmem_chunk_search(None, 0, 0, 1, 1, None, None, None, None, 0, 0, None) == llmem.ERR_ARG
+    assert L.llmem_chunk_search(None, 0, 1 << 40, 1, 2, None, None, None, None, 0, 0, None) == llmem.ERR_ARG

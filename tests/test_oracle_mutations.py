@@ -56,6 +56,10 @@ MUTANTS = [
      "if (score2 >= best_score && score2 > 0) {", 1),
     ("segmented_dp_degree", "score2 = (i128)2 * b * (c->gpu_n / c->tp_n);", "score2 = (i128)2 * b * c->tp_n;", 1),
     ("segmented_cdp_factor", "score2 = (i128)3 * b * c->gpu_n;", "score2 = (i128)2 * b * c->gpu_n;", 1),
+    ("chunk_search_last_minimum", "if (best_cs < 0 || waste < best_waste) { /* strict: the first of equals stays */",
+     "if (best_cs < 0 || waste <= best_waste) {", 1),
+    ("chunk_search_floor", "u128 waste = ceil_div(z.other_p, cs) * cs - z.other_p;",
+     "u128 waste = (z.other_p / cs + 1) * cs - z.other_p;", 1),
     ("frees_forgotten_gather", "      for (int64_t j = 0; j < C; ++j) emit(s, -1, z->gat_chunk);\n", "", 1),
 ]
 

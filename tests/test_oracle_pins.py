@@ -646,3 +646,34 @@ def test_segmented_selection_hand_cases():
     r = oracle.select_segmented(items, bs[:, :2], [0, 0, 3, 5])
     assert r["item"][:, 0].tolist() == [-1, 2, 3] and r["method"][:, 0].tolist() == [4, 2, 3]
     assert r["item"][:, 1].tolist() == [-1, -1, 3]
+
+
+# --------------------------------------------------------------------------
+# extension: chunk size search (Section 4.1, one sentence; waste per Section 4.2's m_p)
+# --------------------------------------------------------------------------
+def test_chunk_search_against_brute_force_and_closed_forms():
+    shapes = [mk(), mk(has_bias=1, pos_len=2048), mk(ffn_kind=1, ffn=5632, layers=7),
+              mk(layers=1, hidden=64, heads=1, ffn=192, vocab=1000, has_bias=1)]
+    for c in shapes:
+        f = cfg_fields(c)
+        other_p = sum(n for k, n in enumerate_tensors(f) if k != "E")
+        for cs_min, step, count in ((1 << 20, 1 << 18, 64), (1000, 7, 500), (other_p, 1, 1), (1, 1, 300)):
+            r = oracle.chunk_search(c, cs_min, step, count)
+            wastes = [-(-other_p // cs) * cs - other_p for cs in range(cs_min, cs_min + step * count, step)]
+            k = wastes.index(min(wastes))                  # first minimum
+            assert r["status"][0] == 0
+            assert int(r["chunk"][0]) == cs_min + k * step and int(r["waste"][0]) == wastes[k]
+        # a candidate that divides other_p wastes nothing and is found among worse neighbours
+        d = next(x for x in range(4097, 100000) if other_p % x == 0) if any(
+            other_p % x == 0 for x in range(4097, 100000)) else None
+        if d:
+            r = oracle.chunk_search(c, d - 3, 1, 7)
+            assert int(r["waste"][0]) == 0 and other_p % int(r["chunk"][0]) == 0
+        # one chunk holds everything: waste = cs - other_p
+        r = oracle.chunk_search(c, other_p + 5, 10, 3)
+        assert (int(r["chunk"][0]), int(r["waste"][0])) == (other_p + 5, 5)
+    bad = mk(layers=0)
+    r = oracle.chunk_search(bad, 1 << 20, 1 << 20, 4)
+    assert r["status"][0] == 1 and r["chunk"][0] == -1 and r["waste"][0] == -1
+    ignored = mk(chunk_elems=0, batch=0)                   # these two fields play no part
+    assert oracle.chunk_search(ignored, 1 << 20, 1 << 20, 4)["status"][0] == 0
