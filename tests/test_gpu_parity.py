@@ -333,3 +333,57 @@ def test_chunk_search(llmem):
     L = llmem.lib()
     assert L.llmem_chunk_search(None, 0, 0, 1, 1, None, None, None, None, 0, 0, None) == llmem.ERR_ARG
     assert L.llmem_chunk_search(None, 0, 1 << 40, 1, 2, None, None, None, None, 0, 0, None) == llmem.ERR_ARG
+
+
+def fuzz_configs(n, seed):
+    """Random admissible and inadmissible records over wide field ranges, small enough for
+    the level-1 oracle: every method, degrees up to 255, up to 40 iterations, both FFN kinds,
+    with and without biases and position embeddings, sequence length 1 included."""
+    rng = np.random.default_rng(seed)
+    c = grids.empty(n)
+    heads = rng.choice([1, 2, 4, 8], size=n)
+    c["heads"] = heads
+    c["hidden"] = heads * rng.integers(8, 129, size=n)
+    c["layers"] = rng.integers(1, 13, size=n)
+    c["ffn"] = rng.integers(16, 4097, size=n)
+    c["vocab"] = rng.integers(1, 70000, size=n)
+    c["pos_len"] = rng.choice([0, 0, 1, 77, 4096], size=n)
+    c["seq"] = rng.choice([1, 2, 17, 512, 4096, 100000], size=n)
+    c["batch"] = rng.integers(1, 300, size=n)
+    c["chunk_elems"] = rng.choice([1 << 16, 1 << 18, 100003, 1 << 22, 1 << 30], size=n)
+    c["base_bytes"] = rng.integers(0, 1 << 34, size=n)
+    c["method"] = rng.integers(0, 4, size=n)
+    gpu_n = rng.choice([1, 2, 3, 4, 6, 8, 12, 16, 60, 64, 240, 255], size=n)
+    c["gpu_n"] = gpu_n
+    tp = np.zeros(n, dtype=np.int64)
+    for i in range(n):
+        degs = grids.valid_tp_degrees(int(gpu_n[i]))
+        tp[i] = rng.choice(degs) if degs and rng.random() < 0.9 else rng.integers(0, 9)
+    c["tp_n"] = tp
+    c["lm_bytes"] = rng.choice([2, 4], size=n)
+    c["ffn_kind"] = rng.integers(0, 2, size=n)
+    c["has_bias"] = rng.integers(0, 2, size=n)
+    c["iters"] = rng.choice([1, 2, 3, 7, 40], size=n)
+    return c
+
+
+def test_fuzz_all_entry_points(llmem):
+    cfgs = fuzz_configs(2500, 42)
+    want = check_estimate(llmem, cfgs)
+    assert (want["status"] == 2).any() and (want["status"] == 0).sum() > 1500
+    assert want["count"].max() < 200000
+    total = check_materialized(llmem, cfgs, want)
+    assert total > 10 * 4608
+    caps = np.array([1 << 28, 1 << 31, 3 << 32, 1 << 36, 1 << 40], dtype=np.int64)
+    sub = cfgs[::5]
+    want_bs, want_st = oracle.max_batch(sub, caps, 12, level=1, threads=8)
+    got_bs, got_st = llmem.max_batch(sub, caps, 12)
+    assert np.array_equal(got_st.cpu().numpy(), want_st) and np.array_equal(got_bs.cpu().numpy(), want_bs)
+    want_bs, want_st = oracle.max_batch(cfgs, caps, 1 << 20, level=2, threads=8)
+    got_bs, got_st = llmem.max_batch(cfgs, caps, 1 << 20)
+    assert np.array_equal(got_st.cpu().numpy(), want_st) and np.array_equal(got_bs.cpu().numpy(), want_bs)
+    for allzero in (False, True):
+        want_sel = oracle.select_method(cfgs, caps, 1 << 20, flags=1 if allzero else 0, level=2, threads=8)
+        got_sel = llmem.select_method(cfgs, caps, 1 << 20, allzero=allzero)
+        for k in ("method", "batch", "bs_list", "status"):
+            assert np.array_equal(got_sel[k].cpu().numpy(), want_sel[k]), k
