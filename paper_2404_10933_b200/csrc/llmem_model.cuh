@@ -112,18 +112,37 @@ struct Plan {
   u64 out1, logit1, shift1;
 };
 
-__device__ __forceinline__ u64 shard_bytes(u64 bytes, u32 method, u32 n) {
+// Division by a partition degree (1 .. 255) without a hardware-emulated 64-bit divide:
+// with m = ceil(2^64 / d), floor(x / d) = high 64 bits of x * m for every x < 2^56
+// (Granlund and Montgomery, "Division by invariant integers using multiplication", 1994,
+// N = 56 dividend bits, 8 divisor bits).  Every byte count divided here is below 2^56.
+struct Recip {
+  u64 m;
+  u32 d;
+};
+
+__device__ __forceinline__ Recip make_recip(u32 d) {
+  Recip r;
+  r.d = d;
+  r.m = d > 1 ? ~0ull / d + 1 : 0;
+  return r;
+}
+
+__device__ __forceinline__ u64 floor_div(u64 x, const Recip& r) { return r.d <= 1 ? x : __umul64hi(x, r.m); }
+__device__ __forceinline__ u64 ceil_div(u64 x, const Recip& r) { return floor_div(x + (r.d - 1), r); }
+
+__device__ __forceinline__ u64 shard_bytes(u64 bytes, u32 method, const Recip& n) {
   return method == LLMEM_METHOD_CDP ? bytes : ceil_div(bytes, n);
 }
 
 // fp16 bytes of a unit of x elements that exist only while computing:
 // ADP holds the whole of param fp16 (m_p,16 undivided in m_peak^dp);
 // DP+TP holds m_p,16 * (1 - tp_n/gpu_n) (m_peak^dp+tp).
-__device__ __forceinline__ u64 gathered_bytes(u64 x, u32 method, u32 n, u32 t) {
+__device__ __forceinline__ u64 gathered_bytes(u64 x, u32 method, const Recip& n, u32 t) {
   u64 whole = 2 * x;
   u64 kept = ceil_div(whole, n);
   if (method == LLMEM_METHOD_ADP) return whole - kept;
-  if (method == LLMEM_METHOD_DPTP) return whole - (whole * t) / n - kept;
+  if (method == LLMEM_METHOD_DPTP) return whole - floor_div(whole * t, n) - kept;  // whole * t < 2^55
   return 0;
 }
 
@@ -143,7 +162,7 @@ __device__ __forceinline__ Plan make_plan(const Cfg& f, u32 method) {
   Plan p;
   p.status = check_combo(method, f.gpu_n, f.tp_n);
   const u64 H = (u64)f.hidden, F = (u64)f.ffn, V = (u64)f.vocab, P = (u64)f.pos_len;
-  const u64 n = f.gpu_n;
+  const Recip rn = make_recip(f.gpu_n);
   p.e_n = 1 + (f.pos_len > 0);
   p.K = f.ffn_kind ? 7 : 6;
   p.gather = (method == LLMEM_METHOD_ADP || method == LLMEM_METHOD_DPTP);
@@ -158,20 +177,19 @@ __device__ __forceinline__ Plan make_plan(const Cfg& f, u32 method) {
   const u64 cs = (u64)f.chunk_elems;
   const u64 chunks = ceil_div(other_p, cs);
   p.offset = (u64)f.base_bytes + tok_p * (u64)f.lm_bytes;  // < 2^60 + 2^49
-  p.p16_embed = shard_bytes(2 * embed_p, method, f.gpu_n);
-  p.p32_embed = shard_bytes(4 * embed_p, method, f.gpu_n);
-  p.p16_chunk = shard_bytes(2 * cs, method, f.gpu_n);
-  p.p32_chunk = shard_bytes(4 * cs, method, f.gpu_n);
-  p.gat_embed = gathered_bytes(embed_p, method, f.gpu_n, p.tp);
-  p.gat_chunk = gathered_bytes(cs, method, f.gpu_n, p.tp);
-  p.os_tok = shard_bytes(8 * tok_p, method, f.gpu_n);
-  p.os_pos = shard_bytes(8 * pos_p, method, f.gpu_n);
-  p.os_hh = shard_bytes(8 * hh_p, method, f.gpu_n);
-  p.os_hf = shard_bytes(8 * hf_p, method, f.gpu_n);
+  p.p16_embed = shard_bytes(2 * embed_p, method, rn);
+  p.p32_embed = shard_bytes(4 * embed_p, method, rn);
+  p.p16_chunk = shard_bytes(2 * cs, method, rn);
+  p.p32_chunk = shard_bytes(4 * cs, method, rn);
+  p.gat_embed = gathered_bytes(embed_p, method, rn, p.tp);
+  p.gat_chunk = gathered_bytes(cs, method, rn, p.tp);
+  p.os_tok = shard_bytes(8 * tok_p, method, rn);
+  p.os_pos = shard_bytes(8 * pos_p, method, rn);
+  p.os_hh = shard_bytes(8 * hh_p, method, rn);
+  p.os_hf = shard_bytes(8 * hf_p, method, rn);
   p.out1 = 2 * (u64)f.seq * H;                              // <= 2^47
   p.logit1 = (u64)f.lm_bytes * (u64)f.seq * V;              // <= 2^54
   p.shift1 = (u64)f.lm_bytes * (u64)(f.seq - 1) * V;
-  (void)n;
   if (chunks >= kCountLimit) {
     p.C = 0;
     p.count = kCountLimit;
