@@ -11,7 +11,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(CSRC, "libllmem.so")
 SOURCES = ("api.cu", "estimate.cu", "events.cu", "scan.cu", "fused.cu")
-HEADERS = ("llmem_model.cuh", "llmem_host.h", "fold.cuh", "expand.cuh", os.path.join("..", "..", "include", "llmem.h"))
+HEADERS = ("llmem_model.cuh", "llmem_host.h", "fold.cuh", "expand.cuh", "ranges.cuh", os.path.join("..", "..", "include", "llmem.h"))
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -3,6 +3,7 @@
 #include <cstring>
 
 #include "llmem_host.h"
+#include "ranges.cuh"
 
 namespace llmem {
 
@@ -56,8 +57,8 @@ extern "C" size_t llmem_scratch_bytes(int op, int64_t n, int64_t total_events) {
       return kScratchHeader + (size_t)((n + 1023) / 1024 + 1) * sizeof(int64_t);
     case LLMEM_OP_SCAN_PEAK:
     case LLMEM_OP_EXPAND_SCAN:
-      // header + a head and a tail partial (32 bytes each) per warp of the persistent grid
-      return kScratchHeader + (size_t)kMaxScanWarps * 2 * 32;
+      // header, block starts and a head and a tail partial per warp of the persistent grid
+      return kStreamScratchBytes;
     default:
       return 0;
   }

@@ -8,6 +8,7 @@
 
 #include "llmem_host.h"
 #include "expand.cuh"
+#include "ranges.cuh"
 
 namespace llmem {
 
@@ -124,18 +125,18 @@ add_block_base_kernel(i64* __restrict__ offsets, i64 n, const u64* __restrict__ 
 // latencies.  Lane l owns events [18 l, 18 l + 18) of a chunk.
 __global__ void __launch_bounds__(kExpThreads)
 expand_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict__ offsets, i64 total,
-              i64* __restrict__ out, i64 chunks_per_warp, int round, int bulk_ok) {
+              i64* __restrict__ out, i64 n_warps, i64 kappa, int round, int bulk_ok) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   ExpandWarpSmem& ws = reinterpret_cast<ExpandWarpSmem*>(smem_raw)[warp];
   const i64 gw = (i64)blockIdx.x * kExpWarps + warp;
-  const i64 nchunks = (total + kExpChunk - 1) / kExpChunk;
-  const i64 c_lo = gw * chunks_per_warp;
-  const i64 c_hi = c_lo + chunks_per_warp < nchunks ? c_lo + chunks_per_warp : nchunks;
+  if (gw >= n_warps) return;
+  // this warp's block of chunks: balanced by events + kappa per segment (ranges.cuh)
+  i64 seg;  // smallest segment whose end lies beyond the current position; gs/ge its range
+  const i64 b_lo = warp_block_start(offsets, n, 0, total, gw, n_warps, kappa, kExpChunk, lane, &seg);
+  const i64 b_hi = warp_block_start(offsets, n, 0, total, gw + 1, n_warps, kappa, kExpChunk, lane, nullptr);
+  const i64 c_lo = b_lo / kExpChunk, c_hi = (b_hi + kExpChunk - 1) / kExpChunk;
   if (c_lo >= c_hi) return;
-
-  // seg: smallest segment whose end lies beyond the current position; gs/ge its range
-  i64 seg = first_segment_after(offsets, n, c_lo * kExpChunk);
   i64 gs = seg < n ? __ldg(offsets + seg) : total;
   i64 ge = seg < n ? __ldg(offsets + seg + 1) : total;
   i64 desc_seg = -1;  // segment described by ws.desc
@@ -356,15 +357,13 @@ extern "C" llmem_status llmem_expand_events(const llmem_config* cfg, int64_t n, 
     configured_dev = dev;
   }
   const i64 nchunks = (total_events + kExpChunk - 1) / kExpChunk;
-  i64 grid = (i64)sm_count() * kExpCtasPerSm;
-  i64 warps = grid * kExpWarps;
+  i64 warps = (i64)sm_count() * kExpCtasPerSm * kExpWarps;
+  if (warps > kMaxStreamWarps) warps = kMaxStreamWarps;
   if (warps > nchunks) warps = nchunks;
-  const i64 chunks_per_warp = (nchunks + warps - 1) / warps;
-  warps = (nchunks + chunks_per_warp - 1) / chunks_per_warp;
-  grid = (warps + kExpWarps - 1) / kExpWarps;
+  const i64 grid = (warps + kExpWarps - 1) / kExpWarps;
   expand_kernel<<<(unsigned)grid, kExpThreads, smem, static_cast<cudaStream_t>(cuda_stream)>>>(
       cfg, n, reinterpret_cast<const i64*>(offsets), total_events, reinterpret_cast<i64*>(delta_out),
-      chunks_per_warp, (flags & LLMEM_FUSE_ROUND) ? 1 : 0, aligned_to(delta_out, 16) ? 1 : 0);
+      warps, kExpSegmentCost, (flags & LLMEM_FUSE_ROUND) ? 1 : 0, aligned_to(delta_out, 16) ? 1 : 0);
   return check_launch("llmem_expand_events");
 }
 

@@ -25,6 +25,12 @@ constexpr int kExpPerLane = LLMEM_EXP_PER_LANE;
 constexpr int kExpChunk = 32 * kExpPerLane;  // 576 events, 4608 bytes: one warp's unit of work
 constexpr int kExpCtasPerSm = LLMEM_EXP_CTAS_PER_SM;
 static_assert(kExpPerLane % 2 == 0 && (kExpPerLane / 2) % 2 == 1, "per-lane span: odd number of 16-byte words");
+// What a segment boundary costs the expansion, in events (descriptor build, cursor seeks):
+// the kappa of the cost-balanced work split.
+#ifndef LLMEM_EXP_SEGMENT_COST
+#define LLMEM_EXP_SEGMENT_COST 6144
+#endif
+constexpr i64 kExpSegmentCost = LLMEM_EXP_SEGMENT_COST;
 constexpr int kRuns = 17;
 
 // A run of events that repeat with a short period: the first `split` events of each

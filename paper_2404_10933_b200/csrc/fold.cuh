@@ -225,10 +225,11 @@ __device__ __forceinline__ Fold3 fold_lane_span(const i64* __restrict__ span) {
 }
 
 // Host launcher of the finishing pass (defined with the scan kernels): one thread per
-// segment folds the partials of segments that cross warp ranges of `range_events` events,
-// defines empty segments, adds m_base + lm_p and marks inadmissible configurations.
+// segment folds the partials of segments that cross the warps' blocks (block j starts at
+// bounds[j], bounds[n_warps] = end), defines empty segments, adds m_base + lm_p and marks
+// inadmissible configurations.
 llmem_status launch_scan_finish(const i64* offsets, i64 n, int shift, const llmem_config* cfg, i64* peak_out,
-                                i64* index_out, i64 range_events, const WarpPartials* partials,
+                                i64* index_out, const i64* bounds, i64 n_warps, const WarpPartials* partials,
                                 cudaStream_t stream);
 
 }  // namespace llmem

@@ -6,6 +6,7 @@
 #include "llmem_host.h"
 #include "expand.cuh"
 #include "fold.cuh"
+#include "ranges.cuh"
 
 // Launch shape (overridable at compile time for tuning sweeps).  The fold adds arithmetic
 // to the expansion, so this kernel wants twice the warps of the plain expansion kernel.
@@ -21,6 +22,11 @@ namespace llmem {
 constexpr int kFusedThreads = LLMEM_FUSED_THREADS;
 constexpr int kFusedWarps = kFusedThreads / 32;
 constexpr int kFusedCtasPerSm = LLMEM_FUSED_CTAS_PER_SM;
+// What a segment boundary costs this kernel, in events: the kappa of the work split.
+#ifndef LLMEM_FUSED_SEGMENT_COST
+#define LLMEM_FUSED_SEGMENT_COST 4096
+#endif
+constexpr i64 kFusedSegmentCost = LLMEM_FUSED_SEGMENT_COST;
 
 // kRoundList: the list is written page-rounded (then the fold takes the values as they
 // are); otherwise raw sizes are written and the fold rounds each value as it reads it.
@@ -28,24 +34,26 @@ constexpr int kFusedCtasPerSm = LLMEM_FUSED_CTAS_PER_SM;
 template <bool kRoundList>
 __global__ void __launch_bounds__(kFusedThreads)
 expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict__ offsets, i64 total,
-                   i64* __restrict__ out, i64 chunks_per_warp, int bulk_ok, i64* __restrict__ peak_out,
-                   i64* __restrict__ index_out, WarpPartials* __restrict__ partials) {
+                   i64* __restrict__ out, i64 n_warps, i64 kappa, int bulk_ok, i64* __restrict__ peak_out,
+                   i64* __restrict__ index_out, i64* __restrict__ bounds, WarpPartials* __restrict__ partials) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   ExpandWarpSmem& ws = reinterpret_cast<ExpandWarpSmem*>(smem_raw)[warp];
   const i64 gw = (i64)blockIdx.x * kFusedWarps + warp;
-  const i64 nchunks = (total + kExpChunk - 1) / kExpChunk;
-  const i64 c_lo = gw * chunks_per_warp;
-  const i64 c_hi = c_lo + chunks_per_warp < nchunks ? c_lo + chunks_per_warp : nchunks;
+  if (gw >= n_warps) return;
+  // this warp's block of chunks: balanced by events + kappa per segment (ranges.cuh)
+  i64 seg;  // smallest segment whose end lies beyond the current position; gs/ge its range
+  const i64 b_lo = warp_block_start(offsets, n, 0, total, gw, n_warps, kappa, kExpChunk, lane, &seg);
+  const i64 b_hi = warp_block_start(offsets, n, 0, total, gw + 1, n_warps, kappa, kExpChunk, lane, nullptr);
+  const i64 c_lo = b_lo / kExpChunk, c_hi = (b_hi + kExpChunk - 1) / kExpChunk;
   WarpPartials* my_partials = partials + gw;
   if (lane == 0) {
     my_partials->head = agg_identity();
     my_partials->tail = agg_identity();
+    bounds[gw] = b_lo;
+    if (gw == n_warps - 1) bounds[n_warps] = total;
   }
   if (c_lo >= c_hi) return;
-
-  // seg: smallest segment whose end lies beyond the current position; gs/ge its range
-  i64 seg = first_segment_after(offsets, n, c_lo * kExpChunk);
   i64 gs = seg < n ? __ldg(offsets + seg) : total;
   i64 ge = seg < n ? __ldg(offsets + seg + 1) : total;
   i64 desc_seg = -1;
@@ -153,9 +161,10 @@ extern "C" llmem_status llmem_expand_scan(const llmem_config* cfg, int64_t n, co
     return LLMEM_ERR_SCRATCH;
   }
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-  WarpPartials* partials = reinterpret_cast<WarpPartials*>(static_cast<unsigned char*>(scratch) + kScratchHeader);
+  i64* bounds = reinterpret_cast<i64*>(static_cast<unsigned char*>(scratch) + kBoundsOffset);
+  WarpPartials* partials = reinterpret_cast<WarpPartials*>(static_cast<unsigned char*>(scratch) + kPartialsOffset);
   if (cudaMemsetAsync(scratch, 0, kScratchHeader, s) != cudaSuccess) return check_launch("llmem_expand_scan (memset)");
-  i64 chunks_per_warp = 1;
+  i64 warps = 1;
   if (total_events > 0) {
     const size_t smem = sizeof(ExpandWarpSmem) * kFusedWarps;
     static thread_local int configured_dev = -1;
@@ -168,24 +177,24 @@ extern "C" llmem_status llmem_expand_scan(const llmem_config* cfg, int64_t n, co
       configured_dev = dev;
     }
     const i64 nchunks = (total_events + kExpChunk - 1) / kExpChunk;
-    i64 warps = (i64)sm_count() * kFusedCtasPerSm * kFusedWarps;
-    if (warps > kMaxScanWarps) warps = kMaxScanWarps;
+    warps = (i64)sm_count() * kFusedCtasPerSm * kFusedWarps;
+    if (warps > kMaxStreamWarps) warps = kMaxStreamWarps;
     if (warps > nchunks) warps = nchunks;
-    chunks_per_warp = (nchunks + warps - 1) / warps;
-    warps = (nchunks + chunks_per_warp - 1) / chunks_per_warp;
     const i64 grid = (warps + kFusedWarps - 1) / kFusedWarps;
     const int bulk_ok = aligned_to(delta_out, 16) ? 1 : 0;
     if (flags & LLMEM_FUSE_ROUND)
       expand_scan_kernel<true><<<(unsigned)grid, kFusedThreads, smem, s>>>(
           cfg, n, reinterpret_cast<const i64*>(offsets), total_events, reinterpret_cast<i64*>(delta_out),
-          chunks_per_warp, bulk_ok, reinterpret_cast<i64*>(peak_out), reinterpret_cast<i64*>(peak_index_out), partials);
+          warps, kFusedSegmentCost, bulk_ok, reinterpret_cast<i64*>(peak_out), reinterpret_cast<i64*>(peak_index_out),
+          bounds, partials);
     else
       expand_scan_kernel<false><<<(unsigned)grid, kFusedThreads, smem, s>>>(
           cfg, n, reinterpret_cast<const i64*>(offsets), total_events, reinterpret_cast<i64*>(delta_out),
-          chunks_per_warp, bulk_ok, reinterpret_cast<i64*>(peak_out), reinterpret_cast<i64*>(peak_index_out), partials);
+          warps, kFusedSegmentCost, bulk_ok, reinterpret_cast<i64*>(peak_out), reinterpret_cast<i64*>(peak_index_out),
+          bounds, partials);
     llmem_status st = check_launch("llmem_expand_scan");
     if (st != LLMEM_OK) return st;
   }
   return launch_scan_finish(reinterpret_cast<const i64*>(offsets), n, 0, cfg, reinterpret_cast<i64*>(peak_out),
-                            reinterpret_cast<i64*>(peak_index_out), chunks_per_warp * kExpChunk, partials, s);
+                            reinterpret_cast<i64*>(peak_index_out), bounds, warps, partials, s);
 }

@@ -26,6 +26,5 @@ llmem_status check_launch(const char* what);
 // Layout of the scratch buffer used by llmem_scan_peak and llmem_event_counts:
 // a 256-byte header whose first word is the device status, then the payload.
 constexpr size_t kScratchHeader = 256;
-constexpr int kMaxScanWarps = 4096;  // upper bound on the warps of the scan's persistent grid
 
 }  // namespace llmem

@@ -20,6 +20,7 @@
 // returns.
 #include "llmem_host.h"
 #include "fold.cuh"
+#include "ranges.cuh"
 
 namespace llmem {
 
@@ -40,6 +41,12 @@ constexpr int kScanWarps = kScanThreads / 32;
 constexpr int kScanPerLane = LLMEM_SCAN_PER_LANE;
 constexpr int kScanChunk = 32 * kScanPerLane;  // 832 events = 6656 bytes: one warp's unit of work
 constexpr int kScanStages = LLMEM_SCAN_STAGES;  // chunks in flight per warp
+// What a segment boundary costs the scan, in events (piece fold, reduction, result, next
+// offsets): the kappa of the cost-balanced work split.
+#ifndef LLMEM_SCAN_SEGMENT_COST
+#define LLMEM_SCAN_SEGMENT_COST 3072
+#endif
+constexpr i64 kScanSegmentCost = LLMEM_SCAN_SEGMENT_COST;
 static_assert(kScanPerLane % 2 == 0 && (kScanPerLane / 2) % 2 == 1, "per-lane span: odd number of 16-byte words");
 
 // ---- mbarrier / TMA primitives ---------------------------------------------
@@ -121,8 +128,8 @@ template <bool kRound>
 __global__ void __launch_bounds__(kScanThreads, 1)
 scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, int shift /* 0 or 1 */,
             const i64* __restrict__ offsets, i64 n, i64 total,
-            i64* __restrict__ peak_out, i64* __restrict__ index_out, i64 chunks_per_warp,
-            WarpPartials* __restrict__ partials, u32* __restrict__ status_word) {
+            i64* __restrict__ peak_out, i64* __restrict__ index_out, i64 n_warps, i64 kappa,
+            i64* __restrict__ bounds, WarpPartials* __restrict__ partials, u32* __restrict__ status_word) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   ScanWarpSmem& ws = reinterpret_cast<ScanWarpSmem*>(smem_raw)[warp];
@@ -130,13 +137,17 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
   const i64 gw = (i64)blockIdx.x * kScanWarps + warp;
   // virtual indices: event e lives at v = e + shift, so that v even <=> 16-byte aligned
   const i64 v_begin = shift, v_end = (i64)shift + total;
-  const i64 nchunks = (v_end + kScanChunk - 1) / kScanChunk;
-  const i64 c_lo = gw * chunks_per_warp;
-  const i64 c_hi = c_lo + chunks_per_warp < nchunks ? c_lo + chunks_per_warp : nchunks;
-
+  if (gw >= n_warps) return;
+  // this warp's block of chunks: balanced by events + kappa per segment (ranges.cuh)
+  i64 seg;  // the segment that contains the first event of the current chunk
+  const i64 b_lo = warp_block_start(offsets, n, shift, v_end, gw, n_warps, kappa, kScanChunk, lane, &seg);
+  const i64 b_hi = warp_block_start(offsets, n, shift, v_end, gw + 1, n_warps, kappa, kScanChunk, lane, nullptr);
+  const i64 c_lo = b_lo / kScanChunk, c_hi = (b_hi + kScanChunk - 1) / kScanChunk;
   if (lane == 0) {
     partials[gw].head = agg_identity();
     partials[gw].tail = agg_identity();
+    bounds[gw] = b_lo;
+    if (gw == n_warps - 1) bounds[n_warps] = v_end;
   }
   if (c_lo >= c_hi) return;
   if (lane == 0) {
@@ -169,20 +180,8 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
   if (lane == 0)
     for (i64 c = c_lo; c < c_hi && c < c_lo + kScanStages; ++c) issue(c);
 
-  // seg: the segment that contains the first event of the current chunk
-  i64 seg, seg_vstart, seg_vend;
-  {
-    const i64 first_v = c_lo * kScanChunk > v_begin ? c_lo * kScanChunk : v_begin;
-    i64 lo = 0, hi = n;  // smallest s with offsets[s+1] + shift > first_v
-    while (lo < hi) {
-      const i64 mid = lo + (hi - lo) / 2;
-      if (__ldg(offsets + mid + 1) + shift > first_v) hi = mid;
-      else lo = mid + 1;
-    }
-    seg = lo;
-    seg_vstart = seg < n ? __ldg(offsets + seg) + shift : v_end;
-    seg_vend = seg < n ? __ldg(offsets + seg + 1) + shift : v_end;
-  }
+  i64 seg_vstart = seg < n ? __ldg(offsets + seg) + shift : v_end;
+  i64 seg_vend = seg < n ? __ldg(offsets + seg + 1) + shift : v_end;
   const i64 warp_vlo = c_lo * kScanChunk;  // segments that start at or after this started in this warp's range
   SegmentFolder folder;
   WarpPartials* my_partials = partials + gw;
@@ -248,18 +247,30 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
   }
 }
 
+// Warp whose block [bounds[j], bounds[j+1]) contains event index v: the largest j with
+// bounds[j] <= v (blocks may be empty, then several share a start and the last one owns it).
+__device__ __forceinline__ i64 owner_of(const i64* __restrict__ bounds, i64 n_warps, i64 v) {
+  i64 lo = 0, hi = n_warps - 1;
+  while (lo < hi) {
+    const i64 mid = lo + (hi - lo + 1) / 2;
+    if (__ldg(bounds + mid) <= v) lo = mid;
+    else hi = mid - 1;
+  }
+  return lo;
+}
+
 // Finish, one thread per segment: fold the partials of segments that cross warp
 // ranges, define empty segments, add m_base + lm_p, and mark inadmissible
 // configurations.
 __global__ void __launch_bounds__(256)
 scan_finish_kernel(const i64* __restrict__ offsets, i64 n, int shift, const llmem_config* __restrict__ cfg,
-                   i64* __restrict__ peak_out, i64* __restrict__ index_out, i64 range_events,
-                   const WarpPartials* __restrict__ partials) {
+                   i64* __restrict__ peak_out, i64* __restrict__ index_out, const i64* __restrict__ bounds,
+                   i64 n_warps, const WarpPartials* __restrict__ partials) {
   for (i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (i64)gridDim.x * blockDim.x) {
     const i64 a = offsets[i] + shift, b = offsets[i + 1] + shift;
     i64 mx = 0, idx = -1;
     if (b > a) {
-      const i64 ca = a / range_events, cb = (b - 1) / range_events;
+      const i64 ca = owner_of(bounds, n_warps, a), cb = owner_of(bounds, n_warps, b - 1);
       if (ca == cb) {  // finished by the warp that owns it
         mx = peak_out[i];
         if (index_out) idx = index_out[i];
@@ -278,14 +289,14 @@ scan_finish_kernel(const i64* __restrict__ offsets, i64 n, int shift, const llme
 }
 
 llmem_status launch_scan_finish(const i64* offsets, i64 n, int shift, const llmem_config* cfg, i64* peak_out,
-                                i64* index_out, i64 range_events, const WarpPartials* partials,
+                                i64* index_out, const i64* bounds, i64 n_warps, const WarpPartials* partials,
                                 cudaStream_t stream) {
   i64 blocks = (n + 255) / 256;
   const i64 cap = (i64)sm_count() * 8;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
-  scan_finish_kernel<<<(unsigned)blocks, 256, 0, stream>>>(offsets, n, shift, cfg, peak_out, index_out,
-                                                          range_events < 1 ? 1 : range_events, partials);
+  scan_finish_kernel<<<(unsigned)blocks, 256, 0, stream>>>(offsets, n, shift, cfg, peak_out, index_out, bounds,
+                                                          n_warps < 1 ? 1 : n_warps, partials);
   return check_launch("llmem_scan_peak (finish)");
 }
 
@@ -316,13 +327,14 @@ extern "C" llmem_status llmem_scan_peak(const int64_t* delta, const int64_t* off
   }
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   u32* status_word = static_cast<u32*>(scratch);
-  WarpPartials* partials = reinterpret_cast<WarpPartials*>(static_cast<unsigned char*>(scratch) + kScratchHeader);
+  i64* bounds = reinterpret_cast<i64*>(static_cast<unsigned char*>(scratch) + kBoundsOffset);
+  WarpPartials* partials = reinterpret_cast<WarpPartials*>(static_cast<unsigned char*>(scratch) + kPartialsOffset);
   if (cudaMemsetAsync(status_word, 0, kScratchHeader, s) != cudaSuccess) return check_launch("llmem_scan_peak (memset)");
 
   const int shift = aligned_to(delta, 16) ? 0 : 1;
   const i64* delta_aligned = reinterpret_cast<const i64*>(delta) - shift;
   const bool round = (flags & LLMEM_FUSE_ROUND) != 0;
-  i64 chunks_per_warp = 1;
+  i64 warps = 1;
   if (total_events > 0) {
     const size_t smem = sizeof(ScanWarpSmem) * kScanWarps;
     static thread_local int configured_dev = -1;
@@ -335,23 +347,23 @@ extern "C" llmem_status llmem_scan_peak(const int64_t* delta, const int64_t* off
       configured_dev = dev;
     }
     const i64 nchunks = (total_events + shift + kScanChunk - 1) / kScanChunk;
-    i64 warps = (i64)sm_count() * kScanWarps;
-    if (warps > kMaxScanWarps) warps = kMaxScanWarps;
+    warps = (i64)sm_count() * kScanWarps;
+    if (warps > kMaxStreamWarps) warps = kMaxStreamWarps;
     if (warps > nchunks) warps = nchunks;
-    chunks_per_warp = (nchunks + warps - 1) / warps;
-    warps = (nchunks + chunks_per_warp - 1) / chunks_per_warp;
     const i64 grid = (warps + kScanWarps - 1) / kScanWarps;
     if (round)
       scan_kernel<true><<<(unsigned)grid, kScanThreads, smem, s>>>(
           delta_aligned, shift, reinterpret_cast<const i64*>(offsets), n, total_events,
-          reinterpret_cast<i64*>(peak_out), reinterpret_cast<i64*>(peak_index_out), chunks_per_warp, partials, status_word);
+          reinterpret_cast<i64*>(peak_out), reinterpret_cast<i64*>(peak_index_out), warps, kScanSegmentCost, bounds,
+          partials, status_word);
     else
       scan_kernel<false><<<(unsigned)grid, kScanThreads, smem, s>>>(
           delta_aligned, shift, reinterpret_cast<const i64*>(offsets), n, total_events,
-          reinterpret_cast<i64*>(peak_out), reinterpret_cast<i64*>(peak_index_out), chunks_per_warp, partials, status_word);
+          reinterpret_cast<i64*>(peak_out), reinterpret_cast<i64*>(peak_index_out), warps, kScanSegmentCost, bounds,
+          partials, status_word);
     llmem_status st = check_launch("llmem_scan_peak");
     if (st != LLMEM_OK) return st;
   }
   return launch_scan_finish(reinterpret_cast<const i64*>(offsets), n, shift, cfg, reinterpret_cast<i64*>(peak_out),
-                            reinterpret_cast<i64*>(peak_index_out), chunks_per_warp * kScanChunk, partials, s);
+                            reinterpret_cast<i64*>(peak_index_out), bounds, warps, partials, s);
 }
