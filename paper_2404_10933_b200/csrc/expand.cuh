@@ -181,17 +181,6 @@ __device__ __forceinline__ void bulk_wait_read() {
 }
 __device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
 
-// smallest s in [lo, n] with offsets[s + 1] > pos (n if none)
-__device__ inline i64 first_segment_after(const i64* __restrict__ offsets, i64 n, i64 pos) {
-  i64 lo = 0, hi = n;
-  while (lo < hi) {
-    i64 mid = lo + (hi - lo) / 2;
-    if (__ldg(offsets + mid + 1) > pos) hi = mid;
-    else lo = mid + 1;
-  }
-  return lo;
-}
-
 // One warp's private shared memory: two chunk buffers (filled, then handed to the
 // TMA engine while the other one is being filled) and the descriptor of the
 // segment the warp is currently inside.
