@@ -47,7 +47,7 @@ FALLBACK_HBM_GBS = 6650.0
 # HBM-bound kernels, from an ncu capture of a 4096-configuration run (summary kept under
 # profiles/; traffic grows in proportion to the number of events).  Set an entry
 # to None when its kernel changes after the capture.
-NCU_TRAFFIC_BYTES_PER_EVENT = {"expand": 7.8206, "scan": 8.0145, "expand_scan": 7.8312}
+NCU_TRAFFIC_BYTES_PER_EVENT = {"expand": 7.8224, "scan": 8.0131, "expand_scan": 7.8262}
 
 
 def measured_peaks():
