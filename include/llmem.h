@@ -271,6 +271,17 @@ llmem_status llmem_chunk_search(const llmem_config* DEV cfg, int64_t n, int64_t 
  * undefined). */
 llmem_status llmem_scratch_status(const void* DEV scratch, void* cuda_stream);
 
+/* No counterpart in the paper: a check of this library's own failure handling.  The scan
+ * kernels wait on copy-completion barriers with a time limit; when a wait runs out they
+ * record LLMEM_ERR_TIMEOUT in the scratch status word and return instead of hanging.  This
+ * call exercises exactly that path without touching any data: one warp waits, for at most
+ * limit_ms (1 .. 2000) milliseconds, on a barrier that nothing completes, gives up and
+ * records the status.  Afterwards llmem_scratch_status(scratch, stream) must return
+ * LLMEM_ERR_TIMEOUT and the CUDA context must be as usable as before.
+ *   scratch  DEV, at least 256 bytes, 256-byte aligned */
+llmem_status llmem_selftest_wait_limit(void* DEV scratch, size_t scratch_bytes, uint32_t limit_ms,
+                                       void* cuda_stream);
+
 /* Text of the last error on the calling thread ("" if none). */
 const char* llmem_last_error(void);
 

@@ -34,6 +34,7 @@ EXPORTS = (
     "llmem_round_events", "llmem_scan_peak", "llmem_max_batch", "llmem_select_method",
     "llmem_scratch_status", "llmem_last_error", "llmem_version", "llmem_event_counts_static",
     "llmem_select_segmented", "llmem_expand_scan", "llmem_chunk_search",
+    "llmem_selftest_wait_limit",
 )
 STATIC_MAX_CONFIGS = 4194304
 
@@ -71,6 +72,7 @@ def lib() -> ctypes.CDLL:
         L.llmem_chunk_search.argtypes = [vp, i64, i64, i64, i32, vp, vp, vp, vp, sz, u32, vp]
         L.llmem_expand_scan.argtypes = [vp, i64, vp, i64, vp, vp, vp, vp, sz, u32, vp]
         L.llmem_select_segmented.argtypes = [vp, vp, vp, i64, i64, i32, vp, vp, vp, vp, sz, u32, vp]
+        L.llmem_selftest_wait_limit.argtypes = [vp, sz, u32, vp]
         L.llmem_scratch_status.argtypes = [vp, vp]
         L.llmem_last_error.restype = ctypes.c_char_p
         L.llmem_version.restype = ctypes.c_int

@@ -81,7 +81,8 @@ constexpr u64 kWaitLimitNs = 2000000000ull;  // 2 s
 // Wait for a phase of an mbarrier, giving up after kWaitLimitNs, or at once when
 // `abort_flag` (optional) shows that another lane of the warp has given up.  Returns
 // false on give-up and raises the flag.
-__device__ __forceinline__ bool mbar_wait_bounded(u64* bar, u32 parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_bounded(u64* bar, u32 parity, volatile int* abort_flag,
+                                                  u64 limit_ns = kWaitLimitNs) {
   // common case: the data has landed, or lands within a few polls (each try_wait
   // already suspends the thread for a hardware-defined interval)
 #pragma unroll 1
@@ -92,7 +93,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(u64* bar, u32 parity, volatile
   for (u32 spin = 0;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
     if (abort_flag && *abort_flag) return false;
-    if ((spin & 63u) == 63u && global_timer_ns() - t0 > kWaitLimitNs) {
+    if ((spin & 63u) == 63u && global_timer_ns() - t0 > limit_ns) {
       if (abort_flag) *abort_flag = 1;
       return false;
     }
@@ -247,6 +248,23 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
   }
 }
 
+// Self-test of the bounded wait: one warp waits on an mbarrier that nothing will ever
+// complete, with the given limit; the wait must give up and the warp records
+// LLMEM_ERR_TIMEOUT exactly as the scan kernel would.  Nothing else is touched.
+__global__ void __launch_bounds__(32)
+wait_limit_selftest_kernel(u32* __restrict__ status_word, u64 limit_ns) {
+  __shared__ u64 bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  __syncwarp();
+  const bool ok = mbar_wait_bounded(&bar, 0, &abort_flag, limit_ns);
+  if (!__all_sync(0xffffffffu, ok) && threadIdx.x == 0) atomicExch(status_word, (u32)LLMEM_ERR_TIMEOUT);
+}
+
 // Warp whose block [bounds[j], bounds[j+1]) contains event index v: the largest j with
 // bounds[j] <= v (blocks may be empty, then several share a start and the last one owns it).
 __device__ __forceinline__ i64 owner_of(const i64* __restrict__ bounds, i64 n_warps, i64 v) {
@@ -366,4 +384,21 @@ extern "C" llmem_status llmem_scan_peak(const int64_t* delta, const int64_t* off
   }
   return launch_scan_finish(reinterpret_cast<const i64*>(offsets), n, shift, cfg, reinterpret_cast<i64*>(peak_out),
                             reinterpret_cast<i64*>(peak_index_out), bounds, warps, partials, s);
+}
+
+extern "C" llmem_status llmem_selftest_wait_limit(void* scratch, size_t scratch_bytes, uint32_t limit_ms,
+                                                  void* cuda_stream) {
+  clear_error();
+  if (!scratch || !aligned_to(scratch, 256) || scratch_bytes < kScratchHeader) {
+    set_error("llmem_selftest_wait_limit: scratch of at least 256 bytes, 256-byte aligned, is required");
+    return LLMEM_ERR_SCRATCH;
+  }
+  if (limit_ms < 1 || limit_ms > 2000) {
+    set_error("llmem_selftest_wait_limit: limit_ms must be in 1 .. 2000");
+    return LLMEM_ERR_ARG;
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(scratch, 0, kScratchHeader, s) != cudaSuccess) return check_launch("llmem_selftest_wait_limit (memset)");
+  wait_limit_selftest_kernel<<<1, 32, 0, s>>>(static_cast<u32*>(scratch), (u64)limit_ms * 1000000ull);
+  return check_launch("llmem_selftest_wait_limit");
 }

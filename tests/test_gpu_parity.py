@@ -387,3 +387,27 @@ def test_fuzz_all_entry_points(llmem):
         got_sel = llmem.select_method(cfgs, caps, 1 << 20, allzero=allzero)
         for k in ("method", "batch", "bs_list", "status"):
             assert np.array_equal(got_sel[k].cpu().numpy(), want_sel[k]), k
+
+
+def test_bounded_wait_gives_up_and_reports(llmem):
+    """Failure handling without a fault: a wait on a barrier that nothing completes runs out
+    after its limit, the status word says so, and the context keeps working."""
+    import time
+    L = llmem.lib()
+    scratch = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    assert L.llmem_scratch_status(scratch.data_ptr(), stream) == llmem.OK
+    t0 = time.perf_counter()
+    assert L.llmem_selftest_wait_limit(scratch.data_ptr(), 256, 50, stream) == llmem.OK
+    assert L.llmem_scratch_status(scratch.data_ptr(), stream) == llmem.ERR_TIMEOUT
+    dt = time.perf_counter() - t0
+    assert 0.045 < dt < 1.0, dt
+    assert b"wait" in L.llmem_last_error()
+    # argument checks
+    assert L.llmem_selftest_wait_limit(scratch.data_ptr(), 256, 0, stream) == llmem.ERR_ARG
+    assert L.llmem_selftest_wait_limit(None, 256, 50, stream) == llmem.ERR_SCRATCH
+    # the context is intact: a scan on the same stream right afterwards is correct
+    cfgs = grids.g1_small()[:8]
+    want = oracle.estimate(cfgs)
+    pipe = llmem.estimate_materialized(cfgs)
+    assert np.array_equal(pipe["peak"].cpu().numpy(), want["peak"])
