@@ -53,9 +53,15 @@ def lib() -> ctypes.CDLL:
     global _lib
     if _lib is None:
         if not os.path.exists(LIB_PATH):
-            raise ImportError(
-                f"{LIB_PATH} is missing: build it with `python -m paper_2404_10933_b200._build` "
-                "(needs nvcc); this package has no CPU fallback")
+            # a source checkout without build artefacts: compile in-tree if nvcc is at hand
+            try:
+                from . import _build
+                _build.build()
+            except Exception as e:  # noqa: BLE001
+                raise ImportError(
+                    f"{LIB_PATH} is missing and could not be built ({e}): build it with "
+                    "`python -m paper_2404_10933_b200._build` (needs nvcc); this package has no CPU "
+                    "fallback") from e
         L = ctypes.CDLL(LIB_PATH)
         vp, i64, i32, u32, sz = (ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_uint32,
                                  ctypes.c_size_t)
