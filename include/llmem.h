@@ -65,7 +65,9 @@ typedef struct __attribute__((aligned(16))) llmem_config {
   uint8_t has_bias;    /* 0 / 1: Linear biases and norm biases present */
   uint8_t iters;       /* fine-tuning iterations spanned by the event list, >= 1;
                           2 or more gives the paper's peak */
-  uint8_t reserved[9]; /* must be 0 */
+  uint8_t act_mode;    /* 0: gradient checkpointing, the layer and embedding outputs are kept (the
+                          paper's m_out); 1: every operator output of every layer is kept */
+  uint8_t reserved[8]; /* must be 0 */
 } llmem_config;
 
 enum { LLMEM_METHOD_CDP = 0, LLMEM_METHOD_ADP = 1, LLMEM_METHOD_TP = 2, LLMEM_METHOD_DPTP = 3,

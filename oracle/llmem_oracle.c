@@ -65,7 +65,8 @@ typedef struct {
   uint8_t ffn_kind;    /* 0: two FFN matrices, 1: three (gated) */
   uint8_t has_bias;
   uint8_t iters;
-  uint8_t reserved[9];
+  uint8_t act_mode;    /* 0: gradient checkpointing (layer outputs kept), 1: every operator output kept */
+  uint8_t reserved[8];
 } oracle_config;
 
 _Static_assert(sizeof(oracle_config) == 64, "record is 64 bytes");
@@ -115,7 +116,8 @@ static int validate_fields(const oracle_config *c, int check_batch) {
   if (c->lm_bytes != 2 && c->lm_bytes != 4) return ST_FIELD;
   if (c->ffn_kind > 1 || c->has_bias > 1) return ST_FIELD;
   if (c->iters < 1) return ST_FIELD;
-  for (int i = 0; i < 9; ++i)
+  if (c->act_mode > 1) return ST_FIELD;
+  for (int i = 0; i < 8; ++i)
     if (c->reserved[i] != 0) return ST_FIELD;
   return ST_OK;
 }
@@ -154,6 +156,10 @@ typedef struct {
   u128 gat_embed, gat_chunk;
   u128 os_tok, os_pos, os_hh, os_hf;
   u128 out, logit, shift, back;
+  /* without gradient checkpointing: attention-score and feed-forward sized outputs */
+  u128 act_attn, act_ffn;
+  int n_ops;         /* operator outputs kept per layer (1 with checkpointing) */
+  int op_kind[16];   /* 0: hidden-sized (out), 1: attention scores, 2: feed-forward sized */
 } sizes_t;
 
 /* Persistent fp16 bytes of a unit of x elements.  CDP keeps all of it
@@ -218,6 +224,23 @@ static void compute_sizes(const oracle_config *c, sizes_t *z) {
   z->out = bs * sl * H * B16;
   z->logit = bs * sl * V * (u128)c->lm_bytes;
   z->shift = bs * (sl - 1) * V * (u128)c->lm_bytes;
+  /* Section 4.2 notes that estimation per operator output is supported when gradient
+   * checkpointing is off, without printing an equation.  Reading: every operator of a layer
+   * keeps its fp16 output until backward.  Forward order of a pre-norm decoder layer:
+   * norm, q, k, v, attention scores, softmax, context, output projection, residual, norm,
+   * feed-forward up (two of them plus their product when gated), activation, feed-forward
+   * down, residual.  The last one is the layer output that checkpointing keeps. */
+  z->act_attn = bs * (u128)c->heads * sl * sl * B16;
+  z->act_ffn = bs * sl * F * B16;
+  if (c->act_mode == 0) {
+    z->n_ops = 1;
+    z->op_kind[0] = 0;
+  } else {
+    static const int plain[14] = {0, 0, 0, 0, 1, 1, 0, 0, 0, 0, 2, 2, 0, 0};
+    static const int gated[16] = {0, 0, 0, 0, 1, 1, 0, 0, 0, 0, 2, 2, 2, 2, 0, 0};
+    z->n_ops = c->ffn_kind ? 16 : 14;
+    for (int k = 0; k < z->n_ops; ++k) z->op_kind[k] = c->ffn_kind ? gated[k] : plain[k];
+  }
   /* phase 4: per-layer share of m_back^tp; for plain TP tp_n = gpu_n */
   if (z->tpback) {
     u128 t = (c->method == M_TP) ? c->gpu_n : c->tp_n;
@@ -229,7 +252,7 @@ static void compute_sizes(const oracle_config *c, sizes_t *z) {
 static u128 event_count_formula(const oracle_config *c, const sizes_t *z) {
   u128 init = 2 + 2 * z->C;
   u128 os = (u128)z->e_n + (u128)z->K * (u128)z->L;
-  u128 allocs = (z->gather ? 1 + z->C : 0) + (u128)z->e_n + (u128)z->L + 3 +
+  u128 allocs = (z->gather ? 1 + z->C : 0) + (u128)z->e_n + (u128)z->L * (u128)z->n_ops + 3 +
                 (z->tpback ? (u128)z->L : 0);
   return init + os + (u128)c->iters * 2 * allocs;
 }
@@ -249,6 +272,10 @@ static void emit(sink_t *s, int sign, u128 bytes) {
   s->n++;
 }
 
+static u128 op_size(const sizes_t *z, int k) {
+  return z->op_kind[k] == 0 ? z->out : (z->op_kind[k] == 1 ? z->act_attn : z->act_ffn);
+}
+
 static void walk_events(const oracle_config *c, const sizes_t *z, sink_t *s) {
   int64_t C = (int64_t)z->C, L = z->L;
   /* phase 1: initialisation (Section 4.1) */
@@ -266,7 +293,9 @@ static void walk_events(const oracle_config *c, const sizes_t *z, sink_t *s) {
     }
     /* phase 3: embedding and layer outputs kept for checkpointed backward,
      * then lm_head logits and the two shifted copies for the loss */
-    for (int64_t i = 0; i < z->e_n + L; ++i) emit(s, +1, z->out);
+    for (int64_t i = 0; i < z->e_n; ++i) emit(s, +1, z->out);
+    for (int64_t l = 0; l < L; ++l)
+      for (int k = 0; k < z->n_ops; ++k) emit(s, +1, op_size(z, k));
     emit(s, +1, z->logit);
     emit(s, +1, z->shift);
     emit(s, +1, z->shift);
@@ -279,7 +308,9 @@ static void walk_events(const oracle_config *c, const sizes_t *z, sink_t *s) {
     emit(s, -1, z->shift);
     emit(s, -1, z->shift);
     emit(s, -1, z->logit);
-    for (int64_t i = 0; i < z->e_n + L; ++i) emit(s, -1, z->out);
+    for (int64_t l = 0; l < L; ++l)
+      for (int k = z->n_ops - 1; k >= 0; --k) emit(s, -1, op_size(z, k));
+    for (int64_t i = 0; i < z->e_n; ++i) emit(s, -1, z->out);
     if (z->gather) {
       for (int64_t j = 0; j < C; ++j) emit(s, -1, z->gat_chunk);
       emit(s, -1, z->gat_embed);
@@ -470,7 +501,9 @@ static void static_phases(const oracle_config *c, phases_t *p) {
 }
 
 static u128 dynamic_phase(const sizes_t *z) {
-  return (u128)(z->e_n + z->L) * page_round(z->out) + page_round(z->logit) +
+  u128 per_layer = 0;
+  for (int k = 0; k < z->n_ops; ++k) per_layer += page_round(op_size(z, k));
+  return (u128)z->e_n * page_round(z->out) + (u128)z->L * per_layer + page_round(z->logit) +
          2 * page_round(z->shift) + (z->tpback ? (u128)z->L * page_round(z->back) : 0);
 }
 

@@ -38,7 +38,8 @@ CONFIG_DTYPE = np.dtype(
         ("ffn_kind", "u1"),
         ("has_bias", "u1"),
         ("iters", "u1"),
-        ("reserved", "u1", (9,)),
+        ("act_mode", "u1"),
+        ("reserved", "u1", (8,)),
     ]
 )
 assert CONFIG_DTYPE.itemsize == 64

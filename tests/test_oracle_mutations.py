@@ -45,8 +45,15 @@ MUTANTS = [
     ("attention_tensor_count", "emit(s, +1, k < 4 ? z->os_hh : z->os_hf);", "emit(s, +1, k < 3 ? z->os_hh : z->os_hf);", 1),
     ("cdp_sharded", "return c->method == M_CDP ? bytes : ceil_div(bytes, c->gpu_n);", "return ceil_div(bytes, c->gpu_n);", 1),
     ("outputs_fp32", "z->out = bs * sl * H * B16;", "z->out = bs * sl * H * B32;", 1),
-    ("embedding_outputs_missing", "for (int64_t i = 0; i < z->e_n + L; ++i) emit(s, +1, z->out);",
-     "for (int64_t i = 0; i < L; ++i) emit(s, +1, z->out);", 1),
+    ("embedding_outputs_missing", "for (int64_t i = 0; i < z->e_n; ++i) emit(s, +1, z->out);",
+     "for (int64_t i = 0; i + 1 < z->e_n; ++i) emit(s, +1, z->out);", 1),
+    ("scores_without_heads", "z->act_attn = bs * (u128)c->heads * sl * sl * B16;", "z->act_attn = bs * sl * sl * B16;", 1),
+    ("one_attention_matrix", "static const int plain[14] = {0, 0, 0, 0, 1, 1, 0,", "static const int plain[14] = {0, 0, 0, 0, 1, 0, 0,", 1),
+    ("gated_like_plain", "static const int gated[16] = {0, 0, 0, 0, 1, 1, 0, 0, 0, 0, 2, 2, 2, 2, 0, 0};",
+     "static const int gated[16] = {0, 0, 0, 0, 1, 1, 0, 0, 0, 0, 2, 2, 0, 0, 0, 0};", 1),
+    ("operator_frees_in_forward_order", "for (int k = z->n_ops - 1; k >= 0; --k) emit(s, -1, op_size(z, k));",
+     "for (int k = 0; k < z->n_ops; ++k) emit(s, -1, op_size(z, k));", 1),
+    ("ffn_outputs_hidden_sized", "z->act_ffn = bs * sl * F * B16;", "z->act_ffn = bs * sl * H * B16;", 1),
     ("collapsed_single_iteration", "u128 rel = c->iters >= 2 ? later : (first > after ? first : after);",
      "u128 rel = later;", 1),
     ("collapsed_os_count", "(u128)z->L * (4 * page_round(z->os_hh) + (u128)(z->K - 4) * page_round(z->os_hf));",

@@ -23,7 +23,7 @@ def mk(**kw):
     c = grids.empty(1)
     base = dict(layers=4, hidden=2048, heads=16, ffn=8192, vocab=65536, pos_len=0, seq=1024,
                 batch=32, chunk_elems=1 << 24, base_bytes=123456789, method=0, gpu_n=1, tp_n=0,
-                lm_bytes=2, ffn_kind=0, has_bias=0, iters=2)
+                lm_bytes=2, ffn_kind=0, has_bias=0, iters=2, act_mode=0)
     base.update(kw)
     for k, v in base.items():
         c[k] = v
@@ -68,6 +68,23 @@ def enumerate_tensors(f):
     if bias:
         t.append(("norm", H))
     return t
+
+
+def layer_operator_outputs(f):
+    """(name, elements) of every operator output of one pre-norm decoder layer in forward
+    order, as forward hooks on a framework model would report them.  With gradient
+    checkpointing only the layer's final output stays allocated."""
+    b, S, H, F, A = f["batch"], f["seq"], f["hidden"], f["ffn"], f["heads"]
+    tok = b * S
+    ops = [("norm1", tok * H), ("q", tok * H), ("k", tok * H), ("v", tok * H),
+           ("scores", b * A * S * S), ("softmax", b * A * S * S), ("context", tok * H),
+           ("o_proj", tok * H), ("residual1", tok * H), ("norm2", tok * H)]
+    if f["ffn_kind"]:
+        ops += [("gate", tok * F), ("up", tok * F), ("act", tok * F), ("gate_x_up", tok * F)]
+    else:
+        ops += [("fc1", tok * F), ("act", tok * F)]
+    ops += [("fc2", tok * H), ("residual2", tok * H)]
+    return ops if f["act_mode"] else ops[-1:]
 
 
 def rnd(x):
@@ -299,8 +316,11 @@ def lifetime_table(f):
                 rows.append((2 * x - part(2 * x), s, s))
             elif m == 3:
                 rows.append((2 * x - (2 * x * t) // n - part(2 * x), s, s))
-        for _ in range(e_n + L):
+        for _ in range(e_n):
             rows.append((out, s, s))
+        for _ in range(L):
+            for _name, elems in layer_operator_outputs(f):
+                rows.append((2 * elems, s, s))
         rows.append((f["lm_bytes"] * f["batch"] * f["seq"] * V, s, s))
         for _ in range(2):
             rows.append((f["lm_bytes"] * f["batch"] * (f["seq"] - 1) * V, s, s))
@@ -677,3 +697,45 @@ def test_chunk_search_against_brute_force_and_closed_forms():
     assert r["status"][0] == 1 and r["chunk"][0] == -1 and r["waste"][0] == -1
     ignored = mk(chunk_elems=0, batch=0)                   # these two fields play no part
     assert oracle.chunk_search(ignored, 1 << 20, 1 << 20, 4)["status"][0] == 0
+
+
+# --------------------------------------------------------------------------
+# extension: every operator output kept (no gradient checkpointing).  The paper prints no
+# equation for it (Section 4.2 only says it is supported): parity unpinned to the paper;
+# the pins below tie the oracle to an independent operator enumeration.
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("meth", ALIGNED)
+@pytest.mark.parametrize("shape", [dict(), dict(ffn_kind=1, ffn=8192, layers=3, batch=16, seq=2048, heads=32)])
+def test_all_operator_outputs_closed_form(shape, meth):
+    c0 = mk(**shape, **meth, act_mode=0)
+    c1 = mk(**shape, **meth, act_mode=1)
+    f1 = cfg_fields(c1)
+    ops = layer_operator_outputs(f1)
+    assert len(ops) == (16 if f1["ffn_kind"] else 14)
+    extra = f1["layers"] * (sum(rnd(2 * e) for _, e in ops) - rnd(2 * ops[-1][1]))
+    assert oracle_peak(c1) == oracle_peak(c0) + extra
+    assert oracle_peak(c1, level=2) == oracle_peak(c1)
+    ev0, ev1 = oracle.expand_events(c0), oracle.expand_events(c1)
+    assert len(ev1) - len(ev0) == f1["iters"] * 2 * f1["layers"] * (len(ops) - 1)
+    assert oracle.event_count(c1, formula=True)[1] == len(ev1)
+    # more heads -> larger attention-score tensors; with checkpointing heads play no part
+    c1h = c1.copy(); c1h["heads"] = f1["heads"] * 2
+    assert oracle_peak(c1h) > oracle_peak(c1)
+
+
+@pytest.mark.parametrize("meth", TINY_METHODS)
+@pytest.mark.parametrize("shape", TINY)
+def test_all_operator_outputs_lifetimes_and_stack(shape, meth):
+    c = mk(**shape, **meth, iters=2, base_bytes=999, act_mode=1)
+    f = cfg_fields(c)
+    rows = lifetime_table(f)
+    want = sweep_peak(rows, 5) + 999 + f["vocab"] * f["hidden"] * f["lm_bytes"]
+    assert oracle_peak(c) == want and oracle_peak(c, level=2) == want
+    raw = oracle.expand_events(c)
+    order = []
+    for d in raw.tolist():            # frees release the most recent live allocation (raw sizes:
+        if d > 0:                     # after rounding these tiny tensors would all look alike)
+            order.append(d)
+        elif d < 0:
+            assert order.pop() == -d
+    assert sorted(int(x) for x in raw if x > 0) == sorted(b for b, a, z in rows if b > 0)
