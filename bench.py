@@ -47,7 +47,7 @@ FALLBACK_HBM_GBS = 6650.0
 # HBM-bound kernels, from an ncu capture of a 4096-configuration run (summary kept under
 # profiles/; traffic grows in proportion to the number of events).  Set an entry
 # to None when its kernel changes after the capture.
-NCU_TRAFFIC_BYTES_PER_EVENT = {"expand": 7.8224, "scan": 8.0131, "expand_scan": 7.8262}
+NCU_TRAFFIC_BYTES_PER_EVENT = {"expand": 7.8216, "scan": 8.0130, "expand_scan": 7.8244}
 
 
 def measured_peaks():
@@ -447,7 +447,7 @@ def run_ours(args):
 # ---------------------------------------------------------------------------
 # Warp instructions executed per unit of work (smsp__inst_executed.sum / units) from ncu
 # captures of these kernels on reduced grids; None once a kernel changes after the capture.
-NCU_WARP_INSTR_PER_UNIT = {"estimate_kernel": 44.81, "max_batch_kernel": 24.70, "select_kernel": 127.83}
+NCU_WARP_INSTR_PER_UNIT = {"estimate_kernel": 37.84, "max_batch_kernel": 25.12, "select_kernel": 131.13}
 
 
 def run_register_paths(args):

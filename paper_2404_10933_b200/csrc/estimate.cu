@@ -7,6 +7,15 @@
 #include "llmem_host.h"
 #include "llmem_model.cuh"
 
+// Resident CTAs per SM the register allocation of the per-configuration kernels aims at
+// (overridable at compile time for tuning sweeps).
+#ifndef LLMEM_EST_MIN_CTAS
+#define LLMEM_EST_MIN_CTAS 3
+#endif
+#ifndef LLMEM_SEARCH_MIN_CTAS
+#define LLMEM_SEARCH_MIN_CTAS 4
+#endif
+
 namespace llmem {
 
 // Peak of one admissible plan at a given batch: m_base + lm_p + largest prefix sum.
@@ -30,6 +39,8 @@ struct Search {
 // with a per-configuration reciprocal.
 struct PageSearch {
   u64 out1, logit1, shift1;  // bytes per sample of a layer output / the logits / a shifted copy
+  u64 attn1, ffn1;           // bytes per sample of a score-sized / ffn-sized operator output
+  u32 n_attn, n_ffn;         // how many of those are kept over all layers (0 with checkpointing)
   u64 q1, recip;             // floor(out1 / tp), ceil(2^64 / tp)
   u64 fixed_a, fixed_b;      // pages that do not depend on the batch (see pages())
   u64 offset;                // m_base + lm_p
@@ -41,7 +52,11 @@ struct PageSearch {
   __device__ __forceinline__ void init(const Plan& p, const StaticSums& s, int bmax) {
     out1 = p.out1; logit1 = p.logit1; shift1 = p.shift1;
     offset = p.offset;
-    n_out = (u32)(p.e_n + p.L);
+    n_out = (u32)(p.e_n + p.L * p.n_x);
+    n_attn = (u32)(p.L * p.n_attn);
+    n_ffn = (u32)(p.L * p.n_ffn);
+    attn1 = n_attn ? p.attn1 : 0;
+    ffn1 = n_ffn ? p.ffn1 : 0;
     n_back = (p.tpback && p.tp > 1) ? (u32)p.L : 0u;
     q1 = 0; r1 = 0; recip = 0;
     if (n_back) {
@@ -59,15 +74,21 @@ struct PageSearch {
     // one iteration: max(init + gather + dyn, init + os); otherwise init + os + gather + dyn
     fixed_a = single_iter ? init_p + gat_p : init_p + os_p + gat_p;
     fixed_b = init_p + os_p;
-    const u64 big = out1 > logit1 ? out1 : logit1;  // >= 2
+    u64 big = out1 > logit1 ? out1 : logit1;  // >= 2
+    if (attn1 > big) big = attn1;               // may be saturated: then nothing fits
+    if (ffn1 > big) big = ffn1;
     const u64 lim = (kSat - 1) / big;                // largest b with b * big < 2^62
     b_safe = lim < (u64)bmax ? (int)lim : bmax;
   }
 
+  template <bool kActs>
   __device__ __forceinline__ u64 pages(u32 b) const {
     const u64 out = (u64)b * out1, logit = (u64)b * logit1, shift = (u64)b * shift1;
     u64 dyn = (u64)n_out * ((out + (kPage - 1)) >> 21) + ((logit + (kPage - 1)) >> 21) +
               2 * ((shift + (kPage - 1)) >> 21);
+    if (kActs) {
+      dyn += (u64)n_attn * (((u64)b * attn1 + (kPage - 1)) >> 21) + (u64)n_ffn * (((u64)b * ffn1 + (kPage - 1)) >> 21);
+    }
     if (n_back) {
       // floor(out / tp) = b q1 + floor(b r1 / tp); b r1 < 2^34, exact with the 64-bit reciprocal
       const u64 back = out - ((u64)b * q1 + __umul64hi((u64)b * r1, recip));
@@ -84,10 +105,16 @@ struct PageSearch {
     const u64 cap = capacity >= (i64)kSat ? kSat - 1 : (u64)(capacity < 0 ? 0 : capacity);
     if (capacity < 0 || cap < offset) return 0;
     const u64 budget = (cap - offset) >> 21;
+    // the operator-output terms are decided once, outside the probe loop
+    return n_attn ? bisect<true>(budget) : bisect<false>(budget);
+  }
+
+  template <bool kActs>
+  __device__ __forceinline__ int bisect(u64 budget) const {
     int lo = 0, hi = b_safe;
     while (lo < hi) {
       const int mid = lo + (hi - lo + 1) / 2;
-      if (pages((u32)mid) <= budget) lo = mid;
+      if (pages<kActs>((u32)mid) <= budget) lo = mid;
       else hi = mid - 1;
     }
     return lo;
@@ -97,7 +124,7 @@ struct PageSearch {
 // ---------------------------------------------------------------------------
 // llmem_estimate_batch
 // ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, LLMEM_EST_MIN_CTAS)
 estimate_kernel(const llmem_config* __restrict__ cfg, i64 n, i64* __restrict__ peak_out,
                 i64* __restrict__ index_out, uint8_t* __restrict__ status_out) {
   for (i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (i64)gridDim.x * blockDim.x) {
@@ -122,10 +149,11 @@ estimate_kernel(const llmem_config* __restrict__ cfg, i64 n, i64* __restrict__ p
           // iteration that attains it, or the last optimizer-state allocation
           const u64 init_n = 2 + 2 * (u64)p.C;
           const u64 gpart = p.gather ? 1 + (u64)p.C : 0;
-          const u64 allocs = gpart + (u64)p.e_n + (u64)p.L + 3 + (p.tpback ? (u64)p.L : 0);
+          const u64 outs = (u64)p.e_n + (u64)p.L * (u64)(p.n_x + p.n_attn + p.n_ffn);
+          const u64 allocs = gpart + outs + 3 + (p.tpback ? (u64)p.L : 0);
           const u64 os_n = (u64)p.e_n + (u64)p.K * (u64)p.L;
           const u64 last = (p.tpback && d.back > 0) ? allocs - 1
-                           : (d.shift > 0 ? gpart + p.e_n + p.L + 2 : gpart + p.e_n + p.L);
+                           : (d.shift > 0 ? gpart + outs + 2 : gpart + outs);
           if (p.iters >= 2) ix = (i64)(init_n + 2 * allocs + os_n + last);
           else if (first_wins) ix = (i64)(init_n + last);
           else ix = (i64)(init_n + 2 * allocs + os_n - 1);
@@ -142,7 +170,7 @@ estimate_kernel(const llmem_config* __restrict__ cfg, i64 n, i64* __restrict__ p
 // llmem_max_batch: one thread per shape, capacities innermost (the peak curve
 // does not depend on the capacity, so the plan is built once)
 // ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, LLMEM_SEARCH_MIN_CTAS)
 max_batch_kernel(const llmem_config* __restrict__ shape, i64 n, const i64* __restrict__ caps,
                  int n_cap, int bmax, int* __restrict__ bs_out, uint8_t* __restrict__ status_out) {
   for (i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (i64)gridDim.x * blockDim.x) {
@@ -168,7 +196,7 @@ max_batch_kernel(const llmem_config* __restrict__ shape, i64 n, const i64* __res
 // llmem_select_method: four lanes per shape, lane k searching method k; the
 // quad exchanges its four batches by shuffle and lane 0 takes the decision.
 // ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, LLMEM_SEARCH_MIN_CTAS)
 select_kernel(const llmem_config* __restrict__ shape, i64 n, const i64* __restrict__ caps, int n_cap,
               int bmax, u32 flags, int* __restrict__ method_out, int* __restrict__ batch_out,
               int* __restrict__ bs_list_out, uint8_t* __restrict__ status_out) {

@@ -9,7 +9,7 @@ namespace llmem {
 
 // Launch shape (overridable at compile time for tuning sweeps).
 #ifndef LLMEM_EXP_THREADS
-#define LLMEM_EXP_THREADS 256
+#define LLMEM_EXP_THREADS 384
 #endif
 #ifndef LLMEM_EXP_PER_LANE
 #define LLMEM_EXP_PER_LANE 18
@@ -31,18 +31,22 @@ static_assert(kExpPerLane % 2 == 0 && (kExpPerLane / 2) % 2 == 1, "per-lane span
 #define LLMEM_EXP_SEGMENT_COST 6144
 #endif
 constexpr i64 kExpSegmentCost = LLMEM_EXP_SEGMENT_COST;
-constexpr int kRuns = 17;
+constexpr int kRuns = 19;
+constexpr int kDynFirst = 2, kDynLast = 15, kOsFirst = 16, kOsLast = 18;  // run indices, see SegDesc
 
-// A run of events that repeat with a short period: the first `split` events of each
-// period have value a, the others b.  Constant runs use period 1.
-struct Run {
-  int cnt, period, split, pad;
-  i64 a, b;
+// A run of events that repeat with a short period (at most 16): position j of a period
+// has value v[(code >> 2j) & 3].  Constant runs use period 1 and code 0.
+struct alignas(16) Run {
+  int cnt, period;
+  u32 code;
+  int pad;
+  i64 a, b, c, pad2;
 };
 
-// The event list of one configuration as runs.  Order: 0-1 initialisation,
-// 2-13 one iteration (allocations, then frees mirrored), 14-16 optimizer states,
-// which follow the first iteration only.
+// The event list of one configuration as runs.  Order: 0-1 initialisation; 2-15 one
+// iteration (gather, embedding outputs, per-layer operator outputs, logits, shifted
+// copies, TP buffers, then the frees mirrored); 16-18 optimizer states, which follow the
+// first iteration only.
 struct SegDesc {
   i64 gstart, gend;  // global event range of the segment
   u32 init_n, dyn_n, os_n;
@@ -50,8 +54,24 @@ struct SegDesc {
   Run run[kRuns];
 };
 
-__device__ __forceinline__ void set_run(Run& r, int cnt, int period, int split, i64 a, i64 b) {
-  r.cnt = cnt; r.period = period; r.split = split; r.pad = 0; r.a = a; r.b = b;
+__device__ __forceinline__ void set_run(Run& r, int cnt, int period, u32 code, i64 a, i64 b, i64 c) {
+  r.cnt = cnt; r.period = period; r.code = code; r.pad = 0; r.a = a; r.b = b; r.c = c; r.pad2 = 0;
+}
+__device__ __forceinline__ void set_const_run(Run& r, int cnt, i64 a) { set_run(r, cnt, 1, 0u, a, a, a); }
+
+// 2-bit value selectors of the operator outputs of one layer in forward order
+// (0 hidden-sized, 1 attention-score sized, 2 feed-forward sized): norm, q, k, v, scores,
+// softmax, context, o-proj, residual, norm, up [x2, product], activation, down, residual.
+__device__ __forceinline__ u32 layer_code(bool gated, bool reversed, int* n_ops) {
+  const int n = gated ? 16 : 14;
+  *n_ops = n;
+  u32 code = 0;
+  for (int k = 0; k < n; ++k) {
+    const int kind = (k == 4 || k == 5) ? 1 : ((k >= 10 && k < n - 2) ? 2 : 0);
+    const int pos = reversed ? n - 1 - k : k;
+    code |= (u32)kind << (2 * pos);
+  }
+  return code;
 }
 
 __device__ inline void build_desc(SegDesc& d, const llmem_config* __restrict__ cfg, i64 gstart, i64 gend, bool round) {
@@ -65,42 +85,56 @@ __device__ inline void build_desc(SegDesc& d, const llmem_config* __restrict__ c
   Plan p = make_plan(f, f.method);
   if (p.status != LLMEM_CFG_OK) return;
   Dyn y = make_dyn(p, (u64)f.batch);
-  if (y.out >= kSat || y.logit >= kSat || y.shift >= kSat) return;
+  if (y.out >= kSat || y.logit >= kSat || y.shift >= kSat || y.attn >= kSat || y.ffn >= kSat) return;
   d.invalid = 0;
 #define LLMEM_V(x) ((i64)(round ? page_round(x) : (x)))
   const int C = (int)p.C, L = p.L;
   const int G = p.gather ? 1 : 0, T = p.tpback ? 1 : 0;
-  set_run(d.run[0], 2, 2, 1, LLMEM_V(p.p16_embed), LLMEM_V(p.p32_embed));
-  set_run(d.run[1], 2 * C, 2, 1, LLMEM_V(p.p16_chunk), LLMEM_V(p.p32_chunk));
+  set_run(d.run[0], 2, 2, 1u << 2, LLMEM_V(p.p16_embed), LLMEM_V(p.p32_embed), 0);
+  set_run(d.run[1], 2 * C, 2, 1u << 2, LLMEM_V(p.p16_chunk), LLMEM_V(p.p32_chunk), 0);
   const i64 ge = LLMEM_V(p.gat_embed), gc = LLMEM_V(p.gat_chunk), out = LLMEM_V(y.out);
   const i64 lg = LLMEM_V(y.logit), sh = LLMEM_V(y.shift), bk = LLMEM_V(y.back);
-  set_run(d.run[2], G, 1, 1, ge, ge);
-  set_run(d.run[3], G * C, 1, 1, gc, gc);
-  set_run(d.run[4], p.e_n + L, 1, 1, out, out);
-  set_run(d.run[5], 1, 1, 1, lg, lg);
-  set_run(d.run[6], 2, 1, 1, sh, sh);
-  set_run(d.run[7], T * L, 1, 1, bk, bk);
-  set_run(d.run[8], T * L, 1, 1, -bk, -bk);
-  set_run(d.run[9], 2, 1, 1, -sh, -sh);
-  set_run(d.run[10], 1, 1, 1, -lg, -lg);
-  set_run(d.run[11], p.e_n + L, 1, 1, -out, -out);
-  set_run(d.run[12], G * C, 1, 1, -gc, -gc);
-  set_run(d.run[13], G, 1, 1, -ge, -ge);
-  const i64 ot = LLMEM_V(p.os_tok), op = LLMEM_V(p.os_pos);
-  set_run(d.run[14], 1, 1, 1, ot, ot);
-  set_run(d.run[15], f.pos_len > 0 ? 1 : 0, 1, 1, op, op);
-  set_run(d.run[16], p.K * L, p.K, 4, LLMEM_V(p.os_hh), LLMEM_V(p.os_hf));
+  const i64 at = LLMEM_V(y.attn), ff = LLMEM_V(y.ffn);
+  int n_ops = 1;
+  u32 fwd = 0, bwd = 0;
+  if (f.act_mode) {
+    fwd = layer_code(f.ffn_kind != 0, false, &n_ops);
+    bwd = layer_code(f.ffn_kind != 0, true, &n_ops);
+  }
+  set_const_run(d.run[2], G, ge);
+  set_const_run(d.run[3], G * C, gc);
+  set_const_run(d.run[4], p.e_n, out);
+  set_run(d.run[5], L * n_ops, n_ops, fwd, out, at, ff);
+  set_const_run(d.run[6], 1, lg);
+  set_const_run(d.run[7], 2, sh);
+  set_const_run(d.run[8], T * L, bk);
+  set_const_run(d.run[9], T * L, -bk);
+  set_const_run(d.run[10], 2, -sh);
+  set_const_run(d.run[11], 1, -lg);
+  set_run(d.run[12], L * n_ops, n_ops, bwd, -out, -at, -ff);
+  set_const_run(d.run[13], p.e_n, -out);
+  set_const_run(d.run[14], G * C, -gc);
+  set_const_run(d.run[15], G, -ge);
+  set_const_run(d.run[16], 1, LLMEM_V(p.os_tok));
+  set_const_run(d.run[17], f.pos_len > 0 ? 1 : 0, LLMEM_V(p.os_pos));
+  // per layer: four H x H tensors, then the feed-forward ones
+  set_run(d.run[18], p.K * L, p.K, p.K == 7 ? 0x1500u : 0x0500u, LLMEM_V(p.os_hh), LLMEM_V(p.os_hf), 0);
 #undef LLMEM_V
   d.init_n = 2u + 2u * (u32)C;
-  const u32 allocs = (u32)(G * (1 + C) + p.e_n + L + 3 + T * L);
+  const u32 allocs = (u32)(G * (1 + C) + p.e_n + L * n_ops + 3 + T * L);
   d.dyn_n = 2 * allocs;
   d.os_n = (u32)(p.e_n + p.K * L);
 }
 
 // Cursor of one thread inside a segment.
 struct Cursor {
-  int r, it, rem, phase, period, split;
-  i64 a, b;
+  int r, it, rem, phase, period;
+  u32 code;
+  i64 a, b, c;
+  __device__ __forceinline__ i64 value(int ph) const {
+    const u32 k = (code >> (2 * ph)) & 3u;
+    return k == 0 ? a : (k == 1 ? b : c);
+  }
 };
 
 __device__ __forceinline__ void enter_run(Cursor& c, const SegDesc& d, int r, int o) {
@@ -108,29 +142,30 @@ __device__ __forceinline__ void enter_run(Cursor& c, const SegDesc& d, int r, in
   c.r = r;
   c.rem = rn.cnt - o;
   c.period = rn.period;
-  c.split = rn.split;
+  c.code = rn.code;
   c.a = rn.a;
   c.b = rn.b;
+  c.c = rn.c;
   c.phase = rn.period == 1 ? 0 : (rn.period == 2 ? (o & 1) : (int)((u32)o % (u32)rn.period));
 }
 
-// Position the cursor on event `pos` (0-based inside the segment).
-__device__ __forceinline__ void seek(Cursor& c, const SegDesc& d, u32 pos) {
-  c.it = 1;
+// Run, offset inside it and iteration of event `pos` (0-based inside the segment).
+__device__ __forceinline__ void locate(const SegDesc& d, u32 pos, int* r_out, int* o_out, int* it_out) {
+  *it_out = 1;
   if (pos < d.init_n) {
-    if (pos < 2) enter_run(c, d, 0, (int)pos);
-    else enter_run(c, d, 1, (int)(pos - 2));
+    *r_out = pos < 2 ? 0 : 1;
+    *o_out = pos < 2 ? (int)pos : (int)(pos - 2);
     return;
   }
   u32 q = pos - d.init_n;
-  int r = 2;
+  int r = kDynFirst;
   if (q >= d.dyn_n) {
     q -= d.dyn_n;
     if (q < d.os_n) {
-      r = 14;
+      r = kOsFirst;
     } else {
       q -= d.os_n;
-      c.it = 2 + (int)(q / d.dyn_n);
+      *it_out = 2 + (int)(q / d.dyn_n);
       q = q % d.dyn_n;
     }
   }
@@ -138,7 +173,15 @@ __device__ __forceinline__ void seek(Cursor& c, const SegDesc& d, u32 pos) {
     q -= (u32)d.run[r].cnt;
     ++r;
   }
-  enter_run(c, d, r, (int)q);
+  *r_out = r;
+  *o_out = (int)q;
+}
+
+// Position the cursor on event `pos`.
+__device__ __forceinline__ void seek(Cursor& c, const SegDesc& d, u32 pos) {
+  int r, o;
+  locate(d, pos, &r, &o, &c.it);
+  enter_run(c, d, r, o);
 }
 
 // Move to the next non-empty run.  After the frees of iteration 1 come the optimizer
@@ -146,11 +189,11 @@ __device__ __forceinline__ void seek(Cursor& c, const SegDesc& d, u32 pos) {
 __device__ __forceinline__ void next_run(Cursor& c, const SegDesc& d) {
   int r = c.r;
   for (int guard = 0; guard < 2 * kRuns; ++guard) {
-    if (r == 13) {
-      if (c.it == 1) r = 14;
-      else { r = 2; ++c.it; }
-    } else if (r == 16) {
-      r = 2;
+    if (r == kDynLast) {
+      if (c.it == 1) r = kOsFirst;
+      else { r = kDynFirst; ++c.it; }
+    } else if (r == kOsLast) {
+      r = kDynFirst;
       c.it = 2;
     } else {
       ++r;
@@ -161,7 +204,7 @@ __device__ __forceinline__ void next_run(Cursor& c, const SegDesc& d) {
 }
 
 __device__ __forceinline__ i64 emit(Cursor& c, const SegDesc& d) {
-  const i64 v = c.phase < c.split ? c.a : c.b;
+  const i64 v = c.value(c.phase);
   if (++c.phase == c.period) c.phase = 0;
   if (--c.rem == 0) next_run(c, d);
   return v;
@@ -194,11 +237,14 @@ struct ExpandWarpSmem {
 // all of a long list) are written as constants; anything else goes through the
 // run cursor event by event.
 __device__ __forceinline__ void fill_span(i64* __restrict__ dst, const SegDesc& d, u32 pos, int cnt) {
-  Cursor c;
-  seek(c, d, pos);
-  if (c.rem >= cnt && c.period <= 2) {
-    const i64 x0 = c.phase < c.split ? c.a : c.b;
-    const i64 x1 = c.period == 1 ? x0 : (c.phase < c.split ? c.b : c.a);
+  int r, o, it;
+  locate(d, pos, &r, &o, &it);
+  const Run& rn = d.run[r];
+  if (rn.cnt - o >= cnt && rn.period <= 2) {
+    // period 1: a everywhere; period 2: a on even offsets of the run, b on odd ones
+    const bool odd = rn.period == 2 && (o & 1);
+    const i64 x0 = odd ? rn.b : rn.a;
+    const i64 x1 = rn.period == 2 ? (odd ? rn.a : rn.b) : rn.a;
     if (cnt == kExpPerLane && (smem_addr(dst) & 15u) == 0) {
       longlong2* v = reinterpret_cast<longlong2*>(dst);
 #pragma unroll
@@ -208,6 +254,9 @@ __device__ __forceinline__ void fill_span(i64* __restrict__ dst, const SegDesc& 
     }
     return;
   }
+  Cursor c;
+  c.it = it;
+  enter_run(c, d, r, o);
   for (int j = 0; j < cnt; ++j) dst[j] = emit(c, d);
 }
 

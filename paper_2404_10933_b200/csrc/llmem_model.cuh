@@ -51,7 +51,7 @@ __device__ __forceinline__ u64 ceil_div(u64 a, u64 b) { return (a + b - 1) / b; 
 struct Cfg {
   int layers, hidden, heads, ffn, vocab, pos_len, seq, batch;
   i64 chunk_elems, base_bytes;
-  u32 method, gpu_n, tp_n, lm_bytes, ffn_kind, has_bias, iters;
+  u32 method, gpu_n, tp_n, lm_bytes, ffn_kind, has_bias, iters, act_mode;
   bool reserved_zero;
 };
 
@@ -66,7 +66,8 @@ __device__ __forceinline__ Cfg load_cfg(const llmem_config* __restrict__ p) {
   u32 w0 = (u32)d.x, w1 = (u32)d.y;
   f.method = w0 & 0xff; f.gpu_n = (w0 >> 8) & 0xff; f.tp_n = (w0 >> 16) & 0xff; f.lm_bytes = w0 >> 24;
   f.ffn_kind = w1 & 0xff; f.has_bias = (w1 >> 8) & 0xff; f.iters = (w1 >> 16) & 0xff;
-  f.reserved_zero = ((w1 >> 24) == 0) && d.z == 0 && d.w == 0;
+  f.act_mode = w1 >> 24;
+  f.reserved_zero = d.z == 0 && d.w == 0;
   return f;
 }
 
@@ -79,7 +80,7 @@ __device__ __forceinline__ int check_fields(const Cfg& f, bool check_batch, bool
             f.seq <= (1 << 26) && f.chunk_elems >= 1 && f.chunk_elems <= (1ll << 40) &&
             f.base_bytes >= 0 && f.base_bytes <= (1ll << 60) && f.gpu_n >= 1 &&
             (f.lm_bytes == 2 || f.lm_bytes == 4) && f.ffn_kind <= 1 && f.has_bias <= 1 &&
-            f.iters >= 1 && f.reserved_zero;
+            f.iters >= 1 && f.act_mode <= 1 && f.reserved_zero;
   if (ok) ok = (f.hidden % f.heads) == 0;
   if (ok && check_batch) ok = f.batch >= 1 && f.batch <= (1 << 26);
   if (ok && check_method) ok = f.method <= 3;
@@ -110,6 +111,11 @@ struct Plan {
   u64 os_tok, os_pos, os_hh, os_hf;
   // per-sample factors of the batch-dependent kinds: out = batch * out1, ...
   u64 out1, logit1, shift1;
+  // operator outputs kept per layer: n_x of the size of a layer output, n_attn attention-score
+  // sized (attn1 per sample, saturating), n_ffn feed-forward sized (ffn1 per sample).  With
+  // gradient checkpointing (act_mode 0) only the layer output itself: 1, 0, 0.
+  int n_x, n_attn, n_ffn;
+  u64 attn1, ffn1;
 };
 
 // Division by a partition degree (1 .. 255) without a hardware-emulated 64-bit divide:
@@ -190,14 +196,22 @@ __device__ __forceinline__ Plan make_plan(const Cfg& f, u32 method) {
   p.out1 = 2 * (u64)f.seq * H;                              // <= 2^47
   p.logit1 = (u64)f.lm_bytes * (u64)f.seq * V;              // <= 2^54
   p.shift1 = (u64)f.lm_bytes * (u64)(f.seq - 1) * V;
+  // Without gradient checkpointing every operator of a pre-norm layer keeps its fp16 output:
+  // norm, q, k, v, scores, softmax, context, o-proj, residual, norm, up (x2 + product when
+  // gated), activation, down, residual: 10 hidden-sized, 2 score-sized, 2 or 4 ffn-sized.
+  p.n_x = f.act_mode ? 10 : 1;
+  p.n_attn = f.act_mode ? 2 : 0;
+  p.n_ffn = f.act_mode ? (f.ffn_kind ? 4 : 2) : 0;
+  p.attn1 = sat_mul(sat_mul(2 * (u64)f.heads, (u64)f.seq), (u64)f.seq);
+  p.ffn1 = 2 * (u64)f.seq * F;                              // <= 2^49
   if (chunks >= kCountLimit) {
     p.C = 0;
     p.count = kCountLimit;
     if (p.status == LLMEM_CFG_OK) p.status = LLMEM_CFG_OVERFLOW;
   } else {
     p.C = (u32)chunks;
-    const u64 allocs = (p.gather ? 1 + chunks : 0) + (u64)p.e_n + (u64)p.L + 3 +
-                       (p.tpback ? (u64)p.L : 0);
+    const u64 allocs = (p.gather ? 1 + chunks : 0) + (u64)p.e_n +
+                       (u64)p.L * (u64)(p.n_x + p.n_attn + p.n_ffn) + 3 + (p.tpback ? (u64)p.L : 0);
     p.count = 2 + 2 * chunks + (u64)p.e_n + (u64)p.K * (u64)p.L + (u64)p.iters * 2 * allocs;
     if (p.count >= kCountLimit && p.status == LLMEM_CFG_OK) p.status = LLMEM_CFG_OVERFLOW;
   }
@@ -206,7 +220,7 @@ __device__ __forceinline__ Plan make_plan(const Cfg& f, u32 method) {
 
 // Batch-dependent raw sizes (saturating).
 struct Dyn {
-  u64 out, logit, shift, back;
+  u64 out, logit, shift, back, attn, ffn;
 };
 
 __device__ __forceinline__ Dyn make_dyn(const Plan& p, u64 batch) {
@@ -216,6 +230,8 @@ __device__ __forceinline__ Dyn make_dyn(const Plan& p, u64 batch) {
   d.shift = sat_mul(batch, p.shift1);
   // ceil(out * (tp-1) / tp) = out - floor(out / tp)   (m_back^tp, one layer's share)
   d.back = p.tpback ? d.out - d.out / p.tp : 0;
+  d.attn = p.n_attn ? sat_mul(batch, p.attn1) : 0;
+  d.ffn = p.n_ffn ? sat_mul(batch, p.ffn1) : 0;
   return d;
 }
 
@@ -237,7 +253,9 @@ __device__ __forceinline__ StaticSums make_static_sums(const Plan& p, bool has_p
 
 // Sum of the rounded batch-dependent allocations of one iteration (phases 3 and 4).
 __device__ __forceinline__ u64 dyn_sum(const Plan& p, const Dyn& d) {
-  u64 s = sat_mul((u64)(p.e_n + p.L), page_round(d.out));
+  u64 s = sat_mul((u64)p.e_n + (u64)p.L * (u64)p.n_x, page_round(d.out));
+  if (p.n_attn) s = sat_add(s, sat_mul((u64)p.L * (u64)p.n_attn, page_round(d.attn)));
+  if (p.n_ffn) s = sat_add(s, sat_mul((u64)p.L * (u64)p.n_ffn, page_round(d.ffn)));
   s = sat_add(s, page_round(d.logit));
   s = sat_add(s, sat_mul(2, page_round(d.shift)));
   if (p.tpback) s = sat_add(s, sat_mul((u64)p.L, page_round(d.back)));

@@ -45,6 +45,7 @@ def mixed_small_grid():
     c = c[::7].copy()                        # 398 configs, every method / degree appears
     c["chunk_elems"] = np.where(np.arange(len(c)) % 3 == 0, 1 << 22, c["chunk_elems"])
     c["iters"] = 1 + (np.arange(len(c)) % 3)
+    c["act_mode"] = (np.arange(len(c)) // 2) % 2          # half of them keep every operator output
     bad = grids.g2_shape_grid(41, 1)[:12].copy()
     bad["layers"][0] = 0
     bad["heads"][1] = 7
@@ -54,8 +55,9 @@ def mixed_small_grid():
     bad["batch"][5], bad["seq"][5], bad["vocab"][5] = 1 << 26, 1 << 26, 1 << 26   # >= 2^62 bytes
     bad["layers"][6], bad["hidden"][6], bad["heads"][6], bad["ffn"][6] = 48, 8192, 64, 32768
     bad["chunk_elems"][6] = 1                                         # >= 2^31 events
-    bad["reserved"][7, 8] = 1
+    bad["reserved"][7, 7] = 1
     bad["lm_bytes"][8] = 3
+    bad["act_mode"][8] = 2
     bad["seq"][9] = 1                                                 # valid: zero-byte shifted logits
     bad["method"][10], bad["gpu_n"][10] = 2, 1                        # valid: zero-byte TP buffers
     bad["method"][11], bad["gpu_n"][11] = 1, 1                        # valid: zero-byte gathers
@@ -364,6 +366,7 @@ def fuzz_configs(n, seed):
     c["ffn_kind"] = rng.integers(0, 2, size=n)
     c["has_bias"] = rng.integers(0, 2, size=n)
     c["iters"] = rng.choice([1, 2, 3, 7, 40], size=n)
+    c["act_mode"] = rng.integers(0, 2, size=n)
     return c
 
 
@@ -411,3 +414,35 @@ def test_bounded_wait_gives_up_and_reports(llmem):
     want = oracle.estimate(cfgs)
     pipe = llmem.estimate_materialized(cfgs)
     assert np.array_equal(pipe["peak"].cpu().numpy(), want["peak"])
+
+
+def test_all_operator_outputs_mode(llmem):
+    """act_mode = 1 (no gradient checkpointing) on realistic shapes: estimate, materialised
+    paths, searches and selection against the oracle; the mode must change the result."""
+    base = grids.g3_sweep(5000, 300)
+    base["chunk_elems"] = 1 << 25
+    on = base.copy(); on["act_mode"] = 1
+    want_off = oracle.estimate(base, threads=8)
+    want_on = check_estimate(llmem, on)
+    assert (want_on["peak"] > want_off["peak"]).all()
+    check_materialized(llmem, on[:60], {k: v[:60] for k, v in want_on.items()})
+    caps = grids.g4_capacities()
+    shapes = grids.g4_search_grid(20, 4); shapes["act_mode"] = 1
+    want_bs, want_st = oracle.max_batch(shapes, caps, grids.G4_BMAX, level=2, threads=8)
+    got_bs, got_st = llmem.max_batch(shapes, caps, grids.G4_BMAX)
+    assert np.array_equal(got_st.cpu().numpy(), want_st) and np.array_equal(got_bs.cpu().numpy(), want_bs)
+    small = shapes[::9].copy(); small["chunk_elems"] = 1 << 25
+    want_bs, _ = oracle.max_batch(small, caps, 10, level=1, threads=8)
+    got_bs, _ = llmem.max_batch(small, caps, 10)
+    assert np.array_equal(got_bs.cpu().numpy(), want_bs)
+    sel = grids.g4_select_grid(20, 4); sel["act_mode"] = 1
+    want = oracle.select_method(sel, caps, grids.G4_BMAX, level=2, threads=8)
+    got = llmem.select_method(sel, caps, grids.G4_BMAX)
+    for k in ("method", "batch", "bs_list", "status"):
+        assert np.array_equal(got[k].cpu().numpy(), want[k]), k
+    # attention scores that overflow 2^62 bytes: status 3, nothing fits
+    huge = on[:2].copy(); huge["seq"] = 1 << 26; huge["heads"] = huge["hidden"]; huge["batch"] = 1 << 10
+    check_estimate(llmem, huge)
+    want_bs, want_st = oracle.max_batch(huge, caps, 64, level=2)
+    got_bs, got_st = llmem.max_batch(huge, caps, 64)
+    assert np.array_equal(got_bs.cpu().numpy(), want_bs) and np.array_equal(got_st.cpu().numpy(), want_st)
