@@ -33,7 +33,11 @@
  * per-event and per-term rounding; public parameter counts of two well known
  * decoders; interval-sweep allocator simulation; invariants; hand cases for
  * rounding and for Algorithm 1.  "parity unpinned": Table 2 and Figures 7-9
- * values (m_base, cs and batch sizes are not printed in the paper).
+ * values (m_base, cs and batch sizes are not printed in the paper); and the
+ * operator list of act_mode = 1 (Section 4.2 allows summing per-operator
+ * outputs without gradient checkpointing but prints neither the operators nor a
+ * number: the list here is a reading, pinned only to an independent
+ * enumeration of the same reading and to its reduction to m_out).
  *
  * All arithmetic is integer.  Intermediate values use unsigned __int128 so
  * that the overflow guard (status 3) is decided exactly.
