@@ -143,6 +143,40 @@ def test_g5_stress_materialized_full(llmem):
         assert np.array_equal(delta[off[i]:off[i + 1]].cpu().numpy(), ev)
 
 
+def test_g5_slice_with_all_operator_outputs(llmem):
+    """A quarter of the stress shapes with every operator output kept: materialised, one-pass
+    and in-register results against the oracle, all configurations at level 2, a sample at
+    level 1 with whole lists."""
+    cfgs = grids.g5_stress(0, 16384).copy()
+    cfgs["act_mode"] = 1
+    dev = llmem.to_device(cfgs)
+    offsets, status = llmem.event_counts(dev)
+    total = int(offsets[-1].item())
+    free, _ = torch.cuda.mem_get_info()
+    if free < total * 8 + (2 << 30):
+        pytest.skip(f"needs {total * 8 / 2**30:.0f} GiB of free device memory")
+    want2 = oracle.estimate(cfgs, level=2, threads=THREADS)
+    assert np.array_equal(status.cpu().numpy(), want2["status"])
+    assert (want2["status"] == 0).all()
+    fused = llmem.estimate_batch(dev)
+    assert np.array_equal(fused["status"].cpu().numpy(), want2["status"])
+    assert np.array_equal(fused["peak"].cpu().numpy(), want2["peak"])
+    delta = torch.empty(total, dtype=torch.int64, device="cuda")
+    one = llmem.expand_scan(dev, offsets, total, fuse_round=True, out=delta)
+    assert torch.equal(one["peak"], fused["peak"]) and torch.equal(one["index"], fused["index"])
+    two = llmem.scan_peak(llmem.expand_events(dev, offsets, total, fuse_round=True), offsets, dev)
+    assert torch.equal(two["peak"], fused["peak"]) and torch.equal(two["index"], fused["index"])
+    idx = sample_indices(len(cfgs), 48, 11)
+    want1 = oracle.estimate(cfgs[idx], level=1, threads=THREADS)
+    assert np.array_equal(fused["peak"].cpu().numpy()[idx], want1["peak"])
+    assert np.array_equal(fused["index"].cpu().numpy()[idx], want1["index"])
+    off = offsets.cpu().numpy()
+    assert np.array_equal(np.diff(off)[idx], want1["count"])
+    for i in idx[:4]:
+        ev = oracle.round_events(oracle.expand_events(cfgs[i:i + 1]))
+        assert np.array_equal(delta[off[i]:off[i + 1]].cpu().numpy(), ev)
+
+
 def test_g4_selection_over_all_degrees_and_splits(llmem):
     """Per shape and capacity, the best of 67 candidates: CDP / ADP / TP on 1..16 devices and
     every admissible DP+TP split.  The CUDA pipeline (max_batch on all 8.8 M candidates, then
