@@ -447,7 +447,7 @@ def run_ours(args):
 # ---------------------------------------------------------------------------
 # Warp instructions executed per unit of work (smsp__inst_executed.sum / units) from ncu
 # captures of these kernels on reduced grids; None once a kernel changes after the capture.
-NCU_WARP_INSTR_PER_UNIT = {"estimate_kernel": 37.84, "max_batch_kernel": 25.12, "select_kernel": 131.13}
+NCU_WARP_INSTR_PER_UNIT = {"estimate_kernel": 37.84, "max_batch_kernel": 11.76, "select_kernel": 67.28}
 
 
 def run_register_paths(args):
@@ -487,7 +487,7 @@ def run_register_paths(args):
             return a, b
         unit_name, n_units, extra = "searches/s", units["max_batch_kernel"] + 4 * units["select_kernel"], {
             "selections": units["select_kernel"]}
-        workload = "G4 max-batch search + Algorithm 1 selection, bisection on batch 1..4096 in registers"
+        workload = "G4 max-batch search + Algorithm 1 selection, bracketed bisection on batch 1..4096 in registers"
         launches = 2
     for _ in range(max(args.warmup, 3)):
         step()

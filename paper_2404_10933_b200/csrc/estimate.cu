@@ -48,6 +48,8 @@ struct PageSearch {
   u32 n_out, n_back;         // outputs kept per iteration; TP backward buffers (0 if none or tp = 1)
   int b_safe;                // probes stay within 1..b_safe; 0: nothing can fit
   bool single_iter;
+  double batches_per_page;   // cu_p / W: batches per page of batch-dependent memory (guided search)
+  double dyn_events;         // N: batch-dependent events of one iteration
 
   __device__ __forceinline__ void init(const Plan& p, const StaticSums& s, int bmax) {
     out1 = p.out1; logit1 = p.logit1; shift1 = p.shift1;
@@ -68,6 +70,7 @@ struct PageSearch {
     if (s.init >= kSat || s.os >= kSat || s.gather >= kSat) {
       b_safe = 0;
       fixed_a = fixed_b = 0;
+      batches_per_page = dyn_events = 0.0;
       return;
     }
     const u64 init_p = s.init >> 21, os_p = s.os >> 21, gat_p = s.gather >> 21;
@@ -79,6 +82,11 @@ struct PageSearch {
     if (ffn1 > big) big = ffn1;
     const u64 lim = (kSat - 1) / big;                // largest b with b * big < 2^62
     b_safe = lim < (u64)bmax ? (int)lim : bmax;
+    const double w = (double)n_out * (double)out1 + (double)logit1 + 2.0 * (double)shift1 +
+                     (double)n_attn * (double)attn1 + (double)n_ffn * (double)ffn1 +
+                     (double)n_back * (double)(out1 - q1);
+    batches_per_page = (double)kPage / w;
+    dyn_events = (double)(n_out + n_attn + n_ffn + 2 * n_back + 3);
   }
 
   template <bool kActs>
@@ -99,19 +107,38 @@ struct PageSearch {
   }
 
   // Section 6: the largest b in 1..bmax with peak(b) <= capacity.  Algorithm 1
-  // increments b until the peak exceeds m_total; the peak never decreases with b,
-  // so bisection finds the same b.
+  // increments b until the peak exceeds m_total; the peak never decreases with b, so any
+  // search that ends with "b fits, b + 1 does not" finds the same b.  The page count is
+  // almost linear in b: with W the bytes all batch-dependent events take per sample and N
+  // their number,  b W / cu_p <= dyn pages(b) <= b W / cu_p + N,  which brackets the answer
+  // within about N cu_p / W + 2 batches.  The bracket is computed in floating point, made
+  // certain by probing its two ends (so the result does not depend on rounding there), and
+  // bisected: four or five probes instead of log2(bmax).
   __device__ __forceinline__ int largest_batch(i64 capacity) const {
     const u64 cap = capacity >= (i64)kSat ? kSat - 1 : (u64)(capacity < 0 ? 0 : capacity);
-    if (capacity < 0 || cap < offset) return 0;
+    if (capacity < 0 || cap < offset || b_safe == 0) return 0;
     const u64 budget = (cap - offset) >> 21;
+    if (budget < fixed_a || (single_iter && budget < fixed_b)) return 0;  // pages(b) is at least that
     // the operator-output terms are decided once, outside the probe loop
-    return n_attn ? bisect<true>(budget) : bisect<false>(budget);
+    return n_attn ? guided<true>(budget) : guided<false>(budget);
   }
 
   template <bool kActs>
-  __device__ __forceinline__ int bisect(u64 budget) const {
-    int lo = 0, hi = b_safe;
+  __device__ __forceinline__ int guided(u64 budget) const {
+    const double room = (double)(budget - fixed_a);
+    const double hi_d = room * batches_per_page, lo_d = (room - dyn_events) * batches_per_page;
+    int hi = hi_d >= (double)b_safe ? b_safe : (int)hi_d + 1;
+    if (hi > b_safe) hi = b_safe;
+    int lo = lo_d <= 2.0 ? 0 : (int)lo_d - 1;
+    if (lo > hi) lo = hi;
+    // invariant of the bisection: lo fits (or is 0) and nothing above hi fits
+    if (lo > 0 && pages<kActs>((u32)lo) > budget) {
+      hi = lo - 1;
+      lo = 0;
+    } else if (hi < b_safe && pages<kActs>((u32)hi + 1) <= budget) {
+      lo = hi + 1;
+      hi = b_safe;
+    }
     while (lo < hi) {
       const int mid = lo + (hi - lo + 1) / 2;
       if (pages<kActs>((u32)mid) <= budget) lo = mid;
