@@ -96,7 +96,8 @@ enum { LLMEM_OP_ESTIMATE = 0, LLMEM_OP_EVENT_COUNTS = 1, LLMEM_OP_EXPAND = 2, LL
                                    llmem_scan_peak: round each delta while reading */
 
 /* Bytes of scratch the operation needs for n configurations and total_events
- * events (0 where it needs none; such calls accept scratch = NULL). */
+ * events (0 where it needs none; such calls accept scratch = NULL).  For
+ * LLMEM_OP_EXPAND the scratch is optional (see llmem_expand_events). */
 size_t llmem_scratch_bytes(int op, int64_t n, int64_t total_events);
 
 /* Sections 4.2 and 5, fused: peak of each configuration without materialising
@@ -163,7 +164,12 @@ llmem_status llmem_event_counts_static(const llmem_config* DEV cfg, int64_t n,
  * iteration.  With LLMEM_FUSE_ROUND the magnitudes are page-rounded.
  *   offsets        DEV [n+1] as written by llmem_event_counts for the same cfg
  *   total_events   HOST value of offsets[n]
- *   delta_out      DEV [total_events], 8-byte aligned (16-byte alignment enables bulk stores) */
+ *   delta_out      DEV [total_events], 8-byte aligned (16-byte alignment enables bulk stores)
+ *   scratch        DEV, optional: llmem_scratch_bytes(LLMEM_OP_EXPAND, ..) bytes, 256-byte aligned.
+ *                  It holds the counter from which the warps of a persistent grid claim blocks
+ *                  of the list; with scratch = NULL (or too small) the same blocks are handed
+ *                  out by the hardware block scheduler, one warp per block.  The list written
+ *                  is the same either way. */
 llmem_status llmem_expand_events(const llmem_config* DEV cfg, int64_t n, const int64_t* DEV offsets,
                                  int64_t total_events, int64_t* DEV delta_out, void* DEV scratch,
                                  size_t scratch_bytes, uint32_t flags, void* cuda_stream);

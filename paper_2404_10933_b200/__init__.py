@@ -189,9 +189,9 @@ def event_counts_static(cfg, offsets_out, status_out=None, *, stream=None):
 
 
 def expand_events(cfg, offsets, total_events: Optional[int] = None, *, fuse_round: bool = False,
-                  out=None, stream=None):
+                  out=None, scratch=None, stream=None):
     """Materialise the signed event list.  ``total_events`` defaults to ``offsets[-1]`` (one
-    device-to-host read)."""
+    device-to-host read).  ``scratch`` (optional, 256 bytes) is allocated when not given."""
     torch = _torch()
     cfg = _as_cfg(cfg)
     n = cfg.shape[0]
@@ -201,8 +201,10 @@ def expand_events(cfg, offsets, total_events: Optional[int] = None, *, fuse_roun
         out = torch.empty(total_events, dtype=torch.int64, device=cfg.device)
     elif out.numel() < total_events or out.dtype != torch.int64:
         raise ValueError("out must be an int64 tensor with at least total_events elements")
-    _check(lib().llmem_expand_events(_ptr(cfg), n, _ptr(offsets), total_events, _ptr(out), None, 0,
-                                     FUSE_ROUND if fuse_round else 0, _stream_ptr(stream)))
+    if scratch is None:
+        scratch = torch.empty(scratch_bytes(OP_EXPAND, n, total_events), dtype=torch.uint8, device=cfg.device)
+    _check(lib().llmem_expand_events(_ptr(cfg), n, _ptr(offsets), total_events, _ptr(out), _ptr(scratch),
+                                     scratch.numel(), FUSE_ROUND if fuse_round else 0, _stream_ptr(stream)))
     return out[:total_events] if out.numel() != total_events else out
 
 

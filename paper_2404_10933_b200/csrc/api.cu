@@ -55,9 +55,12 @@ extern "C" size_t llmem_scratch_bytes(int op, int64_t n, int64_t total_events) {
     case LLMEM_OP_EVENT_COUNTS:
       // header + one partial sum per block of 1024 configurations
       return kScratchHeader + (size_t)((n + 1023) / 1024 + 1) * sizeof(int64_t);
+    case LLMEM_OP_EXPAND:
+      // header only: the work counter
+      return kScratchHeader;
     case LLMEM_OP_SCAN_PEAK:
     case LLMEM_OP_EXPAND_SCAN:
-      // header, block starts and a head and a tail partial per warp of the persistent grid
+      // header, block starts and a head and a tail partial per block of the list
       return kStreamScratchBytes;
     default:
       return 0;

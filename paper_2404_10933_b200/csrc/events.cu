@@ -120,85 +120,159 @@ add_block_base_kernel(i64* __restrict__ offsets, i64 n, const u64* __restrict__ 
 // ---------------------------------------------------------------------------
 // expansion (run tables, cursor and store primitives: expand.cuh)
 // ---------------------------------------------------------------------------
-// Every warp streams its own contiguous range of 576-event chunks: no CTA-wide
-// barrier anywhere, so the warps of an SM drift apart and cover each other's
-// latencies.  Lane l owns events [18 l, 18 l + 18) of a chunk.
+// The list is cut into n_blocks contiguous blocks of equal cost (events + kappa per segment,
+// ranges.cuh), many more than the grid has warps; every warp streams one block of 576-event
+// chunks at a time on its own: no CTA-wide barrier anywhere, so the warps of an SM drift
+// apart and cover each other's latencies.  Lane l owns events [18 l, 18 l + 18) of a chunk.
+// With a work counter (caller-provided scratch) the grid is persistent and a warp that has
+// finished its block claims the next unclaimed one; without, the grid has one warp per block
+// and the hardware block scheduler hands out the CTAs.  Either way SMs that reach HBM faster
+// take more of the list.
+//
+// A full chunk inside one run of equal or two alternating events repeats the chunk written
+// from the same buffer two chunks earlier: the buffer is left as it is and only the bulk
+// store is issued.
 __global__ void __launch_bounds__(kExpThreads)
 expand_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict__ offsets, i64 total,
-              i64* __restrict__ out, i64 n_warps, i64 kappa, int round, int bulk_ok) {
+              i64* __restrict__ out, i64 n_blocks, i64 kappa, int round, int bulk_ok,
+              unsigned long long* __restrict__ work_counter) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   ExpandWarpSmem& ws = reinterpret_cast<ExpandWarpSmem*>(smem_raw)[warp];
-  const i64 gw = (i64)blockIdx.x * kExpWarps + warp;
-  if (gw >= n_warps) return;
-  // this warp's block of chunks: balanced by events + kappa per segment (ranges.cuh)
-  i64 seg;  // smallest segment whose end lies beyond the current position; gs/ge its range
-  const i64 b_lo = warp_block_start(offsets, n, 0, total, gw, n_warps, kappa, kExpChunk, lane, &seg);
-  const i64 b_hi = warp_block_start(offsets, n, 0, total, gw + 1, n_warps, kappa, kExpChunk, lane, nullptr);
-  const i64 c_lo = b_lo / kExpChunk, c_hi = (b_hi + kExpChunk - 1) / kExpChunk;
-  if (c_lo >= c_hi) return;
-  i64 gs = seg < n ? __ldg(offsets + seg) : total;
-  i64 ge = seg < n ? __ldg(offsets + seg + 1) : total;
+  const i64 resident = (i64)gridDim.x * kExpWarps;
   i64 desc_seg = -1;  // segment described by ws.desc
-
   int parity = 0;
-  for (i64 c = c_lo; c < c_hi; ++c, parity ^= 1) {
-    const i64 tb = c * kExpChunk;
-    const i64 te = tb + kExpChunk < total ? tb + kExpChunk : total;
-    i64* buf = ws.buf[parity];
-    // the bulk store issued from this buffer two chunks ago must have read it
-    if (lane == 0) bulk_wait_read<1>();
-    __syncwarp();
-    const i64 span_lo = tb + (i64)lane * kExpPerLane;
-    const i64 span_hi = span_lo + kExpPerLane < te ? span_lo + kExpPerLane : te;
-    i64 pos = tb;
-    while (pos < te) {
-      if (seg >= n) {
-        // offsets do not cover the rest of the chunk: define it as zeros
-        for (i64 e = (span_lo > pos ? span_lo : pos); e < span_hi; ++e) buf[e - tb] = 0;
-        break;
-      }
-      if (desc_seg != seg) {
-        __syncwarp();  // every lane is done with the previous descriptor
-        if (lane == 0) build_desc(ws.desc, cfg + seg, gs, ge, round != 0);
-        __syncwarp();
-        desc_seg = seg;
-      }
-      const i64 piece_end = ge < te ? ge : te;
-      const i64 e = span_lo > pos ? span_lo : pos;
-      const i64 e_end = span_hi < piece_end ? span_hi : piece_end;
-      if (e < e_end) {
-        if (ws.desc.invalid) {
-          for (i64 j = e; j < e_end; ++j) buf[j - tb] = 0;
+  i64 key0 = -1, key1 = -1;  // what the two chunk buffers hold: key of an alternating pattern, or -1
+  for (i64 gw = (i64)blockIdx.x * kExpWarps + warp; gw < n_blocks;) {
+    i64 seg;  // smallest segment whose end lies beyond the current position; gs/ge its range
+    const i64 b_lo = warp_block_start(offsets, n, 0, total, gw, n_blocks, kappa, kExpChunk, lane, &seg);
+    const i64 b_hi = warp_block_start(offsets, n, 0, total, gw + 1, n_blocks, kappa, kExpChunk, lane, nullptr);
+    const i64 c_lo = b_lo / kExpChunk, c_hi = (b_hi + kExpChunk - 1) / kExpChunk;
+    i64 gs = seg < n ? __ldg(offsets + seg) : total;
+    i64 ge = seg < n ? __ldg(offsets + seg + 1) : total;
+    // the alternating run the last such chunk lay in: chunks that end at or before run_end
+    // repeat its pattern (x0 on even positions, x1 on odd ones)
+    i64 run_end = -1, run_key = -1, x0 = 0, x1 = 0;
+
+    for (i64 c = c_lo; c < c_hi; ++c, parity ^= 1) {
+      const i64 tb = c * kExpChunk;
+      const i64 te = tb + kExpChunk < total ? tb + kExpChunk : total;
+      i64* buf = ws.buf[parity];
+      bool alternating = false;
+      if (seg < n && gs <= tb && tb + kExpChunk <= ge) {  // a full chunk inside one segment
+        if (tb + kExpChunk <= run_end) {
+          alternating = true;
         } else {
-          fill_span(buf + (e - tb), ws.desc, (u32)(e - gs), (int)(e_end - e));
+          if (desc_seg != seg) {
+            __syncwarp();  // every lane is done with the previous descriptor
+            if (lane == 0) build_desc(ws.desc, cfg + seg, gs, ge, round != 0);
+            __syncwarp();
+            desc_seg = seg;
+          }
+          if (!ws.desc.invalid) {
+            int r, o, it;
+            locate(ws.desc, (u32)(tb - gs), &r, &o, &it);
+            const Run& rn = ws.desc.run[r];
+            if (rn.cnt - o >= kExpChunk && rn.period <= 2) {
+              // period 1: a everywhere; period 2: a on even offsets of the run, b on odd ones
+              const bool odd = rn.period == 2 && (o & 1);
+              x0 = odd ? rn.b : rn.a;
+              x1 = rn.period == 2 ? (odd ? rn.a : rn.b) : rn.a;
+              run_end = tb + (rn.cnt - o);
+              run_key = (seg << 8) | (i64)(r << 1) | (odd ? 1 : 0);
+              alternating = true;
+            }
+          }
         }
       }
-      pos = piece_end;
-      if (ge <= te) {
-        // the segment ends inside this chunk: move to the next non-empty one
-        do {
-          ++seg;
-          gs = seg < n ? __ldg(offsets + seg) : total;
-          ge = seg < n ? __ldg(offsets + seg + 1) : total;
-        } while (seg < n && ge <= pos);
+      if (alternating) {
+        const i64 key = parity ? key1 : key0;
+        if (key != run_key) {
+          // the buffer holds something else: the bulk store issued from it two chunks ago must
+          // have read it, then every lane writes its span (an even offset: x0 comes first)
+          if (lane == 0) bulk_wait_read<1>();
+          __syncwarp();
+          longlong2* v = reinterpret_cast<longlong2*>(buf + lane * kExpPerLane);
+#pragma unroll
+          for (int j = 0; j < kExpPerLane / 2; ++j) v[j] = make_longlong2(x0, x1);
+          if (parity) key1 = run_key; else key0 = run_key;
+          fence_async_shared();
+          __syncwarp();
+        } else if (lane == 0) {
+          bulk_wait_read<kExpStoresInFlight>();
+        }
+        if (ge == te) {
+          // the segment ends with this chunk: move to the next non-empty one
+          do {
+            ++seg;
+            gs = seg < n ? __ldg(offsets + seg) : total;
+            ge = seg < n ? __ldg(offsets + seg + 1) : total;
+          } while (seg < n && ge <= te);
+        }
+      } else {
+        if (parity) key1 = -1; else key0 = -1;
+        // the bulk store issued from this buffer two chunks ago must have read it
+        if (lane == 0) bulk_wait_read<1>();
+        __syncwarp();
+        const i64 span_lo = tb + (i64)lane * kExpPerLane;
+        const i64 span_hi = span_lo + kExpPerLane < te ? span_lo + kExpPerLane : te;
+        i64 pos = tb;
+        while (pos < te) {
+          if (seg >= n) {
+            // offsets do not cover the rest of the chunk: define it as zeros
+            for (i64 e = (span_lo > pos ? span_lo : pos); e < span_hi; ++e) buf[e - tb] = 0;
+            break;
+          }
+          if (desc_seg != seg) {
+            __syncwarp();  // every lane is done with the previous descriptor
+            if (lane == 0) build_desc(ws.desc, cfg + seg, gs, ge, round != 0);
+            __syncwarp();
+            desc_seg = seg;
+          }
+          const i64 piece_end = ge < te ? ge : te;
+          const i64 e = span_lo > pos ? span_lo : pos;
+          const i64 e_end = span_hi < piece_end ? span_hi : piece_end;
+          if (e < e_end) {
+            if (ws.desc.invalid) {
+              for (i64 j = e; j < e_end; ++j) buf[j - tb] = 0;
+            } else {
+              fill_span(buf + (e - tb), ws.desc, (u32)(e - gs), (int)(e_end - e));
+            }
+          }
+          pos = piece_end;
+          if (ge <= te) {
+            // the segment ends inside this chunk: move to the next non-empty one
+            do {
+              ++seg;
+              gs = seg < n ? __ldg(offsets + seg) : total;
+              ge = seg < n ? __ldg(offsets + seg + 1) : total;
+            } while (seg < n && ge <= pos);
+          }
+        }
+        // generic-proxy writes -> async-proxy read
+        if (bulk_ok) fence_async_shared();
+        __syncwarp();
+      }
+      // hand the chunk to the TMA engine
+      const u32 cnt = (u32)(te - tb);
+      if (bulk_ok) {
+        if (lane == 0) {
+          const u32 even = cnt & ~1u;
+          if (even) bulk_store(out + tb, buf, even * 8u);
+          bulk_commit();
+          if (cnt & 1u) out[tb + cnt - 1] = buf[cnt - 1];
+        }
+      } else {
+        for (u32 i = lane; i < cnt; i += 32) out[tb + i] = buf[i];
+        __syncwarp();  // the buffer may be rewritten two chunks from now
       }
     }
-    // hand the chunk to the TMA engine (generic-proxy writes -> async-proxy read)
-    const u32 cnt = (u32)(te - tb);
-    if (bulk_ok) {
-      fence_async_shared();
-      __syncwarp();
-      if (lane == 0) {
-        const u32 even = cnt & ~1u;
-        if (even) bulk_store(out + tb, buf, even * 8u);
-        bulk_commit();
-        if (cnt & 1u) out[tb + cnt - 1] = buf[cnt - 1];
-      }
-    } else {
-      __syncwarp();
-      for (u32 i = lane; i < cnt; i += 32) out[tb + i] = buf[i];
-    }
+    if (work_counter == nullptr) break;  // one block per warp
+    // the first `resident` blocks are taken by number, the others in order of request
+    unsigned long long ticket = 0;
+    if (lane == 0) ticket = atomicAdd(work_counter, 1ull);
+    ticket = __shfl_sync(0xffffffffu, ticket, 0);
+    gw = resident + (i64)ticket;
   }
   if (lane == 0) bulk_wait_read<0>();
 }
@@ -338,7 +412,6 @@ extern "C" llmem_status llmem_event_counts_static(const llmem_config* cfg, int64
 extern "C" llmem_status llmem_expand_events(const llmem_config* cfg, int64_t n, const int64_t* offsets,
                                             int64_t total_events, int64_t* delta_out, void* scratch,
                                             size_t scratch_bytes, uint32_t flags, void* cuda_stream) {
-  (void)scratch; (void)scratch_bytes;
   clear_error();
   if (n < 0 || total_events < 0) { set_error("llmem_expand_events: negative size"); return LLMEM_ERR_ARG; }
   if (total_events == 0) return LLMEM_OK;
@@ -357,13 +430,20 @@ extern "C" llmem_status llmem_expand_events(const llmem_config* cfg, int64_t n, 
     configured_dev = dev;
   }
   const i64 nchunks = (total_events + kExpChunk - 1) / kExpChunk;
-  i64 warps = (i64)sm_count() * kExpCtasPerSm * kExpWarps;
-  if (warps > kMaxStreamWarps) warps = kMaxStreamWarps;
-  if (warps > nchunks) warps = nchunks;
-  const i64 grid = (warps + kExpWarps - 1) / kExpWarps;
-  expand_kernel<<<(unsigned)grid, kExpThreads, smem, static_cast<cudaStream_t>(cuda_stream)>>>(
+  const i64 resident = (i64)sm_count() * kExpCtasPerSm * kExpWarps;
+  const i64 blocks = stream_warps(resident, LLMEM_EXP_OVERSUB, nchunks, LLMEM_EXP_MIN_CHUNKS);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  // with scratch the warps of a persistent grid claim blocks from a counter in its header
+  unsigned long long* work_counter = nullptr;
+  if (scratch && aligned_to(scratch, 256) && scratch_bytes >= kScratchHeader && blocks > resident) {
+    if (cudaMemsetAsync(scratch, 0, kScratchHeader, s) != cudaSuccess) return check_launch("llmem_expand_events (memset)");
+    work_counter = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(scratch) + kWorkCounterOffset);
+  }
+  const i64 grid_warps = work_counter ? resident : blocks;
+  const i64 grid = (grid_warps + kExpWarps - 1) / kExpWarps;
+  expand_kernel<<<(unsigned)grid, kExpThreads, smem, s>>>(
       cfg, n, reinterpret_cast<const i64*>(offsets), total_events, reinterpret_cast<i64*>(delta_out),
-      warps, kExpSegmentCost, (flags & LLMEM_FUSE_ROUND) ? 1 : 0, aligned_to(delta_out, 16) ? 1 : 0);
+      blocks, kExpSegmentCost, (flags & LLMEM_FUSE_ROUND) ? 1 : 0, aligned_to(delta_out, 16) ? 1 : 0, work_counter);
   return check_launch("llmem_expand_events");
 }
 

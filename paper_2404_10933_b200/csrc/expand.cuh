@@ -31,6 +31,19 @@ static_assert(kExpPerLane % 2 == 0 && (kExpPerLane / 2) % 2 == 1, "per-lane span
 #define LLMEM_EXP_SEGMENT_COST 6144
 #endif
 constexpr i64 kExpSegmentCost = LLMEM_EXP_SEGMENT_COST;
+// Blocks of work per resident warp of the expansion kernel and the fewest chunks a block
+// is given (ranges.cuh).
+#ifndef LLMEM_EXP_OVERSUB
+#define LLMEM_EXP_OVERSUB 36
+#endif
+#ifndef LLMEM_EXP_MIN_CHUNKS
+#define LLMEM_EXP_MIN_CHUNKS 128
+#endif
+// Bulk stores a warp may have in flight from buffers it is not rewriting.
+#ifndef LLMEM_EXP_INFLIGHT
+#define LLMEM_EXP_INFLIGHT 8
+#endif
+constexpr int kExpStoresInFlight = LLMEM_EXP_INFLIGHT;
 constexpr int kRuns = 19;
 constexpr int kDynFirst = 2, kDynLast = 15, kOsFirst = 16, kOsLast = 18;  // run indices, see SegDesc
 

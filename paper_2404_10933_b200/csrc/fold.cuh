@@ -168,6 +168,20 @@ struct SegmentFolder {
     seg_has = true;
   }
 
+  // A piece whose fold every lane already holds (the same value in all lanes).
+  __device__ __forceinline__ void add_uniform(const Agg& g, int lane) {
+    if (lane == 0) {
+      const i64 cand = base + g.mx;
+      if (!lane_has || cand > best_v) {
+        best_v = cand;
+        best_i = g.idx;
+        lane_has = true;
+      }
+    }
+    base += g.sum;
+    seg_has = true;
+  }
+
   // All lanes: reduce the state to one Agg (valid in every lane) and reset it.
   __device__ __forceinline__ Agg take() {
 #pragma unroll

@@ -26,5 +26,8 @@ llmem_status check_launch(const char* what);
 // Layout of the scratch buffer used by llmem_scan_peak and llmem_event_counts:
 // a 256-byte header whose first word is the device status, then the payload.
 constexpr size_t kScratchHeader = 256;
+// Byte offset, inside the header, of the 64-bit counter from which the warps of a streaming
+// kernel claim their next block of work.
+constexpr size_t kWorkCounterOffset = 64;
 
 }  // namespace llmem

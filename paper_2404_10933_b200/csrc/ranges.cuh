@@ -18,7 +18,24 @@
 
 namespace llmem {
 
-constexpr int kMaxStreamWarps = 4096;  // upper bound on the warps of a persistent streaming grid
+#ifndef LLMEM_MAX_STREAM_WARPS
+#define LLMEM_MAX_STREAM_WARPS 65536
+#endif
+constexpr int kMaxStreamWarps = LLMEM_MAX_STREAM_WARPS;  // upper bound on the (virtual) warps of a streaming grid
+
+// Warps of a streaming launch.  `resident` is what the GPU holds at once; the grid may hold
+// `oversub` times as many, so that the hardware block scheduler hands out the blocks as SMs
+// become free (SMs do not all reach HBM at the same rate, and a grid of exactly the resident
+// size ends when its slowest SM does).  No warp gets fewer than `min_chunks` chunks unless
+// the resident warps alone would.
+inline i64 stream_warps(i64 resident, int oversub, i64 nchunks, i64 min_chunks) {
+  i64 warps = resident * (oversub < 1 ? 1 : oversub);
+  const i64 by_work = nchunks / (min_chunks < 1 ? 1 : min_chunks);
+  if (warps > by_work) warps = by_work > resident ? by_work : resident;
+  if (warps > kMaxStreamWarps) warps = kMaxStreamWarps;
+  if (warps > nchunks) warps = nchunks;
+  return warps < 1 ? 1 : warps;
+}
 
 // Smallest s in [0, n] with offsets[s + 1] + kappa * (s + 1) > target (n if none), found by
 // the whole warp: every round the 32 lanes probe 32 evenly spaced candidates, so a round costs

@@ -47,6 +47,13 @@ constexpr int kScanStages = LLMEM_SCAN_STAGES;  // chunks in flight per warp
 #define LLMEM_SCAN_SEGMENT_COST 3072
 #endif
 constexpr i64 kScanSegmentCost = LLMEM_SCAN_SEGMENT_COST;
+// Virtual warps per resident warp and the fewest chunks a virtual warp is given (ranges.cuh).
+#ifndef LLMEM_SCAN_OVERSUB
+#define LLMEM_SCAN_OVERSUB 1
+#endif
+#ifndef LLMEM_SCAN_MIN_CHUNKS
+#define LLMEM_SCAN_MIN_CHUNKS 64
+#endif
 static_assert(kScanPerLane % 2 == 0 && (kScanPerLane / 2) % 2 == 1, "per-lane span: odd number of 16-byte words");
 
 // ---- mbarrier / TMA primitives ---------------------------------------------
@@ -365,9 +372,7 @@ extern "C" llmem_status llmem_scan_peak(const int64_t* delta, const int64_t* off
       configured_dev = dev;
     }
     const i64 nchunks = (total_events + shift + kScanChunk - 1) / kScanChunk;
-    warps = (i64)sm_count() * kScanWarps;
-    if (warps > kMaxStreamWarps) warps = kMaxStreamWarps;
-    if (warps > nchunks) warps = nchunks;
+    warps = stream_warps((i64)sm_count() * kScanWarps, LLMEM_SCAN_OVERSUB, nchunks, LLMEM_SCAN_MIN_CHUNKS);
     const i64 grid = (warps + kScanWarps - 1) / kScanWarps;
     if (round)
       scan_kernel<true><<<(unsigned)grid, kScanThreads, smem, s>>>(
