@@ -47,7 +47,7 @@ FALLBACK_HBM_GBS = 6650.0
 # HBM-bound kernels, from an ncu capture of a 4096-configuration run (summary kept under
 # profiles/; traffic grows in proportion to the number of events).  Set an entry
 # to None when its kernel changes after the capture.
-NCU_TRAFFIC_BYTES_PER_EVENT = {"expand": None, "scan": 8.0130, "expand_scan": None}
+NCU_TRAFFIC_BYTES_PER_EVENT = {"expand": 7.8238, "scan": 8.0130, "expand_scan": 7.8256}
 
 
 def measured_peaks():
@@ -77,7 +77,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "50",
                  "-i", str(self.device_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -136,7 +136,7 @@ def time_oracle(cfgs, threads: int):
     return int(r["count"].sum()), dt
 
 
-def cpu_baseline(sample_configs: int = 16384):
+def cpu_baseline(sample_configs: int = 49152):
     cores = os.cpu_count() or 1
     events, dt = time_oracle(oracle_sample(sample_configs), cores)
     return {"value": events / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
@@ -538,7 +538,7 @@ def run_register_paths(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
     ap.add_argument("--configs", type=int, default=grids.G5_CONFIGS,

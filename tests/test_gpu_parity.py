@@ -215,6 +215,40 @@ def test_expand_into_unaligned_output(llmem):
     assert buf[0].item() == -7 and (buf[1 + total:] == -7).all()
 
 
+def test_long_runs_all_store_paths(llmem):
+    """Lists made of long runs of equal or alternating events (deep/wide decoders): most chunks
+    are issued from a buffer that is not refilled and folded in closed form.  Both kernels,
+    rounded and raw lists, aligned and unaligned outputs, with and without the work counter."""
+    cfgs = grids.g5_stress(3, 40)
+    cfgs["iters"][::3] = 1                     # lists that end with the optimizer states
+    cfgs["iters"][1::7] = 3
+    cfgs["act_mode"][::4] = 1                  # periodic operator-output runs between the long ones
+    dev = llmem.to_device(cfgs)
+    offsets, _ = llmem.event_counts(dev)
+    est = oracle.estimate(cfgs, threads=8)
+    assert (est["status"] == 0).all()
+    total = int(offsets[-1].item())
+    assert total > 1000 * 576
+    no_scratch = torch.empty(0, dtype=torch.uint8, device="cuda")
+    for rounded in (True, False):
+        want, off_want = oracle_lists(cfgs, rounded=rounded)
+        assert np.array_equal(offsets.cpu().numpy(), off_want)
+        for shift in (0, 1):
+            buf = torch.full((total + 4,), -7, dtype=torch.int64, device="cuda")
+            view = buf[shift:shift + total]
+            for scratch in (None, no_scratch):
+                buf.fill_(-7)
+                out = llmem.expand_events(dev, offsets, total, fuse_round=rounded, out=view, scratch=scratch)
+                assert np.array_equal(out.cpu().numpy(), want), (rounded, shift, scratch is None)
+                assert (buf[:shift] == -7).all() and (buf[shift + total:] == -7).all()
+            buf.fill_(-7)
+            r = llmem.expand_scan(dev, offsets, total, fuse_round=rounded, out=view)
+            assert np.array_equal(r["delta"].cpu().numpy(), want), (rounded, shift)
+            assert np.array_equal(r["peak"].cpu().numpy(), est["peak"]), (rounded, shift)
+            assert np.array_equal(r["index"].cpu().numpy(), est["index"]), (rounded, shift)
+            assert (buf[:shift] == -7).all() and (buf[shift + total:] == -7).all()
+
+
 def test_max_batch_and_select_small(llmem):
     shapes = grids.g4_search_grid(0, 8)              # 8 shapes x 4 methods x 16 degrees
     shapes["chunk_elems"] = 1 << 25                  # keeps the literal (level-1) oracle quick
