@@ -62,9 +62,9 @@ struct PageSearch {
     n_back = (p.tpback && p.tp > 1) ? (u32)p.L : 0u;
     q1 = 0; r1 = 0; recip = 0;
     if (n_back) {
-      q1 = out1 / p.tp;
+      recip = p.tp_recip;             // ceil(2^64 / tp), tp >= 2
+      q1 = __umul64hi(out1, recip);   // floor(out1 / tp): exact, out1 < 2^48
       r1 = (u32)(out1 - q1 * p.tp);
-      recip = ~0ull / p.tp + 1;  // ceil(2^64 / tp), tp >= 2
     }
     single_iter = p.iters < 2;
     if (s.init >= kSat || s.os >= kSat || s.gather >= kSat) {

@@ -103,6 +103,7 @@ struct Plan {
   int tpback;     // phase 4 present: TP, DP+TP
   int L, iters;
   u32 tp;         // TP degree of the backward buffers: gpu_n for TP, tp_n for DP+TP
+  u64 tp_recip;   // ceil(2^64 / tp), 0 for tp = 1
   u32 C;          // chunks = ceil(other_p / cs); < 2^31 when status == 0
   u64 count;      // number of events
   u64 offset;     // m_base + lm_p (added unrounded, Section 4.2)
@@ -127,15 +128,46 @@ struct Recip {
   u32 d;
 };
 
-__device__ __forceinline__ Recip make_recip(u32 d) {
+// ceil(2^64 / d) for every degree a configuration record can hold, built at compile time.
+struct RecipTable {
+  u64 m[256];
+};
+constexpr RecipTable make_recip_table() {
+  RecipTable t{};
+  for (unsigned d = 2; d < 256; ++d) t.m[d] = ~0ull / d + 1;
+  return t;
+}
+static __device__ const RecipTable kRecipTable = make_recip_table();
+
+__device__ __forceinline__ Recip make_recip(u32 d) {  // d <= 255
   Recip r;
   r.d = d;
-  r.m = d > 1 ? ~0ull / d + 1 : 0;
+  r.m = __ldg(&kRecipTable.m[d & 255u]);
   return r;
 }
 
 __device__ __forceinline__ u64 floor_div(u64 x, const Recip& r) { return r.d <= 1 ? x : __umul64hi(x, r.m); }
 __device__ __forceinline__ u64 ceil_div(u64 x, const Recip& r) { return floor_div(x + (r.d - 1), r); }
+
+// min(ceil(a / b), 2^31) for a < 2^61, 1 <= b <= 2^40: the number of chunks, or the event
+// limit if there would be that many.  ceil(a / b) >= 2^31 exactly when a > (2^31 - 1) b;
+// below that the double-precision quotient is within one of the integer one (relative error
+// 2^-52 on a value below 2^31) and one multiplication settles it.
+__device__ __forceinline__ u64 chunk_count(u64 a, u64 b) {
+  const u64 lim = kCountLimit - 1;
+  const u64 hi = __umul64hi(b, lim), lo = b * lim;
+  if (hi == 0 && a > lo) return kCountLimit;
+  u64 q = (u64)__double2ull_rz(__ddiv_rn(__ull2double_rn(a), __ull2double_rn(b)));
+  i64 r = (i64)(a - q * b);  // q b <= a + b: no wrap
+  if (r < 0) {
+    --q;
+    r += (i64)b;
+  } else if ((u64)r >= b) {
+    ++q;
+    r -= (i64)b;
+  }
+  return q + (r != 0 ? 1 : 0);
+}
 
 __device__ __forceinline__ u64 shard_bytes(u64 bytes, u32 method, const Recip& n) {
   return method == LLMEM_METHOD_CDP ? bytes : ceil_div(bytes, n);
@@ -175,13 +207,14 @@ __device__ __forceinline__ Plan make_plan(const Cfg& f, u32 method) {
   p.tpback = (method == LLMEM_METHOD_TP || method == LLMEM_METHOD_DPTP);
   p.tp = method == LLMEM_METHOD_TP ? f.gpu_n : f.tp_n;
   if (p.tp == 0) p.tp = 1;  // only reachable with status 2; keeps divisions defined
+  p.tp_recip = make_recip(p.tp).m;
   p.L = f.layers;
   p.iters = (int)f.iters;
   const u64 tok_p = V * H, pos_p = P * H, hh_p = H * H, hf_p = H * F;
   const u64 embed_p = tok_p + pos_p;                       // <= 2^47
   const u64 other_p = other_params(f);                     // < 2^61
   const u64 cs = (u64)f.chunk_elems;
-  const u64 chunks = ceil_div(other_p, cs);
+  const u64 chunks = chunk_count(other_p, cs);
   p.offset = (u64)f.base_bytes + tok_p * (u64)f.lm_bytes;  // < 2^60 + 2^49
   p.p16_embed = shard_bytes(2 * embed_p, method, rn);
   p.p32_embed = shard_bytes(4 * embed_p, method, rn);
@@ -228,8 +261,14 @@ __device__ __forceinline__ Dyn make_dyn(const Plan& p, u64 batch) {
   d.out = sat_mul(batch, p.out1);
   d.logit = sat_mul(batch, p.logit1);
   d.shift = sat_mul(batch, p.shift1);
-  // ceil(out * (tp-1) / tp) = out - floor(out / tp)   (m_back^tp, one layer's share)
-  d.back = p.tpback ? d.out - d.out / p.tp : 0;
+  // ceil(out * (tp-1) / tp) = out - floor(out / tp)   (m_back^tp, one layer's share); the
+  // reciprocal is exact below 2^56, and a saturated output makes the whole peak overflow
+  d.back = 0;
+  if (p.tpback) {
+    if (d.out >= kSat) d.back = kSat;
+    else if (d.out < (1ull << 56)) d.back = d.out - floor_div(d.out, Recip{p.tp_recip, p.tp});
+    else d.back = d.out - d.out / p.tp;
+  }
   d.attn = p.n_attn ? sat_mul(batch, p.attn1) : 0;
   d.ffn = p.n_ffn ? sat_mul(batch, p.ffn1) : 0;
   return d;
