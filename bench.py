@@ -516,6 +516,8 @@ def run_register_paths(args):
     sm = torch.cuda.get_device_properties(0).multi_processor_count
     mhz = clocks.get("sm_mhz") or 1965.0
     peak = sm * 4 * mhz * 1e6
+    # the same ceiling measured: independent 32-bit chains (add/xor, multiply-add, alternating)
+    probe = {name: llmem.int_rate(kind) for kind, name in enumerate(("add_xor", "mad", "add_mad"))}
     instr = None
     if all(NCU_WARP_INSTR_PER_UNIT.get(k) is not None for k in units):
         instr = sum(NCU_WARP_INSTR_PER_UNIT[k] * u for k, u in units.items())
@@ -528,6 +530,8 @@ def run_register_paths(args):
                      "achieved": (instr / (ms * 1e-3)) if instr else None,
                      "frac": (instr / (ms * 1e-3) / peak) if instr else None,
                      "peak_source": "148 SMs x 4 schedulers x sampled SM clock (one warp instruction per cycle each)",
+                     "measured_issue_rates": probe,
+                     "frac_of_measured_add_mad": (instr / (ms * 1e-3) / probe["add_mad"]) if instr else None,
                      "traffic": None},
         "gpu_launches": launches * args.steps, "clocks": clocks,
     }

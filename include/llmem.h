@@ -194,16 +194,20 @@ llmem_status llmem_scan_peak(const int64_t* DEV delta, const int64_t* DEV offset
 /* llmem_expand_events and llmem_scan_peak in one pass (Sections 4.1, 4.2 and 5): the list
  * is written exactly as llmem_expand_events writes it (raw sizes, or page-rounded with
  * LLMEM_FUSE_ROUND) and, while each piece of it is still in shared memory, folded into the
- * per-configuration peak of the page-rounded list.  Outputs are those of
- * llmem_scan_peak(..., cfg, ...) on the rounded list: m_base + lm_p + largest prefix sum,
- * first index attaining it, -1 / -1 for an inadmissible cfg[i].  The list is written to
- * device memory once and not read back.
+ * per-configuration peak of the page-rounded list (a piece that is one run of equal or of
+ * two alternating events is folded in closed form: its prefix sums are arithmetic
+ * progressions).  Outputs are those of llmem_scan_peak(..., cfg, ...) on the rounded list:
+ * m_base + lm_p + largest prefix sum, first index attaining it, -1 / -1 for an
+ * inadmissible cfg[i].  The list is written to device memory once and not read back.
  *   offsets        DEV [n+1]  as written by llmem_event_counts for the same cfg
  *   total_events   HOST value of offsets[n]
  *   delta_out      DEV [total_events]
  *   peak_out       DEV [n]
  *   peak_index_out DEV [n], nullable
- *   scratch        required, llmem_scratch_bytes(LLMEM_OP_EXPAND_SCAN, n, total_events) */
+ *   scratch        required, llmem_scratch_bytes(LLMEM_OP_EXPAND_SCAN, n, total_events) bytes,
+ *                  256-byte aligned; the call clears its header (status word, work counter)
+ *                  and rewrites what it reads, so the buffer may be reused by later calls in
+ *                  the same stream, but not by calls that may run at the same time */
 llmem_status llmem_expand_scan(const llmem_config* DEV cfg, int64_t n, const int64_t* DEV offsets,
                                int64_t total_events, int64_t* DEV delta_out, int64_t* DEV peak_out,
                                int64_t* DEV peak_index_out, void* DEV scratch, size_t scratch_bytes,
@@ -289,6 +293,18 @@ llmem_status llmem_scratch_status(const void* DEV scratch, void* cuda_stream);
  *   scratch  DEV, at least 256 bytes, 256-byte aligned */
 llmem_status llmem_selftest_wait_limit(void* DEV scratch, size_t scratch_bytes, uint32_t limit_ms,
                                        void* cuda_stream);
+
+/* No counterpart in the paper: a probe for the roofline of the kernels that generate events
+ * in registers.  Launches 8 CTAs of 256 threads per SM in which every thread advances eight
+ * independent 32-bit chains for `iters` iterations of 64 counted instructions: kind 0 add
+ * and xor (the integer ALU pipe), 1 multiply-add (the pipe 32-bit multiplies share with
+ * floating point), 2 the two alternating.  The caller times the launch with CUDA events;
+ * *warp_instructions_out receives the number of counted warp instructions it executes
+ * (loop counters and branches excluded), so rate = that / time.
+ *   sink                   DEV, nullable; 8 bytes that the kernel may add to (never in practice)
+ *   warp_instructions_out  HOST, nullable */
+llmem_status llmem_selftest_int_rate(int kind, uint32_t iters, uint64_t* DEV sink,
+                                     int64_t* warp_instructions_out, void* cuda_stream);
 
 /* Text of the last error on the calling thread ("" if none). */
 const char* llmem_last_error(void);

@@ -34,7 +34,7 @@ EXPORTS = (
     "llmem_round_events", "llmem_scan_peak", "llmem_max_batch", "llmem_select_method",
     "llmem_scratch_status", "llmem_last_error", "llmem_version", "llmem_event_counts_static",
     "llmem_select_segmented", "llmem_expand_scan", "llmem_chunk_search",
-    "llmem_selftest_wait_limit",
+    "llmem_selftest_wait_limit", "llmem_selftest_int_rate",
 )
 STATIC_MAX_CONFIGS = 4194304
 
@@ -79,6 +79,7 @@ def lib() -> ctypes.CDLL:
         L.llmem_expand_scan.argtypes = [vp, i64, vp, i64, vp, vp, vp, vp, sz, u32, vp]
         L.llmem_select_segmented.argtypes = [vp, vp, vp, i64, i64, i32, vp, vp, vp, vp, sz, u32, vp]
         L.llmem_selftest_wait_limit.argtypes = [vp, sz, u32, vp]
+        L.llmem_selftest_int_rate.argtypes = [ctypes.c_int, u32, vp, ctypes.POINTER(i64), vp]
         L.llmem_scratch_status.argtypes = [vp, vp]
         L.llmem_last_error.restype = ctypes.c_char_p
         L.llmem_version.restype = ctypes.c_int
@@ -348,3 +349,20 @@ def estimate_materialized(cfg, *, fuse_round: bool = True, stream=None):
     r = scan_peak(delta, offsets, cfg, stream=stream)
     return {"peak": r["peak"], "index": r["index"], "status": status, "offsets": offsets,
             "total_events": total}
+
+
+def int_rate(kind: int = 0, iters: int = 4096, reps: int = 3, stream=None) -> float:
+    """Warp instructions per second of the issue-rate probe (``llmem_selftest_int_rate``):
+    kind 0 add/xor, 1 multiply-add, 2 alternating.  Timed with CUDA events, best of ``reps``."""
+    torch = _torch()
+    count = ctypes.c_int64(0)
+    best = None
+    for _ in range(reps + 1):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        _check(lib().llmem_selftest_int_rate(kind, iters, None, ctypes.byref(count), _stream_ptr(stream)))
+        b.record(stream)
+        b.synchronize()
+        ms = a.elapsed_time(b)
+        best = ms if best is None or ms < best else best
+    return count.value / (best * 1e-3)

@@ -40,9 +40,62 @@ llmem_status check_launch(const char* what) {
   return LLMEM_OK;
 }
 
+// Issue-rate probe: every thread advances eight independent 32-bit chains, 64 counted
+// instructions per loop iteration (the loop's own counter and branch are not counted), so
+// that with 64 resident warps per SM the schedulers never lack an eligible warp.
+// kKind 0: add / xor (the integer ALU), 1: multiply-add, 2: the two alternating.
+template <int kKind>
+__global__ void __launch_bounds__(256)
+int_rate_kernel(unsigned int iters, unsigned int seed, unsigned long long* __restrict__ sink) {
+  unsigned int a[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) a[j] = seed * (unsigned int)(j + 1) + threadIdx.x;
+  const unsigned int c = seed | 1u, m = (seed >> 3) | 3u;
+  for (unsigned int i = 0; i < iters; ++i) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        if (kKind == 0) {
+          asm volatile("add.u32 %0, %0, %1;" : "+r"(a[j]) : "r"(c));
+          asm volatile("xor.b32 %0, %0, %1;" : "+r"(a[j]) : "r"(m));
+        } else if (kKind == 1) {
+          asm volatile("mad.lo.u32 %0, %0, %1, %2;" : "+r"(a[j]) : "r"(m), "r"(c));
+          asm volatile("mad.lo.u32 %0, %0, %1, %2;" : "+r"(a[j]) : "r"(c), "r"(m));
+        } else {
+          asm volatile("add.u32 %0, %0, %1;" : "+r"(a[j]) : "r"(c));
+          asm volatile("mad.lo.u32 %0, %0, %1, %2;" : "+r"(a[j]) : "r"(m), "r"(c));
+        }
+      }
+    }
+  }
+  unsigned int x = 0;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) x ^= a[j];
+  if (x == 0x9e3779b9u && sink) atomicAdd(sink, 1ull);  // keeps the chains alive
+}
+
 }  // namespace llmem
 
 using namespace llmem;
+
+extern "C" llmem_status llmem_selftest_int_rate(int kind, uint32_t iters, uint64_t* sink,
+                                                int64_t* warp_instructions_out, void* cuda_stream) {
+  clear_error();
+  if (kind < 0 || kind > 2 || iters < 1 || iters > (1u << 20)) {
+    set_error("llmem_selftest_int_rate: kind must be 0, 1 or 2 and iters in 1 .. 2^20");
+    return LLMEM_ERR_ARG;
+  }
+  const unsigned grid = (unsigned)sm_count() * 8u;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const unsigned seed = 0x2404u + iters;
+  unsigned long long* dsink = reinterpret_cast<unsigned long long*>(sink);
+  if (kind == 0) int_rate_kernel<0><<<grid, 256, 0, s>>>(iters, seed, dsink);
+  else if (kind == 1) int_rate_kernel<1><<<grid, 256, 0, s>>>(iters, seed, dsink);
+  else int_rate_kernel<2><<<grid, 256, 0, s>>>(iters, seed, dsink);
+  if (warp_instructions_out) *warp_instructions_out = (int64_t)grid * 8 * (int64_t)iters * 64;
+  return check_launch("llmem_selftest_int_rate");
+}
 
 extern "C" const char* llmem_last_error(void) { return g_error; }
 

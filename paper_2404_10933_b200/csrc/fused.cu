@@ -1,8 +1,8 @@
 // llmem_expand_scan: materialise the event list and take its segmented prefix-sum + max
 // in one pass.  Each warp builds a 576-event chunk in its own shared memory exactly as
-// the expansion kernel does, folds it from shared memory while it is still there, and
-// hands it to the TMA engine as one bulk store.  The list is written to HBM once
-// (8 bytes per event) and never read back: the scan costs no HBM traffic at all.
+// the expansion kernel does (or finds that the buffer already holds it), folds it while it
+// is there, and hands it to the TMA engine as one bulk store.  The list is written to HBM
+// once (8 bytes per event) and never read back: the scan costs no HBM traffic at all.
 #include "llmem_host.h"
 #include "expand.cuh"
 #include "fold.cuh"

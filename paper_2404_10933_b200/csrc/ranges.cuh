@@ -1,7 +1,8 @@
 // Work distribution of the kernels that stream over a materialised event list.
 //
-// The list is cut into chunks (one warp's unit of work); every warp of the persistent grid
-// owns one contiguous block of chunks, which is the access pattern HBM likes best.  Blocks of
+// The list is cut into chunks (one warp's unit of work) and the chunks into contiguous blocks,
+// one per warp (scan) or many per warp, claimed on request (expansion); a warp streams a
+// block from end to end, which is the access pattern HBM likes best.  Blocks of
 // equal length would be balanced if every event cost the same, but a segment boundary costs
 // about as much as a thousand events (descriptor, fold reduction, result), and lists of many
 // short segments sit next to each other.  So the blocks are balanced by a cost model instead:
