@@ -450,6 +450,22 @@ def test_bounded_wait_gives_up_and_reports(llmem):
     assert np.array_equal(pipe["peak"].cpu().numpy(), want["peak"])
 
 
+def test_issue_rate_probe(llmem):
+    import ctypes
+    L = llmem.lib()
+    count = ctypes.c_int64(0)
+    stream = llmem._stream_ptr(None)
+    assert L.llmem_selftest_int_rate(0, 16, None, ctypes.byref(count), stream) == llmem.OK
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    assert count.value == sms * 8 * 8 * 16 * 64          # CTAs x warps x iterations x counted instructions
+    assert L.llmem_selftest_int_rate(3, 16, None, None, stream) == llmem.ERR_ARG
+    assert L.llmem_selftest_int_rate(0, 0, None, None, stream) == llmem.ERR_ARG
+    rates = [llmem.int_rate(kind, iters=512, reps=1) for kind in range(3)]
+    torch.cuda.synchronize()
+    assert all(r > 1e11 for r in rates)
+    assert rates[1] < rates[0]                            # 32-bit multiplies issue more slowly than adds
+
+
 def test_all_operator_outputs_mode(llmem):
     """act_mode = 1 (no gradient checkpointing) on realistic shapes: estimate, materialised
     paths, searches and selection against the oracle; the mode must change the result."""
