@@ -12,6 +12,13 @@
 #ifndef LLMEM_EST_MIN_CTAS
 #define LLMEM_EST_MIN_CTAS 3
 #endif
+#ifndef LLMEM_EST_THREADS
+#define LLMEM_EST_THREADS 256
+#endif
+// CTAs per SM the estimate's grid is capped at (its threads stride over the configurations)
+#ifndef LLMEM_EST_GRID_CTAS
+#define LLMEM_EST_GRID_CTAS 8
+#endif
 #ifndef LLMEM_SEARCH_MIN_CTAS
 #define LLMEM_SEARCH_MIN_CTAS 4
 #endif
@@ -151,7 +158,7 @@ struct PageSearch {
 // ---------------------------------------------------------------------------
 // llmem_estimate_batch
 // ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(256, LLMEM_EST_MIN_CTAS)
+__global__ void __launch_bounds__(LLMEM_EST_THREADS, LLMEM_EST_MIN_CTAS)
 estimate_kernel(const llmem_config* __restrict__ cfg, i64 n, i64* __restrict__ peak_out,
                 i64* __restrict__ index_out, uint8_t* __restrict__ status_out) {
   for (i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (i64)gridDim.x * blockDim.x) {
@@ -394,7 +401,7 @@ extern "C" llmem_status llmem_estimate_batch(const llmem_config* cfg, int64_t n,
     set_error("llmem_estimate_batch: cfg must be 16-byte and outputs 8-byte aligned");
     return LLMEM_ERR_ARG;
   }
-  estimate_kernel<<<grid_for(n, 256, 8), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+  estimate_kernel<<<grid_for(n, LLMEM_EST_THREADS, LLMEM_EST_GRID_CTAS), LLMEM_EST_THREADS, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
       cfg, n, reinterpret_cast<i64*>(peak_out), reinterpret_cast<i64*>(peak_index_out), status_out);
   return check_launch("llmem_estimate_batch");
 }

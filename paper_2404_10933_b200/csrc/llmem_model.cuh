@@ -28,11 +28,18 @@ __host__ __device__ __forceinline__ u64 sat_add(u64 a, u64 b) {
   return s > kSat ? kSat : s;
 }
 
-__device__ __forceinline__ u64 sat_mul(u64 a, u64 b) {
-  u64 hi = __umul64hi(a, b);
-  u64 lo = a * b;
-  return (hi != 0 || lo >= kSat) ? kSat : lo;
+// Saturating a * b (b <= 2^62) for a 32-bit factor, which every product of the model has
+// (a count, a batch, a sequence length): two widening multiplies instead of a 64 x 64 product.
+__device__ __forceinline__ u64 sat_mul_u32(u32 a, u64 b) {
+  const u64 lo = (u64)a * (u32)b;          // a * (low half of b)
+  const u64 hi = (u64)a * (u32)(b >> 32);  // a * (high half of b), to be shifted by 32
+  const u64 t = lo + (hi << 32);
+  return (hi >= (1ull << 30) || t < lo || t >= kSat) ? kSat : t;
 }
+
+// zero-extension of a field that check_fields has shown to be non-negative: tells the
+// compiler that the upper half is zero, so products of two such values are one widening multiply
+__device__ __forceinline__ u64 zx(int v) { return (u64)(u32)v; }
 
 // ceil(x / cu_p) * cu_p; x <= 2^62 keeps the result <= 2^62
 __host__ __device__ __forceinline__ u64 page_round(u64 x) { return (x + (kPage - 1)) & ~(kPage - 1); }
@@ -188,18 +195,18 @@ __device__ __forceinline__ u64 gathered_bytes(u64 x, u32 method, const Recip& n,
 // decoder: per layer q, k, v, o (H x H) and 2 or 3 feed-forward matrices (H x F), their
 // biases, two norm vectors; one final norm.  `f` has passed check_fields.
 __device__ __forceinline__ u64 other_params(const Cfg& f) {
-  const u64 H = (u64)f.hidden, F = (u64)f.ffn, bias = f.has_bias;
+  const u64 H = zx(f.hidden), F = zx(f.ffn), bias = f.has_bias;
   const u64 nffn = f.ffn_kind ? 3 : 2;
   const u64 bias_p = bias * (4 * H + (nffn - 1) * F + H);
   const u64 norm_p = 2 * H * (1 + bias);
-  return (u64)f.layers * (4 * H * H + nffn * H * F + bias_p + norm_p) + H * (1 + bias);  // < 2^61
+  return zx(f.layers) * (4 * H * H + nffn * H * F + bias_p + norm_p) + H * (1 + bias);  // < 2^61
 }
 
 // a1: parameter inventory and event sizes.  `f` has passed check_fields.
 __device__ __forceinline__ Plan make_plan(const Cfg& f, u32 method) {
   Plan p;
   p.status = check_combo(method, f.gpu_n, f.tp_n);
-  const u64 H = (u64)f.hidden, F = (u64)f.ffn, V = (u64)f.vocab, P = (u64)f.pos_len;
+  const u64 H = zx(f.hidden), F = zx(f.ffn), V = zx(f.vocab), P = zx(f.pos_len);
   const Recip rn = make_recip(f.gpu_n);
   p.e_n = 1 + (f.pos_len > 0);
   p.K = f.ffn_kind ? 7 : 6;
@@ -226,17 +233,17 @@ __device__ __forceinline__ Plan make_plan(const Cfg& f, u32 method) {
   p.os_pos = shard_bytes(8 * pos_p, method, rn);
   p.os_hh = shard_bytes(8 * hh_p, method, rn);
   p.os_hf = shard_bytes(8 * hf_p, method, rn);
-  p.out1 = 2 * (u64)f.seq * H;                              // <= 2^47
-  p.logit1 = (u64)f.lm_bytes * (u64)f.seq * V;              // <= 2^54
-  p.shift1 = (u64)f.lm_bytes * (u64)(f.seq - 1) * V;
+  p.out1 = 2 * zx(f.seq) * H;                              // <= 2^47
+  p.logit1 = (u64)f.lm_bytes * zx(f.seq) * V;              // <= 2^54
+  p.shift1 = (u64)f.lm_bytes * zx(f.seq - 1) * V;
   // Without gradient checkpointing every operator of a pre-norm layer keeps its fp16 output:
   // norm, q, k, v, scores, softmax, context, o-proj, residual, norm, up (x2 + product when
   // gated), activation, down, residual: 10 hidden-sized, 2 score-sized, 2 or 4 ffn-sized.
   p.n_x = f.act_mode ? 10 : 1;
   p.n_attn = f.act_mode ? 2 : 0;
   p.n_ffn = f.act_mode ? (f.ffn_kind ? 4 : 2) : 0;
-  p.attn1 = sat_mul(sat_mul(2 * (u64)f.heads, (u64)f.seq), (u64)f.seq);
-  p.ffn1 = 2 * (u64)f.seq * F;                              // <= 2^49
+  p.attn1 = sat_mul_u32((u32)f.seq, sat_mul_u32((u32)f.seq, 2 * zx(f.heads)));
+  p.ffn1 = 2 * zx(f.seq) * F;                              // <= 2^49
   if (chunks >= kCountLimit) {
     p.C = 0;
     p.count = kCountLimit;
@@ -258,9 +265,10 @@ struct Dyn {
 
 __device__ __forceinline__ Dyn make_dyn(const Plan& p, u64 batch) {
   Dyn d;
-  d.out = sat_mul(batch, p.out1);
-  d.logit = sat_mul(batch, p.logit1);
-  d.shift = sat_mul(batch, p.shift1);
+  const u32 b32 = (u32)batch;  // batch <= 2^26
+  d.out = sat_mul_u32(b32, p.out1);
+  d.logit = sat_mul_u32(b32, p.logit1);
+  d.shift = sat_mul_u32(b32, p.shift1);
   // ceil(out * (tp-1) / tp) = out - floor(out / tp)   (m_back^tp, one layer's share); the
   // reciprocal is exact below 2^56, and a saturated output makes the whole peak overflow
   d.back = 0;
@@ -269,8 +277,8 @@ __device__ __forceinline__ Dyn make_dyn(const Plan& p, u64 batch) {
     else if (d.out < (1ull << 56)) d.back = d.out - floor_div(d.out, Recip{p.tp_recip, p.tp});
     else d.back = d.out - d.out / p.tp;
   }
-  d.attn = p.n_attn ? sat_mul(batch, p.attn1) : 0;
-  d.ffn = p.n_ffn ? sat_mul(batch, p.ffn1) : 0;
+  d.attn = p.n_attn ? sat_mul_u32(b32, p.attn1) : 0;
+  d.ffn = p.n_ffn ? sat_mul_u32(b32, p.ffn1) : 0;
   return d;
 }
 
@@ -282,22 +290,22 @@ struct StaticSums {
 __device__ __forceinline__ StaticSums make_static_sums(const Plan& p, bool has_pos) {
   StaticSums s;
   s.init = sat_add(sat_add(page_round(p.p16_embed), page_round(p.p32_embed)),
-                   sat_mul(p.C, page_round(p.p16_chunk) + page_round(p.p32_chunk)));
-  s.gather = p.gather ? sat_add(page_round(p.gat_embed), sat_mul(p.C, page_round(p.gat_chunk))) : 0;
+                   sat_mul_u32(p.C, page_round(p.p16_chunk) + page_round(p.p32_chunk)));
+  s.gather = p.gather ? sat_add(page_round(p.gat_embed), sat_mul_u32(p.C, page_round(p.gat_chunk))) : 0;
   const u64 per_layer = 4 * page_round(p.os_hh) + (u64)(p.K - 4) * page_round(p.os_hf);  // < 2^48
   s.os = sat_add(page_round(p.os_tok) + (has_pos ? page_round(p.os_pos) : 0),
-                 sat_mul((u64)p.L, per_layer));
+                 sat_mul_u32((u32)p.L, per_layer));
   return s;
 }
 
 // Sum of the rounded batch-dependent allocations of one iteration (phases 3 and 4).
 __device__ __forceinline__ u64 dyn_sum(const Plan& p, const Dyn& d) {
-  u64 s = sat_mul((u64)p.e_n + (u64)p.L * (u64)p.n_x, page_round(d.out));
-  if (p.n_attn) s = sat_add(s, sat_mul((u64)p.L * (u64)p.n_attn, page_round(d.attn)));
-  if (p.n_ffn) s = sat_add(s, sat_mul((u64)p.L * (u64)p.n_ffn, page_round(d.ffn)));
+  u64 s = sat_mul_u32((u32)(p.e_n + p.L * p.n_x), page_round(d.out));
+  if (p.n_attn) s = sat_add(s, sat_mul_u32((u32)(p.L * p.n_attn), page_round(d.attn)));
+  if (p.n_ffn) s = sat_add(s, sat_mul_u32((u32)(p.L * p.n_ffn), page_round(d.ffn)));
   s = sat_add(s, page_round(d.logit));
-  s = sat_add(s, sat_mul(2, page_round(d.shift)));
-  if (p.tpback) s = sat_add(s, sat_mul((u64)p.L, page_round(d.back)));
+  s = sat_add(s, sat_mul_u32(2u, page_round(d.shift)));
+  if (p.tpback) s = sat_add(s, sat_mul_u32((u32)p.L, page_round(d.back)));
   return s;
 }
 
