@@ -42,6 +42,39 @@ def test_g2_shape_grid_full(llmem):
     assert np.array_equal(got["index"].cpu().numpy()[idx], want1["index"])
 
 
+def test_g2_slice_materialized_claimed_blocks(llmem):
+    """A slice of the shape grid as materialised lists: clusters of short segments next to
+    long ones, long enough (several hundred million events) for the expansion kernels to cut
+    the list into more blocks than warps and hand them out on request."""
+    cfgs = grids.g2_shape_grid(8, 56)
+    dev = llmem.to_device(cfgs)
+    offsets, status = llmem.event_counts(dev)
+    total = int(offsets[-1].item())
+    assert total > 2 * 128 * 576 * 2368      # twice 128 chunks for each of the 2368 resident warps
+    want = oracle.estimate(cfgs, level=1, threads=THREADS)
+    assert np.array_equal(status.cpu().numpy(), want["status"])
+    off = offsets.cpu().numpy()
+    assert np.array_equal(np.diff(off), np.where(want["status"] == 0, want["count"], 0))
+    delta = torch.zeros(total, dtype=torch.int64, device="cuda")
+    one = llmem.expand_scan(dev, offsets, total, fuse_round=True, out=delta)
+    assert np.array_equal(one["peak"].cpu().numpy(), want["peak"])
+    assert np.array_equal(one["index"].cpu().numpy(), want["index"])
+    two_list = llmem.expand_events(dev, offsets, total, fuse_round=True)
+    assert torch.equal(two_list, delta)
+    two = llmem.scan_peak(two_list, offsets, dev, check_status=True)
+    assert np.array_equal(two["peak"].cpu().numpy(), want["peak"])
+    assert np.array_equal(two["index"].cpu().numpy(), want["index"])
+    # whole lists of sampled configurations, shortest and longest included
+    counts = np.diff(off)
+    picks = set(sample_indices(len(cfgs), 40, 9).tolist())
+    picks.update([int(np.argmax(counts)), int(np.argmin(np.where(counts > 0, counts, counts.max())))])
+    for i in sorted(picks):
+        if want["status"][i] != 0:
+            continue
+        ev = oracle.round_events(oracle.expand_events(cfgs[i:i + 1]))
+        assert np.array_equal(delta[off[i]:off[i + 1]].cpu().numpy(), ev), i
+
+
 def test_g3_large_sweep_full(llmem):
     cfgs = grids.g3_sweep()
     assert len(cfgs) == 1 << 20
