@@ -351,6 +351,38 @@ def estimate_materialized(cfg, *, fuse_round: bool = True, stream=None):
             "total_events": total}
 
 
+def estimate_in_slabs(cfg, max_events: int, *, first_config: int = 0, on_slab=None, stream=None):
+    """The materialised path for grids whose event lists do not fit in device memory at
+    once: the configurations are cut into contiguous slabs of at most ``max_events`` events
+    (``grids.slab_bounds``), and every slab is expanded, page-rounded and scanned by
+    ``llmem_expand_scan`` through one list buffer and one scratch buffer that are reused.
+    ``first_config`` restarts an interrupted run at a slab boundary (earlier results are then
+    left at -1).  ``on_slab(lo, hi, delta, offsets)`` is called after each slab with its
+    configuration range, its event list (valid until the next slab) and its local offsets.
+    Returns dict(peak[n], index[n], status[n], bounds): ``bounds`` are the slab boundaries."""
+    torch = _torch()
+    cfg = _as_cfg(cfg)
+    n = cfg.shape[0]
+    offsets, status = event_counts(cfg, stream=stream)
+    bounds = grids.slab_bounds(offsets.cpu().numpy(), max_events, first_config)
+    off_host = offsets.cpu().numpy()
+    sizes = off_host[bounds[1:]] - off_host[bounds[:-1]]
+    capacity = int(sizes.max()) if len(sizes) else 0
+    delta = torch.empty(max(capacity, 1), dtype=torch.int64, device=cfg.device)
+    scratch, _ = _scratch(OP_EXPAND_SCAN, n, capacity, cfg.device)
+    peak = torch.full((n,), -1, dtype=torch.int64, device=cfg.device)
+    index = torch.full((n,), -1, dtype=torch.int64, device=cfg.device)
+    for lo, hi, total in zip(bounds[:-1].tolist(), bounds[1:].tolist(), sizes.tolist()):
+        part = cfg[lo:hi]
+        local, _ = event_counts(part, want_status=False, stream=stream)
+        r = expand_scan(part, local, int(total), fuse_round=True, out=delta, scratch=scratch, stream=stream)
+        peak[lo:hi] = r["peak"]
+        index[lo:hi] = r["index"]
+        if on_slab is not None:
+            on_slab(lo, hi, r["delta"], local)
+    return {"peak": peak, "index": index, "status": status, "bounds": bounds}
+
+
 def int_rate(kind: int = 0, iters: int = 4096, reps: int = 3, stream=None) -> float:
     """Warp instructions per second of the issue-rate probe (``llmem_selftest_int_rate``):
     kind 0 add/xor, 1 multiply-add, 2 alternating.  Timed with CUDA events, best of ``reps``."""

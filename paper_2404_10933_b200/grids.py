@@ -319,3 +319,26 @@ def shard_bounds(weights: np.ndarray, world_size: int) -> np.ndarray:
     cuts = np.searchsorted(csum, targets, side="left")
     bounds = np.concatenate([[0], np.clip(cuts, 0, n), [n]]).astype(np.int64)
     return np.maximum.accumulate(bounds)
+
+
+def slab_bounds(offsets: np.ndarray, max_events: int, first: int = 0) -> np.ndarray:
+    """Cut configurations [first, n) into contiguous slabs whose event lists hold at most
+    ``max_events`` events each, greedily; a configuration with more events than that forms a
+    slab of its own.  ``offsets`` is the exclusive prefix sum of the event counts ([n+1]).
+    Returns the slab boundaries, starting with ``first`` and ending with n (just [first] if
+    first == n)."""
+    offsets = np.asarray(offsets, dtype=np.int64)
+    n = len(offsets) - 1
+    if max_events < 1:
+        raise ValueError("max_events must be positive")
+    if not 0 <= first <= n:
+        raise ValueError("first must lie in 0 .. n")
+    bounds = [first]
+    a = first
+    while a < n:
+        # largest b with offsets[b] - offsets[a] <= max_events, at least a + 1
+        b = int(np.searchsorted(offsets, offsets[a] + max_events, side="right")) - 1
+        b = min(max(b, a + 1), n)
+        bounds.append(b)
+        a = b
+    return np.asarray(bounds, dtype=np.int64)

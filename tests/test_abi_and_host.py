@@ -6,6 +6,7 @@ import os
 import re
 
 import numpy as np
+import pytest
 
 import paper_2404_10933_b200 as llmem
 from paper_2404_10933_b200 import grids
@@ -112,3 +113,27 @@ def test_shard_bounds_balance_weights():
     assert abs(left - w.sum() / 2) <= w.max()
     assert grids.shard_bounds(w, 1).tolist() == [0, 8]
     assert grids.shard_bounds(np.ones(3), 8)[-1] == 3
+
+
+def test_slab_bounds_cover_and_respect_the_budget():
+    from paper_2404_10933_b200 import grids
+    rng = np.random.default_rng(4)
+    counts = rng.integers(0, 5000, size=300)
+    counts[[17, 140]] = 60000                      # larger than the budget: slabs of their own
+    counts[50:60] = 0                              # inadmissible records have no events
+    off = np.concatenate([[0], np.cumsum(counts)]).astype(np.int64)
+    for budget in (1, 4999, 20000, 10 ** 9):
+        for first in (0, 23, 300):
+            b = grids.slab_bounds(off, budget, first)
+            assert b[0] == first and b[-1] == 300 and (np.diff(b) > 0).all()
+            assert len(b) > 1 or first == 300
+            for lo, hi in zip(b[:-1], b[1:]):
+                events = off[hi] - off[lo]
+                assert events <= budget or hi == lo + 1
+                # greedy: the next configuration would not have fitted
+                if hi < 300 and hi > lo + 1:
+                    assert off[hi + 1] - off[lo] > budget
+    with pytest.raises(ValueError):
+        grids.slab_bounds(off, 0)
+    with pytest.raises(ValueError):
+        grids.slab_bounds(off, 10, 301)

@@ -42,6 +42,27 @@ def test_g2_shape_grid_full(llmem):
     assert np.array_equal(got["index"].cpu().numpy()[idx], want1["index"])
 
 
+def test_g2_shape_grid_full_materialised_in_slabs(llmem):
+    """The whole shape grid as materialised lists (4.6e10 events, 365 GB as int64: eight times
+    the device memory one list buffer may take here), slab by slab through one 32 GiB buffer."""
+    cfgs = grids.g2_shape_grid()
+    free, _ = torch.cuda.mem_get_info()
+    budget = 1 << 32                                    # events per slab: 32 GiB of int64
+    if free < budget * 8 + (4 << 30):
+        pytest.skip("needs 36 GiB of free device memory")
+    r = llmem.estimate_in_slabs(cfgs, budget)
+    torch.cuda.synchronize()
+    assert len(r["bounds"]) > 8
+    want2 = oracle.estimate(cfgs, level=2, threads=THREADS)
+    assert np.array_equal(r["status"].cpu().numpy(), want2["status"])
+    peak = r["peak"].cpu().numpy()
+    assert np.array_equal(peak, want2["peak"])
+    idx = sample_indices(len(cfgs), 1500, 12)
+    want1 = oracle.estimate(cfgs[idx], level=1, threads=THREADS)
+    assert np.array_equal(peak[idx], want1["peak"])
+    assert np.array_equal(r["index"].cpu().numpy()[idx], want1["index"])
+
+
 def test_g2_slice_materialized_claimed_blocks(llmem):
     """A slice of the shape grid as materialised lists: clusters of short segments next to
     long ones, long enough (several hundred million events) for the expansion kernels to cut

@@ -450,6 +450,37 @@ def test_bounded_wait_gives_up_and_reports(llmem):
     assert np.array_equal(pipe["peak"].cpu().numpy(), want["peak"])
 
 
+def test_materialised_path_in_slabs(llmem):
+    """Slab by slab through one reused list buffer: same peaks as the oracle, every slab's
+    list bit for bit, restart from a slab boundary."""
+    cfgs = np.concatenate([mixed_small_grid(), grids.g5_stress(11, 3)])
+    want = oracle.estimate(cfgs, threads=8)
+    lists, off = oracle_lists(cfgs, rounded=True)
+    budget = 150_000                                   # the stress-grid lists are larger: slabs of their own
+    assert np.diff(off).max() > budget
+    seen = []
+
+    def on_slab(lo, hi, delta, local):
+        assert np.array_equal(delta.cpu().numpy(), lists[off[lo]:off[hi]])
+        assert np.array_equal(local.cpu().numpy(), off[lo:hi + 1] - off[lo])
+        seen.append((lo, hi))
+
+    r = llmem.estimate_in_slabs(cfgs, budget, on_slab=on_slab)
+    torch.cuda.synchronize()
+    b = r["bounds"]
+    assert len(b) > 10 and seen == list(zip(b[:-1].tolist(), b[1:].tolist()))
+    assert np.array_equal(b, grids.slab_bounds(off, budget))
+    assert np.array_equal(r["status"].cpu().numpy(), want["status"])
+    assert np.array_equal(r["peak"].cpu().numpy(), want["peak"])
+    assert np.array_equal(r["index"].cpu().numpy(), want["index"])
+    # restart at the fifth slab: earlier results stay at -1
+    again = llmem.estimate_in_slabs(cfgs, budget, first_config=int(b[4]))
+    k = int(b[4])
+    assert (again["peak"][:k] == -1).all()
+    assert np.array_equal(again["peak"].cpu().numpy()[k:], want["peak"][k:])
+    assert np.array_equal(again["index"].cpu().numpy()[k:], want["index"][k:])
+
+
 def test_issue_rate_probe(llmem):
     import ctypes
     L = llmem.lib()
