@@ -87,7 +87,10 @@ __device__ __forceinline__ u32 layer_code(bool gated, bool reversed, int* n_ops)
   return code;
 }
 
-__device__ inline void build_desc(SegDesc& d, const llmem_config* __restrict__ cfg, i64 gstart, i64 gend, bool round) {
+// Not inlined: the kernels reach it from two places, and the warps of an SM, each somewhere
+// else in a long kernel, already miss the instruction cache more than anything else
+// ("no instruction" is the top stall on lists of short segments).
+static __device__ __noinline__ void build_desc(SegDesc& d, const llmem_config* __restrict__ cfg, i64 gstart, i64 gend, bool round) {
   d.gstart = gstart;
   d.gend = gend;
   d.invalid = 1;
