@@ -82,6 +82,11 @@ def test_g2_slice_materialized_claimed_blocks(llmem):
     assert np.array_equal(one["index"].cpu().numpy(), want["index"])
     two_list = llmem.expand_events(dev, offsets, total, fuse_round=True)
     assert torch.equal(two_list, delta)
+    # without scratch the same blocks are handed out by the hardware block scheduler
+    two_list.fill_(0)
+    llmem.expand_events(dev, offsets, total, fuse_round=True, out=two_list,
+                        scratch=torch.empty(0, dtype=torch.uint8, device="cuda"))
+    assert torch.equal(two_list, delta)
     two = llmem.scan_peak(two_list, offsets, dev, check_status=True)
     assert np.array_equal(two["peak"].cpu().numpy(), want["peak"])
     assert np.array_equal(two["index"].cpu().numpy(), want["index"])
