@@ -139,8 +139,12 @@ def time_oracle(cfgs, threads: int):
 def cpu_baseline(sample_configs: int = 49152):
     cores = os.cpu_count() or 1
     events, dt = time_oracle(oracle_sample(sample_configs), cores)
+    one_n = max(1, sample_configs // 32)
+    one_events, one_dt = time_oracle(oracle_sample(one_n), 1)
     return {"value": events / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
             "configs_per_sec": sample_configs / dt,
+            "single_thread": {"value": one_events / one_dt, "unit": UNIT, "cores": 1,
+                              "sample": f"first {one_n} configurations, {one_dt:.2f} s"},
             "sample": f"first {sample_configs} of the 65536 stress-grid configurations "
                       f"({events} events), level-1 oracle (explicit list, round, scan) + its bisecting search and selection, "
                       f"{cores} threads, {dt:.2f} s"}
