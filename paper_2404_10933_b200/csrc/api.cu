@@ -82,6 +82,7 @@ using namespace llmem;
 extern "C" llmem_status llmem_selftest_int_rate(int kind, uint32_t iters, uint64_t* sink,
                                                 int64_t* warp_instructions_out, void* cuda_stream) {
   clear_error();
+  TraceRange trace("llmem_selftest_int_rate");
   if (kind < 0 || kind > 2 || iters < 1 || iters > (1u << 20)) {
     set_error("llmem_selftest_int_rate: kind must be 0, 1 or 2 and iters in 1 .. 2^20");
     return LLMEM_ERR_ARG;
@@ -122,6 +123,7 @@ extern "C" size_t llmem_scratch_bytes(int op, int64_t n, int64_t total_events) {
 
 extern "C" llmem_status llmem_scratch_status(const void* scratch, void* cuda_stream) {
   clear_error();
+  TraceRange trace("llmem_scratch_status");
   if (!scratch) {
     set_error("llmem_scratch_status: scratch is null");
     return LLMEM_ERR_ARG;

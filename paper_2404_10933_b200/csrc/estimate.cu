@@ -394,6 +394,7 @@ extern "C" llmem_status llmem_estimate_batch(const llmem_config* cfg, int64_t n,
                                              void* cuda_stream) {
   (void)scratch; (void)scratch_bytes; (void)flags;
   clear_error();
+  TraceRange trace("llmem_estimate_batch");
   if (n < 0) { set_error("llmem_estimate_batch: n < 0"); return LLMEM_ERR_ARG; }
   if (n == 0) return LLMEM_OK;
   if (!cfg || !peak_out) { set_error("llmem_estimate_batch: cfg and peak_out are required"); return LLMEM_ERR_ARG; }
@@ -422,6 +423,7 @@ extern "C" llmem_status llmem_max_batch(const llmem_config* shape, int64_t n,
                                         size_t scratch_bytes, uint32_t flags, void* cuda_stream) {
   (void)scratch; (void)scratch_bytes; (void)flags;
   clear_error();
+  TraceRange trace("llmem_max_batch");
   llmem_status st = check_search_args("llmem_max_batch", shape, n, capacity_bytes, n_cap, bmax);
   if (st != LLMEM_OK || n == 0 || n_cap == 0) return st;
   if (!bs_out || !aligned_to(bs_out, 4)) { set_error("llmem_max_batch: bs_out is required"); return LLMEM_ERR_ARG; }
@@ -437,6 +439,7 @@ extern "C" llmem_status llmem_select_method(const llmem_config* shape, int64_t n
                                             size_t scratch_bytes, uint32_t flags, void* cuda_stream) {
   (void)scratch; (void)scratch_bytes;
   clear_error();
+  TraceRange trace("llmem_select_method");
   llmem_status st = check_search_args("llmem_select_method", shape, n, capacity_bytes, n_cap, bmax);
   if (st != LLMEM_OK || n == 0 || n_cap == 0) return st;
   if (!method_out || !batch_out) { set_error("llmem_select_method: method_out and batch_out are required"); return LLMEM_ERR_ARG; }
@@ -453,6 +456,7 @@ extern "C" llmem_status llmem_select_segmented(const llmem_config* item_cfg, con
                                                size_t scratch_bytes, uint32_t flags, void* cuda_stream) {
   (void)scratch; (void)scratch_bytes; (void)flags;
   clear_error();
+  TraceRange trace("llmem_select_segmented");
   if (n_groups < 0 || n_items < 0 || n_cap < 0) { set_error("llmem_select_segmented: negative size"); return LLMEM_ERR_ARG; }
   if (n_groups == 0 || n_cap == 0) return LLMEM_OK;
   if (!group_offsets || !item_out || (n_items > 0 && (!item_cfg || !bs))) {
@@ -475,6 +479,7 @@ extern "C" llmem_status llmem_chunk_search(const llmem_config* cfg, int64_t n, i
                                            uint32_t flags, void* cuda_stream) {
   (void)scratch; (void)scratch_bytes; (void)flags;
   clear_error();
+  TraceRange trace("llmem_chunk_search");
   if (n < 0) { set_error("llmem_chunk_search: n < 0"); return LLMEM_ERR_ARG; }
   if (cs_min < 1 || cs_step < 1 || n_candidates < 1 ||
       cs_min > (1ll << 40) || cs_step > (1ll << 40) ||

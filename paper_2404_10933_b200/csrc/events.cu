@@ -310,6 +310,7 @@ extern "C" llmem_status llmem_event_counts(const llmem_config* cfg, int64_t n, i
                                            uint32_t flags, void* cuda_stream) {
   (void)flags;
   clear_error();
+  TraceRange trace("llmem_event_counts");
   if (n < 0) { set_error("llmem_event_counts: n < 0"); return LLMEM_ERR_ARG; }
   if (!offsets_out || !aligned_to(offsets_out, 8)) { set_error("llmem_event_counts: offsets_out is required"); return LLMEM_ERR_ARG; }
   if (n > 0 && (!cfg || !aligned_to(cfg, 16))) { set_error("llmem_event_counts: cfg must be a 16-byte aligned device pointer"); return LLMEM_ERR_ARG; }
@@ -413,6 +414,7 @@ extern "C" llmem_status llmem_expand_events(const llmem_config* cfg, int64_t n, 
                                             int64_t total_events, int64_t* delta_out, void* scratch,
                                             size_t scratch_bytes, uint32_t flags, void* cuda_stream) {
   clear_error();
+  TraceRange trace("llmem_expand_events");
   if (n < 0 || total_events < 0) { set_error("llmem_expand_events: negative size"); return LLMEM_ERR_ARG; }
   if (total_events == 0) return LLMEM_OK;
   if (!cfg || !offsets || !delta_out) { set_error("llmem_expand_events: cfg, offsets and delta_out are required"); return LLMEM_ERR_ARG; }
@@ -451,6 +453,7 @@ extern "C" llmem_status llmem_round_events(int64_t* delta, int64_t total_events,
                                            size_t scratch_bytes, uint32_t flags, void* cuda_stream) {
   (void)scratch; (void)scratch_bytes; (void)flags;
   clear_error();
+  TraceRange trace("llmem_round_events");
   if (total_events < 0) { set_error("llmem_round_events: negative size"); return LLMEM_ERR_ARG; }
   if (total_events == 0) return LLMEM_OK;
   if (!delta || !aligned_to(delta, 8)) { set_error("llmem_round_events: delta must be an 8-byte aligned device pointer"); return LLMEM_ERR_ARG; }

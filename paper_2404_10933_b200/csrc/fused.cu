@@ -260,6 +260,7 @@ extern "C" llmem_status llmem_expand_scan(const llmem_config* cfg, int64_t n, co
                                           int64_t* peak_index_out, void* scratch, size_t scratch_bytes,
                                           uint32_t flags, void* cuda_stream) {
   clear_error();
+  TraceRange trace("llmem_expand_scan");
   if (n < 0 || total_events < 0) { set_error("llmem_expand_scan: negative size"); return LLMEM_ERR_ARG; }
   if (n == 0) return LLMEM_OK;
   if (!cfg || !offsets || !peak_out || (total_events > 0 && !delta_out)) {

@@ -6,6 +6,7 @@
 #include <cstddef>
 #include <cstdint>
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include "../../include/llmem.h"
 
@@ -16,6 +17,16 @@ void set_error(const char* fmt, ...);
 void clear_error();
 
 inline bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// An NVTX range around an entry point's host side (argument checks and launches), so that a
+// timeline shows which library call queued which kernels.  Costs a function call through a
+// null pointer check when no tool is attached.
+struct TraceRange {
+  explicit TraceRange(const char* name) { nvtxRangePushA(name); }
+  ~TraceRange() { nvtxRangePop(); }
+  TraceRange(const TraceRange&) = delete;
+  TraceRange& operator=(const TraceRange&) = delete;
+};
 
 // Number of SMs of the current device (cached per thread; 148 on B200).
 int sm_count();

@@ -334,6 +334,7 @@ extern "C" llmem_status llmem_scan_peak(const int64_t* delta, const int64_t* off
                                         int64_t* peak_out, int64_t* peak_index_out, void* scratch,
                                         size_t scratch_bytes, uint32_t flags, void* cuda_stream) {
   clear_error();
+  TraceRange trace("llmem_scan_peak");
   if (n < 0 || total_events < 0) { set_error("llmem_scan_peak: negative size"); return LLMEM_ERR_ARG; }
   if (n == 0) return LLMEM_OK;
   if (!offsets || !peak_out || (total_events > 0 && !delta)) {
@@ -394,6 +395,7 @@ extern "C" llmem_status llmem_scan_peak(const int64_t* delta, const int64_t* off
 extern "C" llmem_status llmem_selftest_wait_limit(void* scratch, size_t scratch_bytes, uint32_t limit_ms,
                                                   void* cuda_stream) {
   clear_error();
+  TraceRange trace("llmem_selftest_wait_limit");
   if (!scratch || !aligned_to(scratch, 256) || scratch_bytes < kScratchHeader) {
     set_error("llmem_selftest_wait_limit: scratch of at least 256 bytes, 256-byte aligned, is required");
     return LLMEM_ERR_SCRATCH;
