@@ -84,6 +84,11 @@ class ClockSampler:
             return
         self.thread = threading.Thread(target=self._read, daemon=True)
         self.thread.start()
+        # nvidia-smi's start-up (driver enumeration) can hold up work submission for tens of
+        # milliseconds: let it finish, i.e. wait for the first sample, before anything is timed
+        deadline = time.time() + 10.0
+        while not self.rows and time.time() < deadline and self.proc.poll() is None:
+            time.sleep(0.05)
 
     def _read(self):
         for line in self.proc.stdout:
@@ -379,7 +384,7 @@ def run_ours(args):
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    e2e_steps = max(1, min(args.steps, 10))
+    e2e_steps = max(1, min(args.steps, 100))
     for _ in range(e2e_steps):
         hp.step_e2e()
     e1.record()
@@ -604,7 +609,8 @@ def run_slab_path(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=1000,
+                    help="timed steps (default 1000, about 6 s: long enough that a stray 0.1 s stall of the box does not move the result)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
     ap.add_argument("--configs", type=int, default=grids.G5_CONFIGS,

@@ -248,6 +248,95 @@ struct ExpandWarpSmem {
   SegDesc desc;
 };
 
+// ---- chunks that repeat -------------------------------------------------------------------
+// A full chunk inside one run of equal events, or of two alternating ones, repeats the chunk
+// issued from the same buffer two chunks earlier.  AlternatingRun remembers the run the last
+// such chunk lay in; BufferKeys what pattern each of the warp's two chunk buffers holds.
+struct AlternatingRun {
+  i64 end = -1;  // chunks that end at or before this list index repeat the pattern
+  i64 key = -1;  // (segment, run, phase): identifies the pattern
+  i64 x0 = 0, x1 = 0;  // the value on even / odd positions of a chunk
+};
+
+struct BufferKeys {
+  i64 key0 = -1, key1 = -1;
+  __device__ __forceinline__ i64 get(int parity) const { return parity ? key1 : key0; }
+  __device__ __forceinline__ void set(int parity, i64 k) {
+    if (parity) key1 = k;
+    else key0 = k;
+  }
+};
+
+// Makes sure the warp's descriptor is that of segment `seg` (range [gs, ge)).
+__device__ __forceinline__ void ensure_desc(ExpandWarpSmem& ws, i64& desc_seg, const llmem_config* __restrict__ cfg,
+                                            i64 seg, i64 gs, i64 ge, bool round, int lane) {
+  if (desc_seg != seg) {
+    __syncwarp();  // every lane is done with the previous descriptor
+    if (lane == 0) build_desc(ws.desc, cfg + seg, gs, ge, round);
+    __syncwarp();
+    desc_seg = seg;
+  }
+}
+
+// Does the full chunk [tb, tb + kExpChunk), which lies inside segment `seg`, consist of one
+// run of period 1 or 2?  Updates `ar` when it enters a new such run.
+__device__ __forceinline__ bool chunk_alternates(AlternatingRun& ar, ExpandWarpSmem& ws, i64& desc_seg,
+                                                 const llmem_config* __restrict__ cfg, i64 seg, i64 gs, i64 ge,
+                                                 i64 tb, bool round, int lane) {
+  if (tb + kExpChunk <= ar.end) return true;
+  ensure_desc(ws, desc_seg, cfg, seg, gs, ge, round, lane);
+  if (ws.desc.invalid) return false;
+  int r, o, it;
+  locate(ws.desc, (u32)(tb - gs), &r, &o, &it);
+  const Run& rn = ws.desc.run[r];
+  if (rn.cnt - o < kExpChunk || rn.period > 2) return false;
+  // period 1: a everywhere; period 2: a on even offsets of the run, b on odd ones
+  const bool odd = rn.period == 2 && (o & 1);
+  ar.x0 = odd ? rn.b : rn.a;
+  ar.x1 = rn.period == 2 ? (odd ? rn.a : rn.b) : rn.a;
+  ar.end = tb + (rn.cnt - o);
+  ar.key = (seg << 8) | (i64)(r << 1) | (odd ? 1 : 0);
+  return true;
+}
+
+// Gets buffer `parity` ready for an alternating chunk: nothing to do if it already holds the
+// pattern (only the number of stores in flight is bounded); otherwise the bulk store issued
+// from it two chunks ago must have read it, then every lane writes its span (an even offset:
+// x0 comes first).
+template <int kStoresInFlight>
+__device__ __forceinline__ void prepare_alternating(const AlternatingRun& ar, BufferKeys& keys, int parity,
+                                                    i64* __restrict__ buf, int lane) {
+  if (keys.get(parity) != ar.key) {
+    if (lane == 0) bulk_wait_read<1>();
+    __syncwarp();
+    longlong2* v = reinterpret_cast<longlong2*>(buf + lane * kExpPerLane);
+#pragma unroll
+    for (int j = 0; j < kExpPerLane / 2; ++j) v[j] = make_longlong2(ar.x0, ar.x1);
+    keys.set(parity, ar.key);
+    fence_async_shared();
+    __syncwarp();
+  } else if (lane == 0) {
+    bulk_wait_read<kStoresInFlight>();
+  }
+}
+
+// Hands chunk [tb, tb + cnt) to the TMA engine (or copies it with plain stores when the
+// output is not 16-byte aligned).
+__device__ __forceinline__ void store_chunk(i64* __restrict__ out, i64 tb, u32 cnt, const i64* __restrict__ buf,
+                                            int bulk_ok, int lane) {
+  if (bulk_ok) {
+    if (lane == 0) {
+      const u32 even = cnt & ~1u;
+      if (even) bulk_store(out + tb, buf, even * 8u);
+      bulk_commit();
+      if (cnt & 1u) out[tb + cnt - 1] = buf[cnt - 1];
+    }
+  } else {
+    for (u32 i = lane; i < cnt; i += 32) out[tb + i] = buf[i];
+    __syncwarp();  // the buffer may be rewritten two chunks from now
+  }
+}
+
 // Write `cnt` events starting at segment position `pos` to dst[0 .. cnt).  Spans that
 // stay inside one run of period 1 or 2 (parameter chunks, gathers, outputs: almost
 // all of a long list) are written as constants; anything else goes through the

@@ -93,7 +93,7 @@ expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __res
   const i64 resident = (i64)gridDim.x * kFusedWarps;
   i64 desc_seg = -1;
   int parity = 0;
-  i64 key0 = -1, key1 = -1;  // what the two chunk buffers hold: key of an alternating pattern, or -1
+  BufferKeys keys;  // what the two chunk buffers hold
   for (i64 gw = (i64)blockIdx.x * kFusedWarps + warp; gw < n_blocks;) {
     i64 seg;  // smallest segment whose end lies beyond the current position; gs/ge its range
     const i64 b_lo = warp_block_start(offsets, n, 0, total, gw, n_blocks, kappa, kExpChunk, lane, &seg);
@@ -110,58 +110,18 @@ expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __res
     i64 gs = seg < n ? __ldg(offsets + seg) : total;
     i64 ge = seg < n ? __ldg(offsets + seg + 1) : total;
     SegmentFolder folder;
-    // the alternating run the last such chunk lay in: chunks that end at or before run_end
-    // repeat its pattern (x0 on even positions, x1 on odd ones)
-    i64 run_end = -1, run_key = -1, x0 = 0, x1 = 0;
+    AlternatingRun ar;  // the alternating run the last such chunk lay in
 
     for (i64 c = c_lo; c < c_hi; ++c, parity ^= 1) {
       const i64 tb = c * kExpChunk;
       const i64 te = tb + kExpChunk < total ? tb + kExpChunk : total;
       i64* buf = ws.buf[parity];
-      bool alternating = false;
-      if (seg < n && gs <= tb && tb + kExpChunk <= ge) {  // a full chunk inside one segment
-        if (tb + kExpChunk <= run_end) {
-          alternating = true;
-        } else {
-          if (desc_seg != seg) {
-            __syncwarp();  // every lane is done with the previous descriptor
-            if (lane == 0) build_desc(ws.desc, cfg + seg, gs, ge, kRoundList);
-            __syncwarp();
-            desc_seg = seg;
-          }
-          if (!ws.desc.invalid) {
-            int r, o, it;
-            locate(ws.desc, (u32)(tb - gs), &r, &o, &it);
-            const Run& rn = ws.desc.run[r];
-            if (rn.cnt - o >= kExpChunk && rn.period <= 2) {
-              // period 1: a everywhere; period 2: a on even offsets of the run, b on odd ones
-              const bool odd = rn.period == 2 && (o & 1);
-              x0 = odd ? rn.b : rn.a;
-              x1 = rn.period == 2 ? (odd ? rn.a : rn.b) : rn.a;
-              run_end = tb + (rn.cnt - o);
-              run_key = (seg << 8) | (i64)(r << 1) | (odd ? 1 : 0);
-              alternating = true;
-            }
-          }
-        }
-      }
+      // a full chunk inside one segment may repeat the one before
+      const bool alternating = seg < n && gs <= tb && tb + kExpChunk <= ge &&
+                               chunk_alternates(ar, ws, desc_seg, cfg, seg, gs, ge, tb, kRoundList, lane);
       if (alternating) {
-        const i64 key = parity ? key1 : key0;
-        if (key != run_key) {
-          // the buffer holds something else: the bulk store issued from it two chunks ago must
-          // have read it, then every lane writes its span (an even offset: x0 comes first)
-          if (lane == 0) bulk_wait_read<1>();
-          __syncwarp();
-          longlong2* v = reinterpret_cast<longlong2*>(buf + lane * kExpPerLane);
-#pragma unroll
-          for (int j = 0; j < kExpPerLane / 2; ++j) v[j] = make_longlong2(x0, x1);
-          if (parity) key1 = run_key; else key0 = run_key;
-          fence_async_shared();
-          __syncwarp();
-        } else if (lane == 0) {
-          bulk_wait_read<kFusedStoresInFlight>();
-        }
-        folder.add_uniform(fold_alternating_chunk(ev<!kRoundList>(x0), ev<!kRoundList>(x1), tb), lane);
+        prepare_alternating<kFusedStoresInFlight>(ar, keys, parity, buf, lane);
+        folder.add_uniform(fold_alternating_chunk(ev<!kRoundList>(ar.x0), ev<!kRoundList>(ar.x1), tb), lane);
         if (ge == te) {
           // the segment ends with this chunk: finish it and move to the next non-empty one
           folder.finish_segment(seg, gs, range_lo, my_partials, peak_out, index_out, lane);
@@ -172,7 +132,7 @@ expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __res
           } while (seg < n && ge <= te);
         }
       } else {
-        if (parity) key1 = -1; else key0 = -1;
+        keys.set(parity, -1);
         // the bulk store issued from this buffer two chunks ago must have read it
         if (lane == 0) bulk_wait_read<1>();
         __syncwarp();
@@ -185,12 +145,7 @@ expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __res
             for (i64 e = (span_lo > pos ? span_lo : pos); e < span_hi; ++e) buf[e - tb] = 0;
             break;
           }
-          if (desc_seg != seg) {
-            __syncwarp();  // every lane is done with the previous descriptor
-            if (lane == 0) build_desc(ws.desc, cfg + seg, gs, ge, kRoundList);
-            __syncwarp();
-            desc_seg = seg;
-          }
+          ensure_desc(ws, desc_seg, cfg, seg, gs, ge, kRoundList, lane);
           const i64 piece_end = ge < te ? ge : te;
           const i64 e = span_lo > pos ? span_lo : pos;
           const i64 e_end = span_hi < piece_end ? span_hi : piece_end;
@@ -226,19 +181,7 @@ expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __res
         if (bulk_ok) fence_async_shared();
         __syncwarp();
       }
-      // hand the chunk to the TMA engine
-      const u32 cnt = (u32)(te - tb);
-      if (bulk_ok) {
-        if (lane == 0) {
-          const u32 even = cnt & ~1u;
-          if (even) bulk_store(out + tb, buf, even * 8u);
-          bulk_commit();
-          if (cnt & 1u) out[tb + cnt - 1] = buf[cnt - 1];
-        }
-      } else {
-        for (u32 i = lane; i < cnt; i += 32) out[tb + i] = buf[i];
-        __syncwarp();  // the buffer may be rewritten two chunks from now
-      }
+      store_chunk(out, tb, (u32)(te - tb), buf, bulk_ok, lane);
     }
     // the current segment may continue into the next block
     folder.finish_range(gs, range_lo, my_partials, lane);
