@@ -160,7 +160,8 @@ def run_reference(args):
     if rank != 0:
         return 0
     cores = os.cpu_count() or 1
-    sample = 4096
+    # each step a bounded sample of the workload, sized so that the whole run stays near 10-20 s
+    sample = int(min(4096, max(256, 4096 * 100 // max(args.steps, 1))))
     cfgs = oracle_sample(sample)
     for _ in range(max(args.warmup, 0)):
         time_oracle(cfgs[:256], cores)
