@@ -262,19 +262,34 @@ class HotPath:
     def step_e2e(self):
         """Host buffers in, host results out: H2D of the configurations and capacities, the
         device-to-host read of the event total that sizes the list, every kernel, and the
-        D2H of peaks and selections."""
-        torch = self.torch
+        D2H of peaks and selections.  The searches and the copy of their results need only the
+        configurations, so they are queued on a second stream and run underneath the
+        expansion; both streams are joined before the step ends."""
+        torch, llmem = self.torch, self.llmem
+        main = torch.cuda.current_stream()
         cfg = self.host_cfg.to("cuda", non_blocking=True)
         caps = self.host_caps.to("cuda", non_blocking=True)
-        offsets, _ = self.llmem.event_counts(cfg)
+        self.fork.record(main)
+        self.side.wait_event(self.fork)
+        with torch.cuda.stream(self.side):
+            llmem.max_batch(cfg, caps, self.bmax, want_status=False)
+            sel = llmem.select_method(cfg, caps, self.bmax, want_bs_list=False, want_status=False)
+            self.host_out["method"].copy_(sel["method"], non_blocking=True)
+            self.host_out["batch"].copy_(sel["batch"], non_blocking=True)
+        offsets, _ = llmem.event_counts(cfg)
         total = int(offsets[-1].item())                      # 8-byte D2H + sync
         if total > self.delta.numel():
             self.delta = torch.empty(total, dtype=torch.int64, device="cuda")
-        r, _, sel = self._materialise_and_search(cfg, caps, offsets, total, False)
+        if self.one_pass:
+            r = llmem.expand_scan(cfg, offsets, total, fuse_round=True, out=self.delta, scratch=self.scan_scratch)
+        else:
+            delta = llmem.expand_events(cfg, offsets, total, fuse_round=True, out=self.delta)
+            r = llmem.scan_peak(delta, offsets, cfg, scratch=self.scan_scratch)
         self.host_out["peak"].copy_(r["peak"], non_blocking=True)
-        self.host_out["method"].copy_(sel["method"], non_blocking=True)
-        self.host_out["batch"].copy_(sel["batch"], non_blocking=True)
-        torch.cuda.current_stream().synchronize()
+        main.wait_stream(self.side)
+        for t in (cfg, caps, sel["method"], sel["batch"]):
+            t.record_stream(self.side)
+        main.synchronize()
         return total
 
     def time_kernel(self, what, reps=5):
