@@ -208,7 +208,8 @@ class HotPath:
         offsets, _ = llmem.event_counts(self.cfg)
         self.total = int(offsets[-1].item())
         self.delta = torch.empty(self.total, dtype=torch.int64, device="cuda")
-        self.scan_scratch = torch.empty(llmem.scratch_bytes(llmem.OP_SCAN_PEAK, self.n, self.total),
+        self.scan_scratch = torch.empty(max(llmem.scratch_bytes(llmem.OP_SCAN_PEAK, self.n, self.total),
+                                            llmem.scratch_bytes(llmem.OP_EXPAND_SCAN, self.n, self.total)),
                                         dtype=torch.uint8, device="cuda")
         self.ev = {k: [] for k in (("expand_scan",) if one_pass else ("expand", "scan"))}
         self.side = torch.cuda.Stream()

@@ -369,7 +369,9 @@ def estimate_in_slabs(cfg, max_events: int, *, first_config: int = 0, on_slab=No
     sizes = off_host[bounds[1:]] - off_host[bounds[:-1]]
     capacity = int(sizes.max()) if len(sizes) else 0
     delta = torch.empty(max(capacity, 1), dtype=torch.int64, device=cfg.device)
-    scratch, _ = _scratch(OP_EXPAND_SCAN, n, capacity, cfg.device)
+    nbytes = max([scratch_bytes(OP_EXPAND_SCAN, int(hi - lo), int(t))
+                  for lo, hi, t in zip(bounds[:-1], bounds[1:], sizes)] + [scratch_bytes(OP_EXPAND_SCAN, 0, 0)])
+    scratch = torch.empty(nbytes, dtype=torch.uint8, device=cfg.device)
     peak = torch.full((n,), -1, dtype=torch.int64, device=cfg.device)
     index = torch.full((n,), -1, dtype=torch.int64, device=cfg.device)
     for lo, hi, total in zip(bounds[:-1].tolist(), bounds[1:].tolist(), sizes.tolist()):

@@ -103,7 +103,6 @@ extern "C" const char* llmem_last_error(void) { return g_error; }
 extern "C" int llmem_version(void) { return 100; }
 
 extern "C" size_t llmem_scratch_bytes(int op, int64_t n, int64_t total_events) {
-  (void)total_events;
   if (n < 0) n = 0;
   switch (op) {
     case LLMEM_OP_EVENT_COUNTS:
@@ -113,9 +112,11 @@ extern "C" size_t llmem_scratch_bytes(int op, int64_t n, int64_t total_events) {
       // header only: the work counter
       return kScratchHeader;
     case LLMEM_OP_SCAN_PEAK:
-    case LLMEM_OP_EXPAND_SCAN:
       // header, block starts and a head and a tail partial per block of the list
       return kStreamScratchBytes;
+    case LLMEM_OP_EXPAND_SCAN:
+      // the same, plus a descriptor per configuration when the segments are short
+      return expand_scan_scratch_bytes(n, total_events);
     default:
       return 0;
   }

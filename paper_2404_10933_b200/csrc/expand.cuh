@@ -267,12 +267,22 @@ struct BufferKeys {
   }
 };
 
-// Makes sure the warp's descriptor is that of segment `seg` (range [gs, ge)).
+// Makes sure the warp's descriptor is that of segment `seg` (range [gs, ge)): copied by the
+// whole warp from `table` (one descriptor per configuration, built beforehand by one thread
+// each) when there is one, else built here by lane 0.
+static_assert(sizeof(SegDesc) % 16 == 0, "descriptors are copied in 16-byte words");
 __device__ __forceinline__ void ensure_desc(ExpandWarpSmem& ws, i64& desc_seg, const llmem_config* __restrict__ cfg,
-                                            i64 seg, i64 gs, i64 ge, bool round, int lane) {
+                                            const SegDesc* __restrict__ table, i64 seg, i64 gs, i64 ge, bool round,
+                                            int lane) {
   if (desc_seg != seg) {
     __syncwarp();  // every lane is done with the previous descriptor
-    if (lane == 0) build_desc(ws.desc, cfg + seg, gs, ge, round);
+    if (table) {
+      const int4* src = reinterpret_cast<const int4*>(table + seg);
+      int4* dst = reinterpret_cast<int4*>(&ws.desc);
+      for (int k = lane; k < (int)(sizeof(SegDesc) / 16); k += 32) dst[k] = __ldg(src + k);
+    } else if (lane == 0) {
+      build_desc(ws.desc, cfg + seg, gs, ge, round);
+    }
     __syncwarp();
     desc_seg = seg;
   }
@@ -281,10 +291,11 @@ __device__ __forceinline__ void ensure_desc(ExpandWarpSmem& ws, i64& desc_seg, c
 // Does the full chunk [tb, tb + kExpChunk), which lies inside segment `seg`, consist of one
 // run of period 1 or 2?  Updates `ar` when it enters a new such run.
 __device__ __forceinline__ bool chunk_alternates(AlternatingRun& ar, ExpandWarpSmem& ws, i64& desc_seg,
-                                                 const llmem_config* __restrict__ cfg, i64 seg, i64 gs, i64 ge,
-                                                 i64 tb, bool round, int lane) {
+                                                 const llmem_config* __restrict__ cfg,
+                                                 const SegDesc* __restrict__ table, i64 seg, i64 gs, i64 ge, i64 tb,
+                                                 bool round, int lane) {
   if (tb + kExpChunk <= ar.end) return true;
-  ensure_desc(ws, desc_seg, cfg, seg, gs, ge, round, lane);
+  ensure_desc(ws, desc_seg, cfg, table, seg, gs, ge, round, lane);
   if (ws.desc.invalid) return false;
   int r, o, it;
   locate(ws.desc, (u32)(tb - gs), &r, &o, &it);

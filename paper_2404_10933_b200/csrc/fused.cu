@@ -42,6 +42,27 @@ constexpr i64 kFusedSegmentCost = LLMEM_FUSED_SEGMENT_COST;
 #define LLMEM_FUSED_MIN_CHUNKS 128
 #endif
 
+// Descriptor of every configuration, one thread each: on lists of short segments the warps of
+// the expansion cross a segment boundary every few chunks, and building the descriptor there
+// (one lane, a thousand dependent instructions) is the larger part of what a boundary costs.
+__global__ void __launch_bounds__(128)
+desc_table_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict__ offsets, int round,
+                  SegDesc* __restrict__ table) {
+  const i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) build_desc(table[i], cfg + i, __ldg(offsets + i), __ldg(offsets + i + 1), round != 0);
+}
+
+// Lists whose segments average fewer events than this get 16 warps per CTA and a descriptor
+// table; longer ones 12 warps and descriptors built where they are needed.
+inline bool long_segments(i64 n, i64 total_events) { return n > 0 && total_events / n >= kFusedLongSegment; }
+
+constexpr size_t kDescTableOffset = (kStreamScratchBytes + 255) / 256 * 256;
+
+size_t expand_scan_scratch_bytes(long long n, long long total_events) {
+  if (n <= 0 || total_events <= 0 || long_segments(n, total_events)) return kStreamScratchBytes;
+  return kDescTableOffset + (size_t)n * sizeof(SegDesc);
+}
+
 // Fold of a full chunk whose events alternate between two values, v0 on even positions and
 // v1 on odd ones (constant runs have v0 == v1): with s = v0 + v1 the prefix sums are
 // k s + v0 after position 2k and (k + 1) s after position 2k + 1, both linear in k, so the
@@ -86,7 +107,7 @@ __global__ void __launch_bounds__(kFusedWarps * 32)
 expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict__ offsets, i64 total,
                    i64* __restrict__ out, i64 n_blocks, i64 kappa, int bulk_ok, i64* __restrict__ peak_out,
                    i64* __restrict__ index_out, i64* __restrict__ bounds, WarpPartials* __restrict__ partials,
-                   unsigned long long* __restrict__ work_counter) {
+                   unsigned long long* __restrict__ work_counter, const SegDesc* __restrict__ table) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   ExpandWarpSmem& ws = reinterpret_cast<ExpandWarpSmem*>(smem_raw)[warp];
@@ -118,7 +139,7 @@ expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __res
       i64* buf = ws.buf[parity];
       // a full chunk inside one segment may repeat the one before
       const bool alternating = seg < n && gs <= tb && tb + kExpChunk <= ge &&
-                               chunk_alternates(ar, ws, desc_seg, cfg, seg, gs, ge, tb, kRoundList, lane);
+                               chunk_alternates(ar, ws, desc_seg, cfg, table, seg, gs, ge, tb, kRoundList, lane);
       if (alternating) {
         prepare_alternating<kFusedStoresInFlight>(ar, keys, parity, buf, lane);
         folder.add_uniform(fold_alternating_chunk(ev<!kRoundList>(ar.x0), ev<!kRoundList>(ar.x1), tb), lane);
@@ -145,7 +166,7 @@ expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __res
             for (i64 e = (span_lo > pos ? span_lo : pos); e < span_hi; ++e) buf[e - tb] = 0;
             break;
           }
-          ensure_desc(ws, desc_seg, cfg, seg, gs, ge, kRoundList, lane);
+          ensure_desc(ws, desc_seg, cfg, table, seg, gs, ge, kRoundList, lane);
           const i64 piece_end = ge < te ? ge : te;
           const i64 e = span_lo > pos ? span_lo : pos;
           const i64 e_end = span_hi < piece_end ? span_hi : piece_end;
@@ -229,8 +250,18 @@ extern "C" llmem_status llmem_expand_scan(const llmem_config* cfg, int64_t n, co
   i64 warps = 1;
   if (total_events > 0) {
     const i64 nchunks = (total_events + kExpChunk - 1) / kExpChunk;
-    const bool long_segments = total_events / n >= kFusedLongSegment;
-    const int warps_per_cta = long_segments ? kFusedWarpsLong : kFusedWarpsShort;
+    const bool long_list = long_segments(n, total_events);
+    const int warps_per_cta = long_list ? kFusedWarpsLong : kFusedWarpsShort;
+    const bool round = (flags & LLMEM_FUSE_ROUND) != 0;
+    const SegDesc* table = nullptr;
+    if (!long_list) {
+      SegDesc* t = reinterpret_cast<SegDesc*>(static_cast<unsigned char*>(scratch) + kDescTableOffset);
+      desc_table_kernel<<<(unsigned)((n + 127) / 128), 128, 0, s>>>(cfg, n, reinterpret_cast<const i64*>(offsets),
+                                                                  round ? 1 : 0, t);
+      llmem_status st = check_launch("llmem_expand_scan (descriptor table)");
+      if (st != LLMEM_OK) return st;
+      table = t;
+    }
     const size_t smem = sizeof(ExpandWarpSmem) * warps_per_cta;
     static thread_local int configured_dev = -1;
     int dev = 0;
@@ -250,13 +281,12 @@ extern "C" llmem_status llmem_expand_scan(const llmem_config* cfg, int64_t n, co
     warps = stream_warps(resident, LLMEM_FUSED_OVERSUB, nchunks, LLMEM_FUSED_MIN_CHUNKS);
     const unsigned grid = (unsigned)(((warps < resident ? warps : resident) + warps_per_cta - 1) / warps_per_cta);
     const int bulk_ok = aligned_to(delta_out, 16) ? 1 : 0;
-    const bool round = (flags & LLMEM_FUSE_ROUND) != 0;
 #define LLMEM_LAUNCH_FUSED(ROUND, WARPS)                                                                        \
   expand_scan_kernel<ROUND, WARPS><<<grid, WARPS * 32, smem, s>>>(                                              \
       cfg, n, reinterpret_cast<const i64*>(offsets), total_events, reinterpret_cast<i64*>(delta_out), warps,    \
       kFusedSegmentCost, bulk_ok, reinterpret_cast<i64*>(peak_out), reinterpret_cast<i64*>(peak_index_out),      \
-      bounds, partials, work_counter)
-    if (long_segments) {
+      bounds, partials, work_counter, table)
+    if (long_list) {
       if (round) LLMEM_LAUNCH_FUSED(true, kFusedWarpsLong); else LLMEM_LAUNCH_FUSED(false, kFusedWarpsLong);
     } else {
       if (round) LLMEM_LAUNCH_FUSED(true, kFusedWarpsShort); else LLMEM_LAUNCH_FUSED(false, kFusedWarpsShort);

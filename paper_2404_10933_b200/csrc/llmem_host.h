@@ -41,4 +41,8 @@ constexpr size_t kScratchHeader = 256;
 // kernel claim their next block of work.
 constexpr size_t kWorkCounterOffset = 64;
 
+// Scratch of llmem_expand_scan: header, block starts, partials and, for lists of short
+// segments, one descriptor per configuration (defined with the kernel).
+size_t expand_scan_scratch_bytes(long long n, long long total_events);
+
 }  // namespace llmem
