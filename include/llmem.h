@@ -204,7 +204,9 @@ llmem_status llmem_scan_peak(const int64_t* DEV delta, const int64_t* DEV offset
  *   delta_out      DEV [total_events]
  *   peak_out       DEV [n]
  *   peak_index_out DEV [n], nullable
- *   scratch        required, llmem_scratch_bytes(LLMEM_OP_EXPAND_SCAN, n, total_events) bytes,
+ *   scratch        required, llmem_scratch_bytes(LLMEM_OP_EXPAND_SCAN, n, total_events) bytes
+ *                  (for the same n and total_events: lists whose segments are short on average
+ *                  need about 1 KB per configuration more, for a table of segment descriptors),
  *                  256-byte aligned; the call clears its header (status word, work counter)
  *                  and rewrites what it reads, so the buffer may be reused by later calls in
  *                  the same stream, but not by calls that may run at the same time */
