@@ -617,7 +617,7 @@ def run_slab_path(args):
         "roofline": {"bound": "hbm", "kernel": "whole step (expand_scan_kernel per slab + counts + host slab loop)",
                      "achieved": achieved, "peak": peak_gbs, "unit": "GB/s", "frac": achieved / peak_gbs,
                      "peak_source": peak_src, "traffic": None},
-        "gpu_launches": steps * (3 + slabs * 5), "clocks": clocks, "fused_equals_materialised": agree,
+        "gpu_launches": steps * (3 + slabs * 6), "clocks": clocks, "fused_equals_materialised": agree,
     }
     print(json.dumps(line))
     return 0 if agree else 4
