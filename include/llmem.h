@@ -78,7 +78,8 @@ typedef enum {
   LLMEM_ERR_ARG = 1,     /* null / misaligned pointer, negative size, bmax out of range */
   LLMEM_ERR_SCRATCH = 2, /* scratch missing, misaligned or too small */
   LLMEM_ERR_CUDA = 3,    /* a CUDA runtime call failed; text in llmem_last_error() */
-  LLMEM_ERR_TIMEOUT = 4  /* a bounded device-side wait ran out (llmem_scratch_status only) */
+  LLMEM_ERR_TIMEOUT = 4, /* a bounded device-side wait ran out (llmem_scratch_status only) */
+  LLMEM_ERR_CHECK = 5    /* an index check of a checked build failed (llmem_scratch_status only) */
 } llmem_status;
 
 /* per-configuration status bytes */
@@ -282,7 +283,8 @@ llmem_status llmem_chunk_search(const llmem_config* DEV cfg, int64_t n, int64_t 
 /* Synchronises cuda_stream and returns the device status word that
  * llmem_scan_peak keeps at the start of its scratch: LLMEM_OK, or
  * LLMEM_ERR_TIMEOUT if a bounded wait inside a kernel gave up (outputs are then
- * undefined). */
+ * undefined), LLMEM_ERR_CHECK if an index check of a checked build failed.  The scratch
+ * may be that of llmem_scan_peak, llmem_expand_scan or llmem_expand_events. */
 llmem_status llmem_scratch_status(const void* DEV scratch, void* cuda_stream);
 
 /* No counterpart in the paper: a check of this library's own failure handling.  The scan
@@ -307,6 +309,13 @@ llmem_status llmem_selftest_wait_limit(void* DEV scratch, size_t scratch_bytes, 
  *   warp_instructions_out  HOST, nullable */
 llmem_status llmem_selftest_int_rate(int kind, uint32_t iters, uint64_t* DEV sink,
                                      int64_t* warp_instructions_out, void* cuda_stream);
+
+/* 1 if the library was compiled with -DLLMEM_DEBUG (csrc/libllmem_debug.so), else 0.  A
+ * checked build tests every index its streaming kernels derive from offsets, block and
+ * segment numbers before using it; a failed test skips the access and leaves its number in
+ * the scratch status word, which llmem_scratch_status reports as LLMEM_ERR_CHECK.  No
+ * counterpart in the paper: it stands in for a memory checker while kernels are changed. */
+int llmem_checked_build(void);
 
 /* Text of the last error on the calling thread ("" if none). */
 const char* llmem_last_error(void);

@@ -22,8 +22,12 @@ from . import grids  # noqa: F401  (input generators; no part of the model)
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "csrc", "libllmem.so")
+# the checked build (-DLLMEM_DEBUG); set LLMEM_CHECKED=1 before the first call to load it instead
+DEBUG_LIB_PATH = os.path.join(_HERE, "csrc", "libllmem_debug.so")
+if os.environ.get("LLMEM_CHECKED") == "1":
+    LIB_PATH = DEBUG_LIB_PATH
 
-OK, ERR_ARG, ERR_SCRATCH, ERR_CUDA, ERR_TIMEOUT = 0, 1, 2, 3, 4
+OK, ERR_ARG, ERR_SCRATCH, ERR_CUDA, ERR_TIMEOUT, ERR_CHECK = 0, 1, 2, 3, 4, 5
 OP_ESTIMATE, OP_EVENT_COUNTS, OP_EXPAND, OP_ROUND, OP_SCAN_PEAK, OP_MAX_BATCH, OP_SELECT, OP_EXPAND_SCAN = range(8)
 SELECT_ALLZERO = 1
 FUSE_ROUND = 2
@@ -34,7 +38,7 @@ EXPORTS = (
     "llmem_round_events", "llmem_scan_peak", "llmem_max_batch", "llmem_select_method",
     "llmem_scratch_status", "llmem_last_error", "llmem_version", "llmem_event_counts_static",
     "llmem_select_segmented", "llmem_expand_scan", "llmem_chunk_search",
-    "llmem_selftest_wait_limit", "llmem_selftest_int_rate",
+    "llmem_selftest_wait_limit", "llmem_selftest_int_rate", "llmem_checked_build",
 )
 STATIC_MAX_CONFIGS = 4194304
 
@@ -56,7 +60,10 @@ def lib() -> ctypes.CDLL:
             # a source checkout without build artefacts: compile in-tree if nvcc is at hand
             try:
                 from . import _build
-                _build.build()
+                if LIB_PATH == DEBUG_LIB_PATH:
+                    _build.build_checked()
+                else:
+                    _build.build()
             except Exception as e:  # noqa: BLE001
                 raise ImportError(
                     f"{LIB_PATH} is missing and could not be built ({e}): build it with "
@@ -83,6 +90,7 @@ def lib() -> ctypes.CDLL:
         L.llmem_scratch_status.argtypes = [vp, vp]
         L.llmem_last_error.restype = ctypes.c_char_p
         L.llmem_version.restype = ctypes.c_int
+        L.llmem_checked_build.restype = ctypes.c_int
         for name in EXPORTS:
             getattr(L, name)  # every declared entry point must be exported
         _lib = L

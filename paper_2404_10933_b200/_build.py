@@ -10,6 +10,7 @@ from concurrent.futures import ThreadPoolExecutor
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(CSRC, "libllmem.so")
+DEBUG_LIB = os.path.join(CSRC, "libllmem_debug.so")
 SOURCES = ("api.cu", "estimate.cu", "events.cu", "scan.cu", "fused.cu")
 HEADERS = ("llmem_model.cuh", "llmem_host.h", "fold.cuh", "expand.cuh", "ranges.cuh", os.path.join("..", "..", "include", "llmem.h"))
 
@@ -61,6 +62,12 @@ def build(force: bool = False, verbose: bool = False, extra_flags=(), out: str |
                            "-cudart", "static"])
     os.replace(tmp, target)
     return target
+
+
+def build_checked(verbose: bool = False) -> str:
+    """The same library with -DLLMEM_DEBUG: every index the streaming kernels derive is tested
+    before use (csrc/libllmem_debug.so; load it by setting LLMEM_CHECKED=1)."""
+    return build(force=True, verbose=verbose, extra_flags=["-DLLMEM_DEBUG"], out=DEBUG_LIB)
 
 
 if __name__ == "__main__":

@@ -102,6 +102,14 @@ extern "C" const char* llmem_last_error(void) { return g_error; }
 
 extern "C" int llmem_version(void) { return 100; }
 
+extern "C" int llmem_checked_build(void) {
+#ifdef LLMEM_DEBUG
+  return 1;
+#else
+  return 0;
+#endif
+}
+
 extern "C" size_t llmem_scratch_bytes(int op, int64_t n, int64_t total_events) {
   if (n < 0) n = 0;
   switch (op) {
@@ -136,6 +144,10 @@ extern "C" llmem_status llmem_scratch_status(const void* scratch, void* cuda_str
   if (e != cudaSuccess) {
     set_error("llmem_scratch_status: %s", cudaGetErrorString(e));
     return LLMEM_ERR_CUDA;
+  }
+  if (word >= 16) {
+    set_error("index check %u of the checked build failed; the access was skipped", word - 16);
+    return LLMEM_ERR_CHECK;
   }
   if (word != 0) {
     set_error("a bounded device-side wait gave up (status word %u)", word);

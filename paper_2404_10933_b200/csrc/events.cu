@@ -135,10 +135,11 @@ add_block_base_kernel(i64* __restrict__ offsets, i64 n, const u64* __restrict__ 
 __global__ void __launch_bounds__(kExpThreads)
 expand_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict__ offsets, i64 total,
               i64* __restrict__ out, i64 n_blocks, i64 kappa, int round, int bulk_ok,
-              unsigned long long* __restrict__ work_counter) {
+              unsigned long long* __restrict__ work_counter, u32* __restrict__ status_word) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   ExpandWarpSmem& ws = reinterpret_cast<ExpandWarpSmem*>(smem_raw)[warp];
+  const Guard g{status_word, n, total};
   const i64 resident = (i64)gridDim.x * kExpWarps;
   i64 desc_seg = -1;  // segment described by ws.desc
   int parity = 0;
@@ -158,7 +159,7 @@ expand_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict
       i64* buf = ws.buf[parity];
       // a full chunk inside one segment may repeat the one before
       const bool alternating = seg < n && gs <= tb && tb + kExpChunk <= ge &&
-                               chunk_alternates(ar, ws, desc_seg, cfg, nullptr, seg, gs, ge, tb, round != 0, lane);
+                               chunk_alternates(ar, ws, desc_seg, cfg, nullptr, seg, gs, ge, tb, round != 0, lane, g);
       if (alternating) {
         prepare_alternating<kExpStoresInFlight>(ar, keys, parity, buf, lane);
         if (ge == te) {
@@ -183,11 +184,11 @@ expand_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict
             for (i64 e = (span_lo > pos ? span_lo : pos); e < span_hi; ++e) buf[e - tb] = 0;
             break;
           }
-          ensure_desc(ws, desc_seg, cfg, nullptr, seg, gs, ge, round != 0, lane);
+          ensure_desc(ws, desc_seg, cfg, nullptr, seg, gs, ge, round != 0, lane, g);
           const i64 piece_end = ge < te ? ge : te;
           const i64 e = span_lo > pos ? span_lo : pos;
           const i64 e_end = span_hi < piece_end ? span_hi : piece_end;
-          if (e < e_end) {
+          if (e < e_end && in_bounds(e >= tb && e_end <= tb + kExpChunk, g, kSiteFill)) {
             if (ws.desc.invalid) {
               for (i64 j = e; j < e_end; ++j) buf[j - tb] = 0;
             } else {
@@ -208,7 +209,7 @@ expand_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict
         if (bulk_ok) fence_async_shared();
         __syncwarp();
       }
-      store_chunk(out, tb, (u32)(te - tb), buf, bulk_ok, lane);
+      store_chunk(out, tb, (u32)(te - tb), buf, bulk_ok, lane, g);
     }
     if (work_counter == nullptr) break;  // one block per warp
     // the first `resident` blocks are taken by number, the others in order of request
@@ -380,15 +381,19 @@ extern "C" llmem_status llmem_expand_events(const llmem_config* cfg, int64_t n, 
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   // with scratch the warps of a persistent grid claim blocks from a counter in its header
   unsigned long long* work_counter = nullptr;
-  if (scratch && aligned_to(scratch, 256) && scratch_bytes >= kScratchHeader && blocks > resident) {
+  u32* status_word = nullptr;  // only written by checked builds
+  if (scratch && aligned_to(scratch, 256) && scratch_bytes >= kScratchHeader) {
     if (cudaMemsetAsync(scratch, 0, kScratchHeader, s) != cudaSuccess) return check_launch("llmem_expand_events (memset)");
-    work_counter = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(scratch) + kWorkCounterOffset);
+    status_word = static_cast<u32*>(scratch);
+    if (blocks > resident)
+      work_counter = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(scratch) + kWorkCounterOffset);
   }
   const i64 grid_warps = work_counter ? resident : blocks;
   const i64 grid = (grid_warps + kExpWarps - 1) / kExpWarps;
   expand_kernel<<<(unsigned)grid, kExpThreads, smem, s>>>(
       cfg, n, reinterpret_cast<const i64*>(offsets), total_events, reinterpret_cast<i64*>(delta_out),
-      blocks, kExpSegmentCost, (flags & LLMEM_FUSE_ROUND) ? 1 : 0, aligned_to(delta_out, 16) ? 1 : 0, work_counter);
+      blocks, kExpSegmentCost, (flags & LLMEM_FUSE_ROUND) ? 1 : 0, aligned_to(delta_out, 16) ? 1 : 0, work_counter,
+      status_word);
   return check_launch("llmem_expand_events");
 }
 

@@ -273,10 +273,12 @@ struct BufferKeys {
 static_assert(sizeof(SegDesc) % 16 == 0, "descriptors are copied in 16-byte words");
 __device__ __forceinline__ void ensure_desc(ExpandWarpSmem& ws, i64& desc_seg, const llmem_config* __restrict__ cfg,
                                             const SegDesc* __restrict__ table, i64 seg, i64 gs, i64 ge, bool round,
-                                            int lane) {
+                                            int lane, const Guard& g) {
   if (desc_seg != seg) {
     __syncwarp();  // every lane is done with the previous descriptor
-    if (table) {
+    if (!in_bounds(seg >= 0 && seg < g.n, g, kSiteDescriptor)) {
+      if (lane == 0) ws.desc.invalid = 1;  // the segment is written as zeros
+    } else if (table) {
       const int4* src = reinterpret_cast<const int4*>(table + seg);
       int4* dst = reinterpret_cast<int4*>(&ws.desc);
       for (int k = lane; k < (int)(sizeof(SegDesc) / 16); k += 32) dst[k] = __ldg(src + k);
@@ -293,9 +295,9 @@ __device__ __forceinline__ void ensure_desc(ExpandWarpSmem& ws, i64& desc_seg, c
 __device__ __forceinline__ bool chunk_alternates(AlternatingRun& ar, ExpandWarpSmem& ws, i64& desc_seg,
                                                  const llmem_config* __restrict__ cfg,
                                                  const SegDesc* __restrict__ table, i64 seg, i64 gs, i64 ge, i64 tb,
-                                                 bool round, int lane) {
+                                                 bool round, int lane, const Guard& g) {
   if (tb + kExpChunk <= ar.end) return true;
-  ensure_desc(ws, desc_seg, cfg, table, seg, gs, ge, round, lane);
+  ensure_desc(ws, desc_seg, cfg, table, seg, gs, ge, round, lane, g);
   if (ws.desc.invalid) return false;
   int r, o, it;
   locate(ws.desc, (u32)(tb - gs), &r, &o, &it);
@@ -334,7 +336,8 @@ __device__ __forceinline__ void prepare_alternating(const AlternatingRun& ar, Bu
 // Hands chunk [tb, tb + cnt) to the TMA engine (or copies it with plain stores when the
 // output is not 16-byte aligned).
 __device__ __forceinline__ void store_chunk(i64* __restrict__ out, i64 tb, u32 cnt, const i64* __restrict__ buf,
-                                            int bulk_ok, int lane) {
+                                            int bulk_ok, int lane, const Guard& g) {
+  if (!in_bounds(tb >= 0 && cnt <= (u32)kExpChunk && tb + (i64)cnt <= g.total, g, kSiteStore)) return;
   if (bulk_ok) {
     if (lane == 0) {
       const u32 even = cnt & ~1u;

@@ -205,9 +205,10 @@ struct SegmentFolder {
   // Segment `seg` (starting at index seg_start) ends here: store its bare result, or, if it
   // began before this warp's range (range_lo), leave the part seen here as the head partial.
   __device__ __forceinline__ void finish_segment(i64 seg, i64 seg_start, i64 range_lo, WarpPartials* my_partials,
-                                                 i64* __restrict__ peak_out, i64* __restrict__ index_out, int lane) {
+                                                 i64* __restrict__ peak_out, i64* __restrict__ index_out, int lane,
+                                                 const Guard& g) {
     const Agg run = take();
-    if (lane == 0) {
+    if (lane == 0 && in_bounds(seg >= 0 && seg < g.n, g, kSiteResult)) {
       if (seg_start >= range_lo) write_raw(seg, run, seg_start, peak_out, index_out);
       else my_partials->head = run;
     }

@@ -111,6 +111,8 @@ expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __res
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   ExpandWarpSmem& ws = reinterpret_cast<ExpandWarpSmem*>(smem_raw)[warp];
+  // the status word is the first word of the scratch header, the work counter sits kWorkCounterOffset into it
+  const Guard g{reinterpret_cast<u32*>(reinterpret_cast<unsigned char*>(work_counter) - kWorkCounterOffset), n, total};
   const i64 resident = (i64)gridDim.x * kFusedWarps;
   i64 desc_seg = -1;
   int parity = 0;
@@ -121,6 +123,7 @@ expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __res
     const i64 b_hi = warp_block_start(offsets, n, 0, total, gw + 1, n_blocks, kappa, kExpChunk, lane, nullptr);
     const i64 c_lo = b_lo / kExpChunk, c_hi = (b_hi + kExpChunk - 1) / kExpChunk;
     const i64 range_lo = c_lo * kExpChunk;  // a segment that starts at or after this started in this block
+    if (!in_bounds(gw >= 0 && gw < kMaxStreamWarps, g, kSiteBlock)) break;
     WarpPartials* my_partials = partials + gw;
     if (lane == 0) {
       my_partials->head = agg_identity();
@@ -139,13 +142,13 @@ expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __res
       i64* buf = ws.buf[parity];
       // a full chunk inside one segment may repeat the one before
       const bool alternating = seg < n && gs <= tb && tb + kExpChunk <= ge &&
-                               chunk_alternates(ar, ws, desc_seg, cfg, table, seg, gs, ge, tb, kRoundList, lane);
+                               chunk_alternates(ar, ws, desc_seg, cfg, table, seg, gs, ge, tb, kRoundList, lane, g);
       if (alternating) {
         prepare_alternating<kFusedStoresInFlight>(ar, keys, parity, buf, lane);
         folder.add_uniform(fold_alternating_chunk(ev<!kRoundList>(ar.x0), ev<!kRoundList>(ar.x1), tb), lane);
         if (ge == te) {
           // the segment ends with this chunk: finish it and move to the next non-empty one
-          folder.finish_segment(seg, gs, range_lo, my_partials, peak_out, index_out, lane);
+          folder.finish_segment(seg, gs, range_lo, my_partials, peak_out, index_out, lane, g);
           do {
             ++seg;
             gs = seg < n ? __ldg(offsets + seg) : total;
@@ -166,11 +169,11 @@ expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __res
             for (i64 e = (span_lo > pos ? span_lo : pos); e < span_hi; ++e) buf[e - tb] = 0;
             break;
           }
-          ensure_desc(ws, desc_seg, cfg, table, seg, gs, ge, kRoundList, lane);
+          ensure_desc(ws, desc_seg, cfg, table, seg, gs, ge, kRoundList, lane, g);
           const i64 piece_end = ge < te ? ge : te;
           const i64 e = span_lo > pos ? span_lo : pos;
           const i64 e_end = span_hi < piece_end ? span_hi : piece_end;
-          if (e < e_end) {
+          if (e < e_end && in_bounds(e >= tb && e_end <= tb + kExpChunk, g, kSiteFill)) {
             if (ws.desc.invalid) {
               for (i64 j = e; j < e_end; ++j) buf[j - tb] = 0;
             } else {
@@ -190,7 +193,7 @@ expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __res
           pos = piece_end;
           if (ge <= te) {
             // the segment ends inside this chunk: finish it and move to the next non-empty one
-            folder.finish_segment(seg, gs, range_lo, my_partials, peak_out, index_out, lane);
+            folder.finish_segment(seg, gs, range_lo, my_partials, peak_out, index_out, lane, g);
             do {
               ++seg;
               gs = seg < n ? __ldg(offsets + seg) : total;
@@ -202,7 +205,7 @@ expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __res
         if (bulk_ok) fence_async_shared();
         __syncwarp();
       }
-      store_chunk(out, tb, (u32)(te - tb), buf, bulk_ok, lane);
+      store_chunk(out, tb, (u32)(te - tb), buf, bulk_ok, lane, g);
     }
     // the current segment may continue into the next block
     folder.finish_range(gs, range_lo, my_partials, lane);

@@ -23,6 +23,34 @@ constexpr u64 kPage = 2ull * 1024ull * 1024ull;  // cu_p, Section 4.2
 constexpr u64 kSat = 1ull << 62;                 // bytes limit (exclusive)
 constexpr u64 kCountLimit = 1ull << 31;          // events limit (exclusive)
 
+// Checked builds (-DLLMEM_DEBUG, csrc/libllmem_debug.so): the streaming kernels test every
+// index they derive from offsets, block numbers and segment numbers before using it.  A
+// failed test records 16 + its site number in the scratch status word (the largest one wins)
+// and the access is skipped; nothing traps.  In normal builds in_bounds() is the constant
+// true and the tests cost nothing.
+#ifdef LLMEM_DEBUG
+constexpr bool kChecked = true;
+#else
+constexpr bool kChecked = false;
+#endif
+constexpr u32 kCheckBase = 16;  // status words from here on name a failed check
+
+struct Guard {
+  u32* word;  // scratch status word, or null
+  i64 n;      // configurations
+  i64 total;  // events
+};
+
+enum CheckSite : u32 { kSiteStore = 1, kSiteDescriptor = 2, kSiteBlock = 3, kSiteResult = 4, kSiteLoad = 5, kSiteFill = 6 };
+
+__device__ __forceinline__ bool in_bounds(bool ok, const Guard& g, u32 site) {
+  if (kChecked && !ok) {
+    if (g.word) atomicMax(g.word, kCheckBase + site);
+    return false;
+  }
+  return true;
+}
+
 __host__ __device__ __forceinline__ u64 sat_add(u64 a, u64 b) {
   u64 s = a + b;  // a, b <= 2^62: no wrap
   return s > kSat ? kSat : s;

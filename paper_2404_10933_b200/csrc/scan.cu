@@ -146,6 +146,8 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
   // virtual indices: event e lives at v = e + shift, so that v even <=> 16-byte aligned
   const i64 v_begin = shift, v_end = (i64)shift + total;
   if (gw >= n_warps) return;
+  const Guard guard{status_word, n, total};
+  if (!in_bounds(gw < kMaxStreamWarps, guard, kSiteBlock)) return;
   // this warp's block of chunks: balanced by events + kappa per segment (ranges.cuh)
   i64 seg;  // the segment that contains the first event of the current chunk
   const i64 b_lo = warp_block_start(offsets, n, shift, v_end, gw, n_warps, kappa, kScanChunk, lane, &seg);
@@ -177,7 +179,7 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
     // ragged first / last element (at most one each): plain loads
     if (a_lo > v_lo) dst[v_lo - t0] = delta_aligned[v_lo];
     if (a_hi < v_hi && v_hi - 1 >= a_lo) dst[v_hi - 1 - t0] = delta_aligned[v_hi - 1];
-    if (a_hi > a_lo) {
+    if (a_hi > a_lo && in_bounds(a_lo >= v_begin && a_hi <= v_end && a_hi - a_lo <= kScanChunk, guard, kSiteLoad)) {
       const u32 bytes = (u32)((a_hi - a_lo) * 8);
       mbar_arrive_expect_tx(&ws.full[s], bytes);
       bulk_load(dst + (a_lo - t0), delta_aligned + a_lo, bytes, &ws.full[s]);
@@ -221,7 +223,7 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
       if (lane == 0 && c + kScanStages < c_hi) issue(c + kScanStages);
       folder.add_spans<kScanPerLane>(f, t0, lane);
       if (seg_vend == v_hi) {
-        folder.finish_segment(seg, seg_vstart, warp_vlo, my_partials, peak_out, index_out, lane);
+        folder.finish_segment(seg, seg_vstart, warp_vlo, my_partials, peak_out, index_out, lane, guard);
         next_segment(v_hi);
       }
       continue;
@@ -235,7 +237,7 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
       folder.add_piece(g, lane);
       pos = pb;
       if (seg_vend <= v_hi) {
-        folder.finish_segment(seg, seg_vstart, warp_vlo, my_partials, peak_out, index_out, lane);
+        folder.finish_segment(seg, seg_vstart, warp_vlo, my_partials, peak_out, index_out, lane, guard);
         next_segment(pos);
       }
     }

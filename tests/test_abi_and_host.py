@@ -137,3 +137,15 @@ def test_slab_bounds_cover_and_respect_the_budget():
         grids.slab_bounds(off, 0)
     with pytest.raises(ValueError):
         grids.slab_bounds(off, 10, 301)
+
+
+def test_checked_build_exports_the_same_entry_points():
+    from paper_2404_10933_b200 import _build
+    assert llmem.lib().llmem_checked_build() == 0
+    if not os.path.exists(_build.DEBUG_LIB):
+        _build.build_checked()
+    D = ctypes.CDLL(_build.DEBUG_LIB)
+    for name in declared_symbols():
+        getattr(D, name)
+    D.llmem_checked_build.restype = ctypes.c_int
+    assert D.llmem_checked_build() == 1

@@ -481,6 +481,54 @@ def test_materialised_path_in_slabs(llmem):
     assert np.array_equal(again["index"].cpu().numpy()[k:], want["index"][k:])
 
 
+CHECKED_SCRIPT = r"""
+import numpy as np, torch
+import oracle
+import paper_2404_10933_b200 as llmem
+from paper_2404_10933_b200 import grids
+L = llmem.lib()
+assert L.llmem_checked_build() == 1
+import tests.test_gpu_parity as t
+tiny = grids.g2_shape_grid(7, 1)
+tiny["layers"] = 1 + (np.arange(len(tiny)) % 3)
+tiny["hidden"], tiny["heads"], tiny["ffn"] = 256, 4, 1024
+for cfgs in (t.mixed_small_grid(), grids.g5_stress(5, 48), tiny, grids.g2_shape_grid(3, 6)):
+    want = oracle.estimate(cfgs, threads=8)
+    dev = llmem.to_device(cfgs)
+    offsets, _ = llmem.event_counts(dev)
+    total = int(offsets[-1].item())
+    for shift in (0, 1):
+        buf = torch.zeros(total + 2, dtype=torch.int64, device="cuda")
+        view = buf[shift:shift + total]
+        header = torch.zeros(256, dtype=torch.uint8, device="cuda")
+        llmem.expand_events(dev, offsets, total, fuse_round=True, out=view, scratch=header)
+        assert L.llmem_scratch_status(header.data_ptr(), None) == llmem.OK, L.llmem_last_error()
+        r = llmem.scan_peak(view, offsets, dev)
+        assert L.llmem_scratch_status(r["scratch"].data_ptr(), None) == llmem.OK, L.llmem_last_error()
+        one = llmem.expand_scan(dev, offsets, total, fuse_round=True, out=view)
+        assert L.llmem_scratch_status(one["scratch"].data_ptr(), None) == llmem.OK, L.llmem_last_error()
+        for res in (r, one):
+            assert np.array_equal(res["peak"].cpu().numpy(), want["peak"])
+            assert np.array_equal(res["index"].cpu().numpy(), want["index"])
+print("checked build ok")
+"""
+
+
+def test_checked_build_finds_nothing_and_agrees(llmem):
+    """The library compiled with its index checks on (every offset, block and segment index the
+    streaming kernels derive is tested before use) runs the same grids: no check fires and the
+    results are those of the oracle.  It runs in a process of its own because a process loads
+    one build of the library."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, LLMEM_CHECKED="1", PYTHONPATH=root)
+    p = subprocess.run([sys.executable, "-c", CHECKED_SCRIPT], cwd=root, env=env, capture_output=True, text=True,
+                       timeout=600)
+    assert p.returncode == 0 and "checked build ok" in p.stdout, p.stdout + p.stderr
+
+
 def test_issue_rate_probe(llmem):
     import ctypes
     L = llmem.lib()
