@@ -473,7 +473,7 @@ def run_ours(args):
 # ---------------------------------------------------------------------------
 # Warp instructions executed per unit of work (smsp__inst_executed.sum / units) from ncu
 # captures of these kernels on reduced grids; None once a kernel changes after the capture.
-NCU_WARP_INSTR_PER_UNIT = {"estimate_kernel": 30.88, "max_batch_kernel": 11.38, "select_kernel": 64.93}
+NCU_WARP_INSTR_PER_UNIT = {"estimate_kernel": 30.88, "max_batch_kernel": 11.40, "select_kernel": 65.03}
 
 
 def run_register_paths(args):

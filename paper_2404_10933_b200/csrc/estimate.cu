@@ -17,7 +17,11 @@
 #endif
 // CTAs per SM the estimate's grid is capped at (its threads stride over the configurations)
 #ifndef LLMEM_EST_GRID_CTAS
-#define LLMEM_EST_GRID_CTAS 8
+#define LLMEM_EST_GRID_CTAS 32
+#endif
+// the same for the two search kernels
+#ifndef LLMEM_SEARCH_GRID_CTAS
+#define LLMEM_SEARCH_GRID_CTAS 256
 #endif
 #ifndef LLMEM_SEARCH_MIN_CTAS
 #define LLMEM_SEARCH_MIN_CTAS 4
@@ -427,7 +431,7 @@ extern "C" llmem_status llmem_max_batch(const llmem_config* shape, int64_t n,
   llmem_status st = check_search_args("llmem_max_batch", shape, n, capacity_bytes, n_cap, bmax);
   if (st != LLMEM_OK || n == 0 || n_cap == 0) return st;
   if (!bs_out || !aligned_to(bs_out, 4)) { set_error("llmem_max_batch: bs_out is required"); return LLMEM_ERR_ARG; }
-  max_batch_kernel<<<grid_for(n, 256, 8), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+  max_batch_kernel<<<grid_for(n, 256, LLMEM_SEARCH_GRID_CTAS), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
       shape, n, reinterpret_cast<const i64*>(capacity_bytes), n_cap, bmax, bs_out, status_out);
   return check_launch("llmem_max_batch");
 }
@@ -443,7 +447,7 @@ extern "C" llmem_status llmem_select_method(const llmem_config* shape, int64_t n
   llmem_status st = check_search_args("llmem_select_method", shape, n, capacity_bytes, n_cap, bmax);
   if (st != LLMEM_OK || n == 0 || n_cap == 0) return st;
   if (!method_out || !batch_out) { set_error("llmem_select_method: method_out and batch_out are required"); return LLMEM_ERR_ARG; }
-  select_kernel<<<grid_for(4 * n, 256, 8), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+  select_kernel<<<grid_for(4 * n, 256, LLMEM_SEARCH_GRID_CTAS), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
       shape, n, reinterpret_cast<const i64*>(capacity_bytes), n_cap, bmax, flags, method_out,
       batch_out, bs_list_out, status_out);
   return check_launch("llmem_select_method");
