@@ -14,7 +14,8 @@ other path are timed alone after the step and reported next to it.
 
 `value` is alloc-events per second over all ranks with the configurations already
 resident in HBM; `e2e` is the same pass through the public API starting from pinned
-host buffers, with the host<->device copies inside the timed region.  The roofline
+host buffers, with every step's host<->device copies inside the timed region (the steps
+run as a two-stage pipeline: step i + 1's inputs come in while step i computes).  The roofline
 block reports the dominant kernel against the measured HBM copy bandwidth.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
@@ -260,38 +261,59 @@ class HotPath:
         return {"peak": r["peak"], "index": r["index"], "bs": bs, "method": sel["method"],
                 "batch": sel["batch"], "offsets": offsets}
 
-    def step_e2e(self):
-        """Host buffers in, host results out: H2D of the configurations and capacities, the
-        device-to-host read of the event total that sizes the list, every kernel, and the
-        D2H of peaks and selections.  The searches and the copy of their results need only the
-        configurations, so they are queued on a second stream and run underneath the
-        expansion; both streams are joined before the step ends."""
+    def run_e2e(self, steps: int):
+        """`steps` end-to-end steps as a two-stage pipeline, the way a caller with a stream of
+        batches would drive the library: while step i computes on the main stream, the copy
+        stream brings in the configurations of step i + 1, counts their events and hands the
+        total to the host (which needs it to size the list), and afterwards takes step i's
+        results back.  Every step still moves its own inputs and outputs; nothing is reused
+        between steps but the buffers."""
         torch, llmem = self.torch, self.llmem
-        main = torch.cuda.current_stream()
-        cfg = self.host_cfg.to("cuda", non_blocking=True)
-        caps = self.host_caps.to("cuda", non_blocking=True)
-        self.fork.record(main)
-        self.side.wait_event(self.fork)
-        with torch.cuda.stream(self.side):
+        main, copy = torch.cuda.current_stream(), self.side
+        if not hasattr(self, "host_total"):
+            self.host_total = torch.zeros(2, dtype=torch.int64).pin_memory()
+
+        def stage(k):
+            copy.wait_stream(main) if k == 0 else None
+            with torch.cuda.stream(copy):
+                cfg = self.host_cfg.to("cuda", non_blocking=True)
+                caps = self.host_caps.to("cuda", non_blocking=True)
+                offsets, _ = llmem.event_counts(cfg)
+                self.host_total[k % 2:k % 2 + 1].copy_(offsets[-1:], non_blocking=True)
+                ready = torch.cuda.Event()
+                ready.record(copy)
+            return cfg, caps, offsets, ready
+
+        nxt = stage(0)
+        for i in range(steps):
+            cfg, caps, offsets, ready = nxt
+            ready.synchronize()                               # the host needs this step's event total
+            total = int(self.host_total[i % 2])
+            if total > self.delta.numel():
+                self.delta = torch.empty(total, dtype=torch.int64, device="cuda")
+            main.wait_event(ready)
+            for t in (cfg, caps, offsets):
+                t.record_stream(main)
+            if i + 1 < steps:
+                nxt = stage(i + 1)
+            if self.one_pass:
+                r = llmem.expand_scan(cfg, offsets, total, fuse_round=True, out=self.delta, scratch=self.scan_scratch)
+            else:
+                delta = llmem.expand_events(cfg, offsets, total, fuse_round=True, out=self.delta)
+                r = llmem.scan_peak(delta, offsets, cfg, scratch=self.scan_scratch)
             llmem.max_batch(cfg, caps, self.bmax, want_status=False)
             sel = llmem.select_method(cfg, caps, self.bmax, want_bs_list=False, want_status=False)
-            self.host_out["method"].copy_(sel["method"], non_blocking=True)
-            self.host_out["batch"].copy_(sel["batch"], non_blocking=True)
-        offsets, _ = llmem.event_counts(cfg)
-        total = int(offsets[-1].item())                      # 8-byte D2H + sync
-        if total > self.delta.numel():
-            self.delta = torch.empty(total, dtype=torch.int64, device="cuda")
-        if self.one_pass:
-            r = llmem.expand_scan(cfg, offsets, total, fuse_round=True, out=self.delta, scratch=self.scan_scratch)
-        else:
-            delta = llmem.expand_events(cfg, offsets, total, fuse_round=True, out=self.delta)
-            r = llmem.scan_peak(delta, offsets, cfg, scratch=self.scan_scratch)
-        self.host_out["peak"].copy_(r["peak"], non_blocking=True)
-        main.wait_stream(self.side)
-        for t in (cfg, caps, sel["method"], sel["batch"]):
-            t.record_stream(self.side)
+            done = torch.cuda.Event()
+            done.record(main)
+            copy.wait_event(done)
+            with torch.cuda.stream(copy):
+                self.host_out["peak"].copy_(r["peak"], non_blocking=True)
+                self.host_out["method"].copy_(sel["method"], non_blocking=True)
+                self.host_out["batch"].copy_(sel["batch"], non_blocking=True)
+            for t in (r["peak"], sel["method"], sel["batch"]):
+                t.record_stream(copy)
+        main.wait_stream(copy)
         main.synchronize()
-        return total
 
     def time_kernel(self, what, reps=5):
         """Mean launch time (ms) of one of the HBM-bound kernels on the resident grid."""
@@ -396,17 +418,19 @@ def run_ours(args):
     agree = bool(torch.equal(fused["peak"], out["peak"]) and torch.equal(fused["index"], out["index"]))
 
     # ---- end to end from host buffers ----
-    for _ in range(min(args.warmup, 3)):
-        hp.step_e2e()
+    hp.run_e2e(min(args.warmup, 3))
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     e2e_steps = max(1, min(args.steps, 100))
-    for _ in range(e2e_steps):
-        hp.step_e2e()
+    hp.run_e2e(e2e_steps)
     e1.record()
     barrier()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1))
+    # what came back to the host must be what the device-resident step computed
+    e2e_agree = bool(torch.equal(hp.host_out["peak"], out["peak"].cpu()) and
+                     torch.equal(hp.host_out["method"], out["method"].cpu()) and
+                     torch.equal(hp.host_out["batch"], out["batch"].cpu()))
     e2e_value = total_events_all * e2e_steps / (e2e_ms * 1e-3)
 
     if rank != 0:
@@ -458,14 +482,14 @@ def run_ours(args):
                 "d2h_bytes_per_step": hp.d2h_bytes, "ms_per_step": e2e_ms / e2e_steps},
         "gpu_launches": hp.kernels_per_step * args.steps,
         "clocks": clocks,
-        "fused_equals_materialised": agree,
+        "fused_equals_materialised": agree, "e2e_equals_resident": e2e_agree,
     }
     if args.cpu_baseline:
         line["cpu_baseline"] = cpu_baseline()
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
-    return 0 if agree else 4
+    return 0 if (agree and e2e_agree) else 4
 
 
 # ---------------------------------------------------------------------------
