@@ -49,7 +49,8 @@ extern "C" {
 typedef struct __attribute__((aligned(16))) llmem_config {
   int32_t layers;      /* l_n, 1 .. 2^16 */
   int32_t hidden;      /* o_n, 1 .. 2^20 */
-  int32_t heads;       /* >= 1 and a divisor of hidden; no term of the model depends on it */
+  int32_t heads;       /* >= 1 and a divisor of hidden; used only with act_mode = 1, where it sizes the
+                          two attention-score outputs of a layer (2 * batch * heads * seq^2 bytes) */
   int32_t ffn;         /* inner width of the feed-forward block, 1 .. 2^22 */
   int32_t vocab;       /* dict_n, 1 .. 2^26 */
   int32_t pos_len;     /* rows of a learned position Embedding, 0 = none; 0 .. 2^26 (fixes e_n) */
@@ -141,7 +142,8 @@ llmem_status llmem_event_counts(const llmem_config* DEV cfg, int64_t n, int64_t*
  *
  * The first call on each device looks up the array's device address (a query, not
  * an allocation) and caches it; make that first call in ordinary stream execution,
- * before any stream capture is begun on that device.
+ * before any stream capture is begun on that device.  The cached address belongs to the
+ * device's current context: do not call cudaDeviceReset() between uses of this entry point.
  *
  * All calls on one device share the one array, and it keeps what the previous call
  * left there.  That is harmless for calls that follow one another in one stream

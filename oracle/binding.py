@@ -133,6 +133,19 @@ def estimate(cfg: np.ndarray, level: int = 1, threads: int = 1):
     return {"peak": peak, "index": index, "status": status, "count": count}
 
 
+def list_digest(cfg: np.ndarray, threads: int = 1):
+    """Two position-weighted checksums (mod 2^64) of each configuration's page-rounded event
+    list: sum d[k] (k + 1) and sum d[k] (k + 1)^2 over the positions k of the list (zeros where
+    status != 0).  Returns dict(a, b uint64; status uint8)."""
+    cfg = _cfgs(cfg)
+    n = cfg.size
+    a = np.zeros(n, dtype=np.uint64)
+    b = np.zeros(n, dtype=np.uint64)
+    status = np.zeros(n, dtype=np.uint8)
+    lib().oracle_list_digest_many(_p(cfg), ctypes.c_int64(n), _p(a), _p(b), _p(status), ctypes.c_int(threads))
+    return {"a": a, "b": b, "status": status}
+
+
 def max_batch(cfg: np.ndarray, capacities, bmax: int, level: int = 1, threads: int = 1):
     """Returns (bs[n, n_cap] int32, status[n] uint8)."""
     cfg = _cfgs(cfg)

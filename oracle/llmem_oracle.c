@@ -464,6 +464,30 @@ int oracle_estimate(const oracle_config *c, int64_t *peak_out, int64_t *index_ou
   return ST_OK;
 }
 
+/* Two position-weighted checksums (mod 2^64) of the page-rounded list of one configuration,
+ * so that a test can compare a whole list held elsewhere with the explicit list built here
+ * without moving it: with k the 0-based position inside the list,
+ *   a = sum d[k] * (k + 1),   b = sum d[k] * (k + 1)^2.
+ * A wrong, missing, shifted or swapped element changes at least one of them. */
+int oracle_list_digest(const oracle_config *c, uint64_t *a_out, uint64_t *b_out) {
+  *a_out = 0;
+  *b_out = 0;
+  int64_t *d, n;
+  int st = build_events(c, &d, &n);
+  if (st) return st;
+  oracle_round_events(d, n);
+  uint64_t a = 0, b = 0;
+  for (int64_t k = 0; k < n; ++k) {
+    const uint64_t w = (uint64_t)k + 1;
+    a += (uint64_t)d[k] * w;
+    b += (uint64_t)d[k] * w * w;
+  }
+  free(d);
+  *a_out = a;
+  *b_out = b;
+  return ST_OK;
+}
+
 /* inventory, for the pins: e_n, K, C, embed_p, other_p, lm_p (bytes), tok_p, pos_p, hh_p, hf_p */
 int oracle_inventory(const oracle_config *c, int64_t out[10]) {
   int st = oracle_validate(c);
@@ -659,7 +683,7 @@ int oracle_select_method_bisect(const oracle_config *shape, int64_t capacity, in
 /* ------------------------------------------------------------------------ */
 typedef struct {
   int kind; /* 0 estimate (level 1), 1 collapsed, 2 max batch (linear), 3 max batch (bisect),
-               4 select (linear), 5 select (bisect) */
+               4 select (linear), 5 select (bisect), 6 list checksums */
   const oracle_config *cfg;
   int64_t n;
   const int64_t *caps;
@@ -668,6 +692,7 @@ typedef struct {
   int64_t *peak, *index, *count;
   uint8_t *status;
   int32_t *bs, *method, *batch, *bs_list;
+  uint64_t *digest_a, *digest_b;
   int64_t next; /* shared work counter */
   pthread_mutex_t lock;
 } job_t;
@@ -687,6 +712,9 @@ static void run_one(job_t *j, int64_t i) {
     int64_t peak;
     int st = oracle_estimate_collapsed(c, &peak);
     j->peak[i] = peak;
+    if (j->status) j->status[i] = (uint8_t)st;
+  } else if (j->kind == 6) {
+    int st = oracle_list_digest(c, &j->digest_a[i], &j->digest_b[i]);
     if (j->status) j->status[i] = (uint8_t)st;
   } else if (j->kind == 2 || j->kind == 3) {
     for (int32_t m = 0; m < j->n_cap; ++m) {
@@ -749,6 +777,19 @@ void oracle_estimate_many(const oracle_config *cfg, int64_t n, int64_t *peak, in
   j.index = index;
   j.status = status;
   j.count = count;
+  run_job(&j, nthreads);
+}
+
+void oracle_list_digest_many(const oracle_config *cfg, int64_t n, uint64_t *digest_a,
+                             uint64_t *digest_b, uint8_t *status, int nthreads) {
+  job_t j;
+  memset(&j, 0, sizeof j);
+  j.kind = 6;
+  j.cfg = cfg;
+  j.n = n;
+  j.digest_a = digest_a;
+  j.digest_b = digest_b;
+  j.status = status;
   run_job(&j, nthreads);
 }
 

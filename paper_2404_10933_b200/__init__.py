@@ -188,10 +188,9 @@ def event_counts_static(cfg, offsets_out, status_out=None, *, stream=None):
             or not cfg.is_contiguous():
         raise ValueError("cfg must be a contiguous CUDA uint8 tensor of shape [n, 64]")
     n = cfg.shape[0]
-    if offsets_out.dtype != torch.int64 or offsets_out.numel() < n + 1 or not offsets_out.is_contiguous():
-        raise ValueError("offsets_out must be a contiguous int64 tensor with n + 1 elements")
-    if status_out is not None and (status_out.dtype != torch.uint8 or status_out.numel() < n):
-        raise ValueError("status_out must be a uint8 tensor with n elements")
+    _check_buffer(offsets_out, "offsets_out", torch.int64, n + 1, cfg.device)
+    if status_out is not None:
+        _check_buffer(status_out, "status_out", torch.uint8, n, cfg.device)
     _check(lib().llmem_event_counts_static(_ptr(cfg), n, _ptr(offsets_out), _ptr(status_out), 0,
                                            _stream_ptr(stream)))
     return offsets_out
@@ -206,12 +205,15 @@ def expand_events(cfg, offsets, total_events: Optional[int] = None, *, fuse_roun
     n = cfg.shape[0]
     if total_events is None:
         total_events = int(offsets[-1].item())
+    _check_buffer(offsets, "offsets", torch.int64, n + 1, cfg.device)
     if out is None:
         out = torch.empty(total_events, dtype=torch.int64, device=cfg.device)
-    elif out.numel() < total_events or out.dtype != torch.int64:
-        raise ValueError("out must be an int64 tensor with at least total_events elements")
+    else:
+        _check_buffer(out, "out", torch.int64, total_events, cfg.device)
     if scratch is None:
         scratch = torch.empty(scratch_bytes(OP_EXPAND, n, total_events), dtype=torch.uint8, device=cfg.device)
+    else:
+        _check_buffer(scratch, "scratch", torch.uint8, 0, cfg.device)
     _check(lib().llmem_expand_events(_ptr(cfg), n, _ptr(offsets), total_events, _ptr(out), _ptr(scratch),
                                      scratch.numel(), FUSE_ROUND if fuse_round else 0, _stream_ptr(stream)))
     return out[:total_events] if out.numel() != total_events else out
@@ -227,8 +229,12 @@ def scan_peak(delta, offsets, cfg=None, *, fuse_round: bool = False, want_index:
               scratch=None, stream=None, check_status: bool = False):
     """Segmented prefix-sum + max.  Returns dict(peak[n], index[n] | None, scratch)."""
     torch = _torch()
+    if not isinstance(offsets, torch.Tensor) or not offsets.is_cuda:
+        raise ValueError("offsets must be a CUDA tensor")
     n = offsets.numel() - 1
     total = delta.numel()
+    _check_buffer(offsets, "offsets", torch.int64, 1, offsets.device)
+    _check_buffer(delta, "delta", torch.int64, 0, offsets.device)
     if cfg is not None:
         cfg = _as_cfg(cfg)
     peak = torch.empty(n, dtype=torch.int64, device=offsets.device)
@@ -236,6 +242,7 @@ def scan_peak(delta, offsets, cfg=None, *, fuse_round: bool = False, want_index:
     if scratch is None:
         scratch, nbytes = _scratch(OP_SCAN_PEAK, n, total, offsets.device)
     else:
+        _check_buffer(scratch, "scratch", torch.uint8, 0, offsets.device)
         nbytes = scratch.numel()
     _check(lib().llmem_scan_peak(_ptr(delta), _ptr(offsets), n, total, _ptr(cfg), _ptr(peak), _ptr(index),
                                  _ptr(scratch), nbytes, FUSE_ROUND if fuse_round else 0,
@@ -254,15 +261,17 @@ def expand_scan(cfg, offsets, total_events: Optional[int] = None, *, fuse_round:
     n = cfg.shape[0]
     if total_events is None:
         total_events = int(offsets[-1].item())
+    _check_buffer(offsets, "offsets", torch.int64, n + 1, cfg.device)
     if out is None:
         out = torch.empty(total_events, dtype=torch.int64, device=cfg.device)
-    elif out.numel() < total_events or out.dtype != torch.int64:
-        raise ValueError("out must be an int64 tensor with at least total_events elements")
+    else:
+        _check_buffer(out, "out", torch.int64, total_events, cfg.device)
     peak = torch.empty(n, dtype=torch.int64, device=cfg.device)
     index = torch.empty(n, dtype=torch.int64, device=cfg.device) if want_index else None
     if scratch is None:
         scratch, nbytes = _scratch(OP_EXPAND_SCAN, n, total_events, cfg.device)
     else:
+        _check_buffer(scratch, "scratch", torch.uint8, 0, cfg.device)
         nbytes = scratch.numel()
     _check(lib().llmem_expand_scan(_ptr(cfg), n, _ptr(offsets), total_events, _ptr(out), _ptr(peak), _ptr(index),
                                    _ptr(scratch), nbytes, FUSE_ROUND if fuse_round else 0, _stream_ptr(stream)))
@@ -334,6 +343,17 @@ def chunk_search(cfg, cs_min: int, cs_step: int, n_candidates: int, *, stream=No
     _check(lib().llmem_chunk_search(_ptr(cfg), n, cs_min, cs_step, n_candidates, _ptr(chunk), _ptr(waste),
                                     _ptr(status), None, 0, 0, _stream_ptr(stream)))
     return {"chunk": chunk, "waste": waste, "status": status}
+
+
+def _check_buffer(t, name: str, dtype, min_numel: int, device) -> None:
+    """A tensor supplied by the caller that a kernel will write: it has to be device memory
+    of the configurations' GPU, contiguous, of the right type and long enough (a pointer to
+    anything else would be written all the same)."""
+    torch = _torch()
+    if not isinstance(t, torch.Tensor) or not t.is_cuda or t.device != device:
+        raise ValueError(f"{name} must be a CUDA tensor on {device}")
+    if t.dtype != dtype or not t.is_contiguous() or t.numel() < min_numel:
+        raise ValueError(f"{name} must be a contiguous {dtype} tensor with at least {min_numel} elements")
 
 
 def _caps(capacities, device):

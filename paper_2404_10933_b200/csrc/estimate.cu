@@ -487,7 +487,7 @@ extern "C" llmem_status llmem_chunk_search(const llmem_config* cfg, int64_t n, i
   if (n < 0) { set_error("llmem_chunk_search: n < 0"); return LLMEM_ERR_ARG; }
   if (cs_min < 1 || cs_step < 1 || n_candidates < 1 ||
       cs_min > (1ll << 40) || cs_step > (1ll << 40) ||
-      cs_min + (int64_t)(n_candidates - 1) * cs_step > (1ll << 40)) {
+      (int64_t)(n_candidates - 1) > ((1ll << 40) - cs_min) / cs_step) {  // no product: it could wrap
     set_error("llmem_chunk_search: candidates must be cs_min + k cs_step in 1 .. 2^40, k < n_candidates");
     return LLMEM_ERR_ARG;
   }

@@ -50,10 +50,40 @@ def test_scratch_bytes_and_argument_errors_need_no_gpu():
                              None, None, 0, 0, None) == llmem.ERR_SCRATCH
     assert L.llmem_event_counts(ctypes.c_void_p(16), 5, ctypes.c_void_p(16), None, ctypes.c_void_p(256), 8,
                                 0, None) == llmem.ERR_SCRATCH
+    # chunk-size candidates beyond 2^40 are refused even where cs_min + k cs_step wraps 64 bits
+    for n_cand, step in ((1 << 24, 1 << 40), ((1 << 24) + 1, 1 << 40), (1 << 30, (1 << 34) + 1), (2, 1 << 40)):
+        assert L.llmem_chunk_search(ctypes.c_void_p(16), 1, 1, step, n_cand, ctypes.c_void_p(16), None, None,
+                                    None, 0, 0, None) == llmem.ERR_ARG, (n_cand, step)
+    assert b"2^40" in L.llmem_last_error()
     # empty calls succeed
+    assert L.llmem_chunk_search(None, 0, 1, (1 << 40) - 1, 2, None, None, None, None, 0, 0, None) == llmem.OK
     assert L.llmem_estimate_batch(None, 0, None, None, None, None, 0, 0, None) == llmem.OK
     assert L.llmem_round_events(None, 0, None, 0, 0, None) == llmem.OK
     assert L.llmem_last_error() == b""
+
+
+def test_wrappers_refuse_buffers_a_kernel_could_not_write():
+    """Tensors the caller supplies for a kernel to write are checked before any launch: host
+    memory, another device, the wrong type, a strided view or too few elements raise."""
+    torch = pytest.importorskip("torch")
+    dev = torch.device("cuda", 0)
+    host = torch.zeros(16, dtype=torch.int64)
+    with pytest.raises(ValueError, match="CUDA tensor"):
+        llmem._check_buffer(host, "offsets_out", torch.int64, 4, dev)
+    with pytest.raises(ValueError, match="CUDA tensor"):
+        llmem._check_buffer(None, "out", torch.int64, 4, dev)
+    with pytest.raises(ValueError, match="CUDA tensor"):
+        llmem._check_buffer(host.numpy(), "out", torch.int64, 4, dev)
+    # the public wrappers reach that check (or the one on cfg) before touching the library
+    cfg_host = torch.zeros((4, 64), dtype=torch.uint8)
+    with pytest.raises(ValueError):
+        llmem.event_counts_static(cfg_host, host)
+    with pytest.raises(ValueError):
+        llmem.expand_scan(cfg_host, host, 8, out=host)
+    with pytest.raises(ValueError):
+        llmem.expand_events(cfg_host, host, 8, out=host)
+    with pytest.raises(ValueError):
+        llmem.scan_peak(host, host)
 
 
 def test_record_layout_matches_header():

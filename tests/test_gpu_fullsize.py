@@ -1,8 +1,13 @@
 """Parity at the full sizes of the five configuration grids, in the launch
-configuration the benchmark times.  Where the level-1 oracle (explicit event list)
-would take too long for every element, all elements are compared with the oracle's
-level-2 evaluation (shown equal to level 1 by the CPU pins) and a seeded sample is
-compared with level 1, including event-list slices and peak positions."""
+configuration the benchmark times.  Every peak, peak position, status and event count of
+the shape grid, the large sweep and the stress grid is compared with the oracle's level 1
+(explicit event list, rounding, linear scan); whole materialised lists are compared with
+the oracle's explicit lists through position-weighted checksums of every segment and
+element by element on samples.  Only the 75.5 M searches of the max-batch grid rest on the
+oracle's bisecting level 2 (shown equal to the literal increment by the CPU pins), with the
+defining property checked against level 1 on a sample."""
+import os
+
 import numpy as np
 import pytest
 
@@ -12,7 +17,7 @@ from paper_2404_10933_b200 import grids
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
-THREADS = 16
+THREADS = os.cpu_count() or 16
 
 
 @pytest.fixture(scope="module")
@@ -24,43 +29,98 @@ def llmem():
     return m
 
 
+_LEVEL1 = {}
+
+
+def level1(name, make_cfgs):
+    """Level-1 oracle results of a whole grid, computed once per test session."""
+    if name not in _LEVEL1:
+        cfgs = make_cfgs()
+        _LEVEL1[name] = (cfgs, oracle.estimate(cfgs, level=1, threads=THREADS))
+    return _LEVEL1[name]
+
+
 def sample_indices(n, k, seed):
     return np.sort(np.random.default_rng(seed).choice(n, size=min(k, n), replace=False))
 
 
+def assert_equals_level1(got, want, status=None, offsets=None):
+    """peak, index (and status, event counts where given) of every configuration."""
+    assert np.array_equal(got["peak"].cpu().numpy(), want["peak"])
+    assert np.array_equal(got["index"].cpu().numpy(), want["index"])
+    if status is not None:
+        assert np.array_equal(status.cpu().numpy(), want["status"])
+    if offsets is not None:
+        counts = np.diff(offsets.cpu().numpy())
+        assert np.array_equal(counts, np.where(want["status"] == 0, want["count"], 0))
+
+
+def device_list_digests(delta, offsets, slab_events=1 << 27):
+    """The two checksums of oracle.list_digest for every segment of a list on the device,
+    with plain torch integer ops (wrapping 64-bit arithmetic), slab by slab."""
+    off = offsets.cpu().numpy()
+    n = len(off) - 1
+    dev = delta.device
+    a = torch.zeros(n, dtype=torch.int64, device=dev)
+    b = torch.zeros(n, dtype=torch.int64, device=dev)
+    s0 = 0
+    while s0 < n:
+        s1 = int(np.searchsorted(off, off[s0] + slab_events, side="right")) - 1
+        s1 = min(max(s1, s0 + 1), n)
+        lo, hi = int(off[s0]), int(off[s1])
+        if hi > lo:
+            starts = torch.from_numpy(off[s0:s1] - lo).to(dev)
+            ends = torch.from_numpy(off[s0 + 1:s1 + 1] - lo).to(dev)
+            seg = torch.repeat_interleave(torch.arange(s1 - s0, device=dev), ends - starts)
+            k1 = torch.arange(hi - lo, device=dev) - starts[seg] + 1
+            del seg
+            t = delta[lo:hi] * k1
+            for out in (a, b):
+                cs = torch.cat([torch.zeros(1, dtype=torch.int64, device=dev), torch.cumsum(t, 0)])
+                out[s0:s1] = cs[ends] - cs[starts]
+                del cs
+                t *= k1
+            del t, k1
+        s0 = s1
+    return a.cpu().numpy().view(np.uint64), b.cpu().numpy().view(np.uint64)
+
+
+def assert_lists_equal_oracle(delta, offsets, cfgs):
+    """Every segment of the list against the oracle's explicit page-rounded list."""
+    want = oracle.list_digest(cfgs, threads=THREADS)
+    a, b = device_list_digests(delta, offsets)
+    assert np.array_equal(a, want["a"])
+    assert np.array_equal(b, want["b"])
+
+
 def test_g2_shape_grid_full(llmem):
-    cfgs = grids.g2_shape_grid()
+    cfgs, want1 = level1("g2", grids.g2_shape_grid)
     assert len(cfgs) == 4096 * 32 * 29
     got = llmem.estimate_batch(cfgs)
-    want2 = oracle.estimate(cfgs, level=2, threads=THREADS)
-    assert np.array_equal(got["status"].cpu().numpy(), want2["status"])
-    peak = got["peak"].cpu().numpy()
-    assert np.array_equal(peak, want2["peak"])
-    idx = sample_indices(len(cfgs), 1500, 2)
-    want1 = oracle.estimate(cfgs[idx], level=1, threads=THREADS)
-    assert np.array_equal(peak[idx], want1["peak"])
-    assert np.array_equal(got["index"].cpu().numpy()[idx], want1["index"])
+    offsets, _ = llmem.event_counts(cfgs)
+    assert_equals_level1(got, want1, got["status"], offsets)
 
 
 def test_g2_shape_grid_full_materialised_in_slabs(llmem):
     """The whole shape grid as materialised lists (4.6e10 events, 365 GB as int64: eight times
     the device memory one list buffer may take here), slab by slab through one 32 GiB buffer."""
-    cfgs = grids.g2_shape_grid()
+    cfgs, want1 = level1("g2", grids.g2_shape_grid)
     free, _ = torch.cuda.mem_get_info()
     budget = 1 << 32                                    # events per slab: 32 GiB of int64
-    if free < budget * 8 + (4 << 30):
-        pytest.skip("needs 36 GiB of free device memory")
-    r = llmem.estimate_in_slabs(cfgs, budget)
+    if free < budget * 8 + (12 << 30):
+        pytest.skip("needs 44 GiB of free device memory")
+    # whole lists of two slabs, every segment, against the oracle's explicit lists
+    checked = []
+
+    def on_slab(lo, hi, delta, local_offsets):
+        if len(checked) in (0, 5):
+            assert_lists_equal_oracle(delta, local_offsets, cfgs[lo:hi])
+        checked.append((lo, hi))
+
+    r = llmem.estimate_in_slabs(cfgs, budget, on_slab=on_slab)
     torch.cuda.synchronize()
-    assert len(r["bounds"]) > 8
-    want2 = oracle.estimate(cfgs, level=2, threads=THREADS)
-    assert np.array_equal(r["status"].cpu().numpy(), want2["status"])
-    peak = r["peak"].cpu().numpy()
-    assert np.array_equal(peak, want2["peak"])
-    idx = sample_indices(len(cfgs), 1500, 12)
-    want1 = oracle.estimate(cfgs[idx], level=1, threads=THREADS)
-    assert np.array_equal(peak[idx], want1["peak"])
-    assert np.array_equal(r["index"].cpu().numpy()[idx], want1["index"])
+    assert len(r["bounds"]) > 8 and len(checked) == len(r["bounds"]) - 1
+    assert_equals_level1(r, want1, r["status"])
 
 
 def test_g2_slice_materialized_claimed_blocks(llmem):
@@ -102,22 +162,12 @@ def test_g2_slice_materialized_claimed_blocks(llmem):
 
 
 def test_g3_large_sweep_full(llmem):
-    cfgs = grids.g3_sweep()
+    cfgs, want1 = level1("g3", grids.g3_sweep)
     assert len(cfgs) == 1 << 20
+    assert (want1["status"] == 0).all()
     got = llmem.estimate_batch(cfgs)
-    want2 = oracle.estimate(cfgs, level=2, threads=THREADS)
-    peak = got["peak"].cpu().numpy()
-    assert (want2["status"] == 0).all()
-    assert np.array_equal(got["status"].cpu().numpy(), want2["status"])
-    assert np.array_equal(peak, want2["peak"])
-    idx = sample_indices(len(cfgs), 3000, 3)
-    want1 = oracle.estimate(cfgs[idx], level=1, threads=THREADS)
-    assert np.array_equal(peak[idx], want1["peak"])
-    assert np.array_equal(got["index"].cpu().numpy()[idx], want1["index"])
-    # event counts of the whole sweep
     offsets, _ = llmem.event_counts(cfgs)
-    counts = np.diff(offsets.cpu().numpy())
-    assert np.array_equal(counts[idx], want1["count"])
+    assert_equals_level1(got, want1, got["status"], offsets)
 
 
 def test_g4_max_batch_and_selection_full(llmem):
@@ -130,35 +180,35 @@ def test_g4_max_batch_and_selection_full(llmem):
     bs = bs.cpu().numpy()
     st = st.cpu().numpy()
     del dev
-    # every 16th shape in full against the bisecting oracle
-    sub = np.arange(0, 1 << 17, 16)
-    rows = (sub[:, None] * 64 + np.arange(64)[None, :]).reshape(-1)
-    want_bs, want_st = oracle.max_batch(search[rows], caps, bmax, level=2, threads=THREADS)
-    assert np.array_equal(st[rows], want_st)
-    assert np.array_equal(bs[rows], want_bs)
-    # the defining property with the level-1 estimate on a sample of the rest
+    # all 75.5 M searches against the bisecting oracle
+    want_bs, want_st = oracle.max_batch(search, caps, bmax, level=2, threads=THREADS)
+    assert np.array_equal(st, want_st)
+    assert np.array_equal(bs, want_bs)
+    del want_bs
+    # the defining property (b fits, b + 1 does not) with the level-1 estimate on a sample of
+    # the rest: every capacity of 4000 searches, evaluated as two batched oracle calls
     ok = np.flatnonzero(st == 0)
-    for i in sample_indices(len(ok), 120, 4):
-        r = ok[i]
-        for m in (0, 5, 8):
-            b = int(bs[r, m])
-            c = search[r:r + 1].copy()
-            if b >= 1:
-                c["batch"] = b
-                e = oracle.estimate(c)
-                assert e["status"][0] == 0 and e["peak"][0] <= caps[m]
-            if b < bmax:
-                c["batch"] = b + 1
-                e = oracle.estimate(c)
-                assert e["status"][0] != 0 or e["peak"][0] > caps[m]
+    pick = ok[sample_indices(len(ok), 4000, 4)]
+    ncap = len(caps)
+    b = bs[pick].astype(np.int64)                                   # [4000, ncap]
+    at = np.repeat(search[pick], ncap)
+    above = at.copy()
+    at["batch"] = np.maximum(b, 1).reshape(-1)
+    above["batch"] = np.minimum(b + 1, bmax).reshape(-1)
+    e_at = oracle.estimate(at, level=1, threads=THREADS)
+    e_above = oracle.estimate(above, level=1, threads=THREADS)
+    capm = np.tile(caps, len(pick))
+    fits = (e_at["status"] == 0) & (e_at["peak"] <= capm)
+    assert np.array_equal(fits, b.reshape(-1) >= 1)             # b = 0 exactly when batch 1 does not fit
+    too_big = (e_above["status"] != 0) | (e_above["peak"] > capm)
+    assert too_big[b.reshape(-1) < bmax].all()
     assert (st[search["method"] != 3] == 0).all()
     sel_cfg = grids.g4_select_grid()
     assert len(sel_cfg) == (1 << 17) * 16
     got = llmem.select_method(sel_cfg, caps, bmax)
-    rows = (sub[:, None] * 16 + np.arange(16)[None, :]).reshape(-1)
-    want = oracle.select_method(sel_cfg[rows], caps, bmax, level=2, threads=THREADS)
+    want = oracle.select_method(sel_cfg, caps, bmax, level=2, threads=THREADS)
     for k in ("method", "batch", "bs_list", "status"):
-        assert np.array_equal(got[k].cpu().numpy()[rows], want[k]), k
+        assert np.array_equal(got[k].cpu().numpy(), want[k]), k
     # selection is consistent with the search results of the same shapes everywhere
     bl = got["bs_list"].cpu().numpy()
     bs4 = np.maximum(bs.reshape(1 << 17, 4, 16, len(caps)), 0).transpose(0, 2, 3, 1).reshape(-1, len(caps), 4)
@@ -167,71 +217,64 @@ def test_g4_max_batch_and_selection_full(llmem):
 
 
 def test_g5_stress_materialized_full(llmem):
-    cfgs = grids.g5_stress()
+    cfgs, want1 = level1("g5", grids.g5_stress)
     assert len(cfgs) == 1 << 16
+    assert (want1["status"] == 0).all()
     dev = llmem.to_device(cfgs)
     offsets, status = llmem.event_counts(dev)
     total = int(offsets[-1].item())
     free, _ = torch.cuda.mem_get_info()
-    if free < total * 8 + (2 << 30):
-        pytest.skip(f"needs {total * 8 / 2**30:.0f} GiB of free device memory")
+    if free < 2 * total * 8 + (12 << 30):
+        pytest.skip(f"needs {2 * total * 8 / 2**30 + 12:.0f} GiB of free device memory")
     assert 4_000_000_000 < total < 8_000_000_000
     delta = llmem.expand_events(dev, offsets, total, fuse_round=True)
     r = llmem.scan_peak(delta, offsets, dev, check_status=True)
-    fused = llmem.estimate_batch(dev)
-    peak = r["peak"].cpu().numpy()
-    index = r["index"].cpu().numpy()
-    assert np.array_equal(peak, fused["peak"].cpu().numpy())
-    assert np.array_equal(index, fused["index"].cpu().numpy())
-    want2 = oracle.estimate(cfgs, level=2, threads=THREADS)
-    assert (want2["status"] == 0).all() and (status.cpu().numpy() == 0).all()
-    assert np.array_equal(peak, want2["peak"])
-    idx = sample_indices(len(cfgs), 96, 5)
-    want1 = oracle.estimate(cfgs[idx], level=1, threads=THREADS)
-    assert np.array_equal(peak[idx], want1["peak"])
-    assert np.array_equal(index[idx], want1["index"])
+    assert_equals_level1(r, want1, status, offsets)
+    assert_equals_level1(llmem.estimate_batch(dev), want1)
+    # the whole list, every segment, against the oracle's explicit lists
+    assert_lists_equal_oracle(delta, offsets, cfgs)
+    # the one-pass variant at full size: same peaks, and the same list bit for bit
+    delta_one = torch.zeros(total, dtype=torch.int64, device="cuda")
+    one = llmem.expand_scan(dev, offsets, total, fuse_round=True, out=delta_one)
+    assert_equals_level1(one, want1)
+    assert torch.equal(delta_one, delta)
+    del delta
+    # whole event lists of a few configurations, element by element
     off = offsets.cpu().numpy()
-    assert np.array_equal(np.diff(off)[idx], want1["count"])
-    # the one-pass variant at full size: same list, same peaks
-    delta.fill_(0)
-    one = llmem.expand_scan(dev, offsets, total, fuse_round=True, out=delta)
-    assert torch.equal(one["peak"], r["peak"]) and torch.equal(one["index"], r["index"])
-    # whole event lists of a few configurations, bit for bit
-    for i in idx[:6]:
+    for i in sample_indices(len(cfgs), 6, 5):
         ev = oracle.round_events(oracle.expand_events(cfgs[i:i + 1]))
-        assert np.array_equal(delta[off[i]:off[i + 1]].cpu().numpy(), ev)
+        assert np.array_equal(delta_one[off[i]:off[i + 1]].cpu().numpy(), ev)
 
 
 def test_g5_slice_with_all_operator_outputs(llmem):
     """A quarter of the stress shapes with every operator output kept: materialised, one-pass
-    and in-register results against the oracle, all configurations at level 2, a sample at
-    level 1 with whole lists."""
-    cfgs = grids.g5_stress(0, 16384).copy()
-    cfgs["act_mode"] = 1
+    and in-register results of every configuration against the oracle's level 1, and the
+    whole one-pass list against the oracle's explicit lists."""
+    def make():
+        c = grids.g5_stress(0, 16384).copy()
+        c["act_mode"] = 1
+        return c
+    cfgs, want1 = level1("g5_ops", make)
+    assert (want1["status"] == 0).all()
     dev = llmem.to_device(cfgs)
     offsets, status = llmem.event_counts(dev)
     total = int(offsets[-1].item())
     free, _ = torch.cuda.mem_get_info()
-    if free < total * 8 + (2 << 30):
-        pytest.skip(f"needs {total * 8 / 2**30:.0f} GiB of free device memory")
-    want2 = oracle.estimate(cfgs, level=2, threads=THREADS)
-    assert np.array_equal(status.cpu().numpy(), want2["status"])
-    assert (want2["status"] == 0).all()
+    if free < 2 * total * 8 + (12 << 30):
+        pytest.skip(f"needs {2 * total * 8 / 2**30 + 12:.0f} GiB of free device memory")
     fused = llmem.estimate_batch(dev)
-    assert np.array_equal(fused["status"].cpu().numpy(), want2["status"])
-    assert np.array_equal(fused["peak"].cpu().numpy(), want2["peak"])
+    assert_equals_level1(fused, want1, fused["status"], offsets)
+    assert np.array_equal(status.cpu().numpy(), want1["status"])
     delta = torch.empty(total, dtype=torch.int64, device="cuda")
     one = llmem.expand_scan(dev, offsets, total, fuse_round=True, out=delta)
-    assert torch.equal(one["peak"], fused["peak"]) and torch.equal(one["index"], fused["index"])
-    two = llmem.scan_peak(llmem.expand_events(dev, offsets, total, fuse_round=True), offsets, dev)
-    assert torch.equal(two["peak"], fused["peak"]) and torch.equal(two["index"], fused["index"])
-    idx = sample_indices(len(cfgs), 48, 11)
-    want1 = oracle.estimate(cfgs[idx], level=1, threads=THREADS)
-    assert np.array_equal(fused["peak"].cpu().numpy()[idx], want1["peak"])
-    assert np.array_equal(fused["index"].cpu().numpy()[idx], want1["index"])
+    assert_equals_level1(one, want1)
+    assert_lists_equal_oracle(delta, offsets, cfgs)
+    two_list = llmem.expand_events(dev, offsets, total, fuse_round=True)
+    assert torch.equal(two_list, delta)
+    two = llmem.scan_peak(two_list, offsets, dev, check_status=True)
+    assert_equals_level1(two, want1)
     off = offsets.cpu().numpy()
-    assert np.array_equal(np.diff(off)[idx], want1["count"])
-    for i in idx[:4]:
+    for i in sample_indices(len(cfgs), 4, 11):
         ev = oracle.round_events(oracle.expand_events(cfgs[i:i + 1]))
         assert np.array_equal(delta[off[i]:off[i + 1]].cpu().numpy(), ev)
 
@@ -239,8 +282,8 @@ def test_g5_slice_with_all_operator_outputs(llmem):
 def test_g4_selection_over_all_degrees_and_splits(llmem):
     """Per shape and capacity, the best of 67 candidates: CDP / ADP / TP on 1..16 devices and
     every admissible DP+TP split.  The CUDA pipeline (max_batch on all 8.8 M candidates, then
-    the segmented decision) runs at full size; every fourth shape is compared with the oracle
-    end to end (its own batches, its own decision)."""
+    the segmented decision) runs at full size and every shape is compared with the oracle end
+    to end (its own batches, its own decision)."""
     caps = grids.g4_capacities()
     cand, offsets = grids.g4_all_splits_grid()
     k = len(grids.all_split_candidates())
@@ -249,14 +292,10 @@ def test_g4_selection_over_all_degrees_and_splits(llmem):
     bs, st = llmem.max_batch(dev, caps, grids.G4_BMAX)
     got = llmem.select_segmented(dev, bs, offsets)
     assert int(st.max()) == 0
-    sub = np.arange(0, 1 << 17, 4)
-    rows = (sub[:, None] * k + np.arange(k)[None, :]).reshape(-1)
-    want_bs, _ = oracle.max_batch(cand[rows], caps, grids.G4_BMAX, level=2, threads=THREADS)
-    assert np.array_equal(bs.cpu().numpy()[rows], want_bs)
-    want = oracle.select_segmented(cand[rows], want_bs, np.arange(len(sub) + 1, dtype=np.int64) * k)
-    item = got["item"].cpu().numpy()[sub]
-    local = np.where(item >= 0, item - (sub * k)[:, None], -1)
-    assert np.array_equal(local, np.where(want["item"] >= 0, want["item"] - (np.arange(len(sub)) * k)[:, None], -1))
-    assert np.array_equal(got["method"].cpu().numpy()[sub], want["method"])
-    assert np.array_equal(got["batch"].cpu().numpy()[sub], want["batch"])
+    want_bs, _ = oracle.max_batch(cand, caps, grids.G4_BMAX, level=2, threads=THREADS)
+    assert np.array_equal(bs.cpu().numpy(), want_bs)
+    want = oracle.select_segmented(cand, want_bs, offsets)
+    assert np.array_equal(got["item"].cpu().numpy(), want["item"])
+    assert np.array_equal(got["method"].cpu().numpy(), want["method"])
+    assert np.array_equal(got["batch"].cpu().numpy(), want["batch"])
     assert set(np.unique(want["method"]).tolist()) >= {0, 1, 4}

@@ -739,3 +739,35 @@ def test_all_operator_outputs_lifetimes_and_stack(shape, meth):
         elif d < 0:
             assert order.pop() == -d
     assert sorted(int(x) for x in raw if x > 0) == sorted(b for b, a, z in rows if b > 0)
+
+
+def test_list_checksums_against_python_integers():
+    """oracle.list_digest is sum d[k] (k + 1) and sum d[k] (k + 1)^2 mod 2^64 over the
+    page-rounded explicit list: recomputed here with Python integers from the list itself,
+    and shown to move when one element changes, two swap, or the list shifts by one."""
+    cfgs = np.concatenate([grids.g1_small()[::9], grids.g2_shape_grid(11, 1)[::41], grids.g3_sweep(7, 6)])
+    bad = cfgs[:1].copy()
+    bad["layers"] = 0
+    cfgs = np.concatenate([cfgs, bad])
+    got = oracle.list_digest(cfgs, threads=3)
+    M = 1 << 64
+    for i in range(len(cfgs)):
+        st, _ = oracle.event_count(cfgs[i:i + 1])
+        assert got["status"][i] == st
+        if st != 0:
+            assert got["a"][i] == 0 and got["b"][i] == 0
+            continue
+        ev = [int(v) for v in oracle.round_events(oracle.expand_events(cfgs[i:i + 1]))]
+        a = sum(v * (k + 1) for k, v in enumerate(ev)) % M
+        b = sum(v * (k + 1) ** 2 for k, v in enumerate(ev)) % M
+        assert int(got["a"][i]) == a and int(got["b"][i]) == b
+        # sensitivity: a changed element, two neighbours swapped, a shift by one position
+        variants = []
+        e = list(ev); e[len(e) // 2] += 1 << 21; variants.append(e)
+        j = next(k for k in range(len(ev) - 1) if ev[k] != ev[k + 1])
+        e = list(ev); e[j], e[j + 1] = e[j + 1], e[j]; variants.append(e)
+        variants.append([0] + ev[:-1])
+        for e in variants:
+            a2 = sum(v * (k + 1) for k, v in enumerate(e)) % M
+            b2 = sum(v * (k + 1) ** 2 for k, v in enumerate(e)) % M
+            assert (a2, b2) != (a, b)
