@@ -12,7 +12,7 @@ CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(CSRC, "libllmem.so")
 DEBUG_LIB = os.path.join(CSRC, "libllmem_debug.so")
 SOURCES = ("api.cu", "estimate.cu", "events.cu", "scan.cu", "fused.cu")
-HEADERS = ("llmem_model.cuh", "llmem_host.h", "fold.cuh", "expand.cuh", "ranges.cuh", os.path.join("..", "..", "include", "llmem.h"))
+HEADERS = ("llmem_model.cuh", "llmem_host.h", "fold.cuh", "expand.cuh", "ranges.cuh", "spans.cuh", os.path.join("..", "..", "include", "llmem.h"))
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -44,22 +44,25 @@ constexpr i64 kExpSegmentCost = LLMEM_EXP_SEGMENT_COST;
 #define LLMEM_EXP_INFLIGHT 8
 #endif
 constexpr int kExpStoresInFlight = LLMEM_EXP_INFLIGHT;
-constexpr int kRuns = 19;
-constexpr int kDynFirst = 2, kDynLast = 15, kOsFirst = 16, kOsLast = 18;  // run indices, see SegDesc
+constexpr int kRuns = 16;
+constexpr int kDynFirst = 2, kDynLast = 13, kOsFirst = 14, kOsLast = 15;  // run indices, see SegDesc
 
 // A run of events that repeat with a short period (at most 16): position j of a period
 // has value v[(code >> 2j) & 3].  Constant runs use period 1 and code 0.
 struct alignas(16) Run {
   int cnt, period;
   u32 code;
-  int pad;
-  i64 a, b, c, pad2;
+  int start;  // events of the same group (initialisation / one iteration / optimizer states) before this run
+  i64 a, b, c;
+  i64 links;  // byte 0: the next non-empty run during the first iteration, byte 1: during later ones
 };
 
-// The event list of one configuration as runs.  Order: 0-1 initialisation; 2-15 one
-// iteration (gather, embedding outputs, per-layer operator outputs, logits, shifted
-// copies, TP buffers, then the frees mirrored); 16-18 optimizer states, which follow the
-// first iteration only.
+// The event list of one configuration as runs.  Order: 0-1 initialisation (embedding unit,
+// chunks); 2-13 one iteration (gathered embedding unit, gathered chunks, embedding and layer
+// outputs, per-layer operator outputs, logits with the two shifted copies, TP buffers, then
+// the frees mirrored); 14-15 optimizer states (embedding tensors, layer tensors), which
+// follow the first iteration only.  Neighbouring events of equal size share a run, and the
+// logits and their two copies form one run of period 3, so that a list has few runs.
 struct SegDesc {
   i64 gstart, gend;  // global event range of the segment
   u32 init_n, dyn_n, os_n;
@@ -68,7 +71,7 @@ struct SegDesc {
 };
 
 __device__ __forceinline__ void set_run(Run& r, int cnt, int period, u32 code, i64 a, i64 b, i64 c) {
-  r.cnt = cnt; r.period = period; r.code = code; r.pad = 0; r.a = a; r.b = b; r.c = c; r.pad2 = 0;
+  r.cnt = cnt; r.period = period; r.code = code; r.start = 0; r.a = a; r.b = b; r.c = c; r.links = 0;
 }
 __device__ __forceinline__ void set_const_run(Run& r, int cnt, i64 a) { set_run(r, cnt, 1, 0u, a, a, a); }
 
@@ -117,25 +120,45 @@ static __device__ __noinline__ void build_desc(SegDesc& d, const llmem_config* _
     fwd = layer_code(f.ffn_kind != 0, false, &n_ops);
     bwd = layer_code(f.ffn_kind != 0, true, &n_ops);
   }
+  // with gradient checkpointing a layer keeps one output of the size of an embedding output:
+  // one run; otherwise the layers' operator outputs form a periodic run of their own
+  const int plain_layers = f.act_mode ? 0 : L;
   set_const_run(d.run[2], G, ge);
   set_const_run(d.run[3], G * C, gc);
-  set_const_run(d.run[4], p.e_n, out);
-  set_run(d.run[5], L * n_ops, n_ops, fwd, out, at, ff);
-  set_const_run(d.run[6], 1, lg);
-  set_const_run(d.run[7], 2, sh);
-  set_const_run(d.run[8], T * L, bk);
-  set_const_run(d.run[9], T * L, -bk);
-  set_const_run(d.run[10], 2, -sh);
-  set_const_run(d.run[11], 1, -lg);
-  set_run(d.run[12], L * n_ops, n_ops, bwd, -out, -at, -ff);
-  set_const_run(d.run[13], p.e_n, -out);
-  set_const_run(d.run[14], G * C, -gc);
-  set_const_run(d.run[15], G, -ge);
-  set_const_run(d.run[16], 1, LLMEM_V(p.os_tok));
-  set_const_run(d.run[17], f.pos_len > 0 ? 1 : 0, LLMEM_V(p.os_pos));
+  set_const_run(d.run[4], p.e_n + plain_layers, out);
+  set_run(d.run[5], f.act_mode ? L * n_ops : 0, n_ops, fwd, out, at, ff);
+  set_run(d.run[6], 3, 3, 0x14u, lg, sh, 0);     // logits, shifted copy, shifted copy
+  set_const_run(d.run[7], T * L, bk);
+  set_const_run(d.run[8], T * L, -bk);
+  set_run(d.run[9], 3, 3, 0x05u, -lg, -sh, 0);   // the copies, then the logits
+  set_run(d.run[10], f.act_mode ? L * n_ops : 0, n_ops, bwd, -out, -at, -ff);
+  set_const_run(d.run[11], p.e_n + plain_layers, -out);
+  set_const_run(d.run[12], G * C, -gc);
+  set_const_run(d.run[13], G, -ge);
+  // token embedding states, then those of the position embedding if there is one
+  set_run(d.run[14], f.pos_len > 0 ? 2 : 1, 2, 1u << 2, LLMEM_V(p.os_tok), LLMEM_V(p.os_pos), 0);
   // per layer: four H x H tensors, then the feed-forward ones
-  set_run(d.run[18], p.K * L, p.K, p.K == 7 ? 0x1500u : 0x0500u, LLMEM_V(p.os_hh), LLMEM_V(p.os_hf), 0);
+  set_run(d.run[15], p.K * L, p.K, p.K == 7 ? 0x1500u : 0x0500u, LLMEM_V(p.os_hh), LLMEM_V(p.os_hf), 0);
 #undef LLMEM_V
+  // where each run starts inside its group
+  d.run[1].start = 2;
+  for (int r = kDynFirst + 1; r <= kDynLast; ++r) d.run[r].start = d.run[r - 1].start + d.run[r - 1].cnt;
+  for (int r = kOsFirst + 1; r <= kOsLast; ++r) d.run[r].start = d.run[r - 1].start + d.run[r - 1].cnt;
+  // which run follows each run: in the first iteration the optimizer states follow the frees
+  for (int r = 0; r < kRuns; ++r) {
+    i64 links = 0;
+    for (int later = 0; later < 2; ++later) {
+      int nx = r;
+      for (int guard = 0; guard < 2 * kRuns; ++guard) {
+        if (nx == kDynLast) nx = later ? kDynFirst : kOsFirst;
+        else if (nx == kOsLast) nx = kDynFirst;
+        else ++nx;
+        if (d.run[nx].cnt > 0) break;
+      }
+      links |= (i64)nx << (8 * later);
+    }
+    d.run[r].links = links;
+  }
   d.init_n = 2u + 2u * (u32)C;
   const u32 allocs = (u32)(G * (1 + C) + p.e_n + L * n_ops + 3 + T * L);
   d.dyn_n = 2 * allocs;

@@ -151,6 +151,46 @@ struct SegmentFolder {
     seg_has = true;
   }
 
+  // The same for spans of any length: `ix` is relative to t0, and a lane that holds no
+  // events passes has == false (and sum 0).
+  __device__ __forceinline__ void add_lane_folds(i64 sum, i64 mx, int ix, bool has, i64 t0, int lane) {
+    i64 inc = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const i64 o = __shfl_up_sync(0xffffffffu, inc, d);
+      if (lane >= d) inc += o;
+    }
+    if (has) {
+      const i64 cand = base + (inc - sum) + mx;
+      if (!lane_has || cand > best_v) {
+        best_v = cand;
+        best_i = t0 + ix;
+        lane_has = true;
+      }
+    }
+    base += __shfl_sync(0xffffffffu, inc, 31);
+    if (__any_sync(0xffffffffu, has)) seg_has = true;
+  }
+
+  // A piece whose fold lane `src` holds: joins through lane 0's candidate.
+  __device__ __forceinline__ void add_from_lane(const Agg& g, int src, int lane) {
+    const i64 g_sum = __shfl_sync(0xffffffffu, g.sum, src);
+    const i64 g_mx = __shfl_sync(0xffffffffu, g.mx, src);
+    const i64 g_idx = __shfl_sync(0xffffffffu, g.idx, src);
+    const bool g_valid = __shfl_sync(0xffffffffu, (int)g.valid, src) != 0;
+    if (!g_valid) return;
+    if (lane == 0) {
+      const i64 cand = base + g_mx;
+      if (!lane_has || cand > best_v) {
+        best_v = cand;
+        best_i = g_idx;
+        lane_has = true;
+      }
+    }
+    base += g_sum;
+    seg_has = true;
+  }
+
   // A piece already folded by the warp (result in lane 0): joins through lane 0's candidate.
   __device__ __forceinline__ void add_piece(const Agg& g, int lane) {
     const i64 g_sum = __shfl_sync(0xffffffffu, g.sum, 0);
