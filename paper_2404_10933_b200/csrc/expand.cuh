@@ -64,7 +64,8 @@ struct alignas(16) Run {
 // follow the first iteration only.  Neighbouring events of equal size share a run, and the
 // logits and their two copies form one run of period 3, so that a list has few runs.
 struct SegDesc {
-  i64 gstart, gend;  // global event range of the segment
+  i64 first_part;  // where the parts of a long segment start in the list of parts (-1: not cut into parts)
+  i64 reserved;
   u32 init_n, dyn_n, os_n;
   int invalid;
   Run run[kRuns];
@@ -94,8 +95,8 @@ __device__ __forceinline__ u32 layer_code(bool gated, bool reversed, int* n_ops)
 // else in a long kernel, already miss the instruction cache more than anything else
 // ("no instruction" is the top stall on lists of short segments).
 static __device__ __noinline__ void build_desc(SegDesc& d, const llmem_config* __restrict__ cfg, i64 gstart, i64 gend, bool round) {
-  d.gstart = gstart;
-  d.gend = gend;
+  d.first_part = -1;
+  d.reserved = 0;
   d.invalid = 1;
   d.init_n = d.dyn_n = d.os_n = 0;
   if (gend <= gstart) return;

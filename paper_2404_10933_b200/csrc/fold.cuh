@@ -279,12 +279,28 @@ __device__ __forceinline__ Fold3 fold_lane_span(const i64* __restrict__ span) {
   return fold3(fold3(f0, f1), fold3(f2, f3));
 }
 
+// What a warp reports for one part of a long segment that several warps write (fused.cu): the
+// largest prefix sum inside the part, counted from the segment's start, and its position.
+struct PartResult {
+  i64 mx, idx;
+  i64 has, pad;
+};
+
+// Segments cut into parts, for the finishing pass: segment i has more than `lane_max` events,
+// its parts of `part` events each report to results[first_part[i] ...].
+struct PartsOfSegments {
+  const i64* first_part = nullptr;  // one entry per segment, stride `stride` bytes; null: no segment is cut
+  size_t stride = 0;
+  const PartResult* results = nullptr;
+  i64 lane_max = 0, part = 1;
+};
+
 // Host launcher of the finishing pass (defined with the scan kernels): one thread per
 // segment folds the partials of segments that cross the warps' blocks (block j starts at
-// bounds[j], bounds[n_warps] = end), defines empty segments, adds m_base + lm_p and marks
-// inadmissible configurations.
+// bounds[j], bounds[n_warps] = end), joins the parts of segments written in parts, defines
+// empty segments, adds m_base + lm_p and marks inadmissible configurations.
 llmem_status launch_scan_finish(const i64* offsets, i64 n, int shift, const llmem_config* cfg, i64* peak_out,
                                 i64* index_out, const i64* bounds, i64 n_warps, const WarpPartials* partials,
-                                cudaStream_t stream);
+                                cudaStream_t stream, PartsOfSegments parts = PartsOfSegments());
 
 }  // namespace llmem

@@ -292,13 +292,27 @@ __device__ __forceinline__ i64 owner_of(const i64* __restrict__ bounds, i64 n_wa
 __global__ void __launch_bounds__(256)
 scan_finish_kernel(const i64* __restrict__ offsets, i64 n, int shift, const llmem_config* __restrict__ cfg,
                    i64* __restrict__ peak_out, i64* __restrict__ index_out, const i64* __restrict__ bounds,
-                   i64 n_warps, const WarpPartials* __restrict__ partials) {
+                   i64 n_warps, const WarpPartials* __restrict__ partials, PartsOfSegments parts) {
   for (i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (i64)gridDim.x * blockDim.x) {
     const i64 a = offsets[i] + shift, b = offsets[i + 1] + shift;
     i64 mx = 0, idx = -1;
     if (b > a) {
       const i64 ca = owner_of(bounds, n_warps, a), cb = owner_of(bounds, n_warps, b - 1);
-      if (ca == cb) {  // finished by the warp that owns it
+      const i64 n_parts = parts.first_part != nullptr && b - a > parts.lane_max ? (b - a + parts.part - 1) / parts.part : 1;
+      if (n_parts > 1) {
+        // written in parts: theirs are prefix sums from the segment's start, so the first of the
+        // largest is the segment's
+        const i64 first = *reinterpret_cast<const i64*>(reinterpret_cast<const unsigned char*>(parts.first_part) + (size_t)i * parts.stride);
+        bool has = false;
+        for (i64 j = 0; j < n_parts && first >= 0; ++j) {
+          const PartResult r = parts.results[first + j];
+          if (r.has && (!has || r.mx > mx)) {
+            mx = r.mx;
+            idx = r.idx - a;
+            has = true;
+          }
+        }
+      } else if (ca == cb) {  // finished by the warp that owns it
         mx = peak_out[i];
         if (index_out) idx = index_out[i];
       } else {
@@ -317,13 +331,13 @@ scan_finish_kernel(const i64* __restrict__ offsets, i64 n, int shift, const llme
 
 llmem_status launch_scan_finish(const i64* offsets, i64 n, int shift, const llmem_config* cfg, i64* peak_out,
                                 i64* index_out, const i64* bounds, i64 n_warps, const WarpPartials* partials,
-                                cudaStream_t stream) {
+                                cudaStream_t stream, PartsOfSegments parts) {
   i64 blocks = (n + 255) / 256;
   const i64 cap = (i64)sm_count() * 8;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   scan_finish_kernel<<<(unsigned)blocks, 256, 0, stream>>>(offsets, n, shift, cfg, peak_out, index_out, bounds,
-                                                          n_warps < 1 ? 1 : n_warps, partials);
+                                                          n_warps < 1 ? 1 : n_warps, partials, parts);
   return check_launch("llmem_scan_peak (finish)");
 }
 

@@ -28,46 +28,40 @@ struct TableRun {
   u32 links;
 };
 
-__device__ __forceinline__ int4 load_run_head(const SegDesc* __restrict__ d, int r) {
-  return __ldg(reinterpret_cast<const int4*>(&d->run[r]));
+// (plain loads: a descriptor may sit in the table in device memory or in a copy of it in
+// shared memory)
+__device__ __forceinline__ int4 load_run_head(const SegDesc* d, int r) {
+  return *reinterpret_cast<const int4*>(&d->run[r]);
 }
 
-__device__ __forceinline__ TableRun load_run(const SegDesc* __restrict__ d, int r) {
+__device__ __forceinline__ TableRun load_run(const SegDesc* d, int r) {
   const int4* p = reinterpret_cast<const int4*>(&d->run[r]);
-  const int4 h = __ldg(p);
-  const longlong2 ab = __ldg(reinterpret_cast<const longlong2*>(p + 1));
-  const longlong2 cl = __ldg(reinterpret_cast<const longlong2*>(p + 2));
+  const int4 h = *p;
+  const longlong2 ab = *reinterpret_cast<const longlong2*>(p + 1);
+  const longlong2 cl = *reinterpret_cast<const longlong2*>(p + 2);
   return TableRun{h.x, h.y, (u32)h.z, h.w, ab.x, ab.y, cl.x, (u32)cl.y};
 }
 
-// Asks for the descriptors of segments [first, first + count) to be brought towards the SM:
-// lane l touches the l-th 128-byte line of that stretch of the table.  A descriptor is read
-// for the first time when its segment begins, and the table of a long list is in device
-// memory by then; without this every segment would begin with a chain of such misses.
-__device__ __forceinline__ void prefetch_descriptors(const SegDesc* __restrict__ table, i64 first, int count, i64 n,
-                                                     int lane) {
-  if (first >= n) return;
-  const i64 last = first + count < n ? first + count : n;
-  const unsigned char* lo = reinterpret_cast<const unsigned char*>(table + first);
-  const unsigned char* hi = reinterpret_cast<const unsigned char*>(table + last);
-  const unsigned char* p = lo + (size_t)lane * 128;
-#ifdef LLMEM_SPANS_PREFETCH_L1
-  if (p < hi) asm volatile("prefetch.global.L1 [%0];\n" ::"l"(p));
-#else
-  if (p < hi) asm volatile("prefetch.global.L2 [%0];\n" ::"l"(p));
-#endif
+// Asks for the whole of one descriptor to be brought into the L2 cache: its records are read
+// one at a time as the walk of the segment reaches them, and the table of a long list is in
+// device memory by then, so without this every run would begin with a miss.
+__device__ __forceinline__ void prefetch_descriptor(const SegDesc* d) {
+  const unsigned char* p = reinterpret_cast<const unsigned char*>(d);
+#pragma unroll
+  for (int k = 0; k < (int)((sizeof(SegDesc) + 127) / 128); ++k) asm volatile("prefetch.global.L2 [%0];\n" ::"l"(p + 128 * k));
+  asm volatile("prefetch.global.L2 [%0];\n" ::"l"(p + sizeof(SegDesc) - 16));
 }
 
 // init_n, dyn_n, os_n, invalid of a descriptor
-__device__ __forceinline__ int4 load_desc_counts(const SegDesc* __restrict__ d) {
-  return __ldg(reinterpret_cast<const int4*>(d) + 1);
+__device__ __forceinline__ int4 load_desc_counts(const SegDesc* d) {
+  return *(reinterpret_cast<const int4*>(d) + 1);
 }
 
 // Run, offset inside it and iteration of event `pos` (0-based inside the segment) of a valid
 // descriptor.  Inside an iteration the run is found by bisection on the runs' start positions
 // (empty runs share their start with the next run, so the last run that starts at or before
 // the position is the non-empty one that holds it).
-__device__ __forceinline__ void locate_in_table(const SegDesc* __restrict__ d, const int4& counts, u32 pos,
+__device__ __forceinline__ void locate_in_table(const SegDesc* d, const int4& counts, u32 pos,
                                                 int* r_out, int* o_out, int* it_out) {
   const u32 init_n = (u32)counts.x, dyn_n = (u32)counts.y, os_n = (u32)counts.z;
   *it_out = 1;
@@ -155,7 +149,7 @@ struct SpanCursor {
   }
 
   // Position the cursor on event `pos` of the segment described by `desc`.
-  __device__ __forceinline__ void seek(const SegDesc* __restrict__ desc, u32 pos, i64 seg_remaining) {
+  __device__ __forceinline__ void seek(const SegDesc* desc, u32 pos, i64 seg_remaining) {
     const int4 counts = load_desc_counts(desc);
     if (counts.w) {
       enter_zeros(seg_remaining);
@@ -169,7 +163,7 @@ struct SpanCursor {
   }
 
   // Position the cursor on the first event of the segment described by `desc`.
-  __device__ __forceinline__ void start(const SegDesc* __restrict__ desc, i64 seg_remaining) {
+  __device__ __forceinline__ void start(const SegDesc* desc, i64 seg_remaining) {
     if (load_desc_counts(desc).w) {
       enter_zeros(seg_remaining);
       return;
@@ -379,6 +373,30 @@ __device__ __forceinline__ void emit_piece_by_warp(i64* __restrict__ buf, int l0
     cur.phase = (int)(ph - (ph / period) * period);
   }
   cur.rem -= m;
+}
+
+// Sum of the next m page-rounded events (1 <= m <= rem) of the cursor's run, which are passed
+// over without being written; the cursor moves as in emit_piece_by_warp.
+template <bool kRoundFold>
+__device__ __forceinline__ i64 skip_piece(int m, SpanCursor& cur) {
+  i64 sum;
+  if (cur.period <= 2) {
+    const bool odd = cur.period == 2 && cur.phase;
+    const i64 y0 = ev<kRoundFold>(odd ? cur.b : cur.a);
+    const i64 y1 = ev<kRoundFold>(cur.period == 2 ? (odd ? cur.a : cur.b) : cur.a);
+    sum = (i64)((m + 1) >> 1) * y0 + (i64)(m >> 1) * y1;
+    if (cur.period == 2) cur.phase ^= (m & 1);
+  } else {
+    const u32 period = (u32)cur.period, phase = (u32)cur.phase;
+    u32 n_b, n_c;
+    count_kinds(cur.code, period, phase, (u32)m, &n_b, &n_c);
+    sum = (i64)((u32)m - n_b - n_c) * ev<kRoundFold>(cur.a) + (i64)n_b * ev<kRoundFold>(cur.b) +
+          (i64)n_c * ev<kRoundFold>(cur.c);
+    const u32 ph = phase + (u32)m;
+    cur.phase = (int)(ph - (ph / period) * period);
+  }
+  cur.rem -= m;
+  return sum;
 }
 
 }  // namespace llmem
