@@ -158,6 +158,21 @@ llmem_status llmem_event_counts_static(const llmem_config* DEV cfg, int64_t n,
                                        int64_t* DEV offsets_out, uint8_t* DEV status_out,
                                        uint32_t flags, void* cuda_stream);
 
+/* No counterpart in the paper: support for grids whose event lists do not fit in device
+ * memory at once (Section 4.2's shapes times every batch, method and degree give lists of
+ * hundreds of gigabytes).  Cuts configurations [first, n) into contiguous slabs of at most
+ * max_events events each, greedily (every slab takes as many configurations as fit; a
+ * configuration with more events than max_events is a slab of its own), so that each slab can
+ * be expanded and scanned through one reusable list buffer.
+ *   offsets     DEV [n+1]  as written by llmem_event_counts
+ *   bounds_out  DEV [max_slabs+1]  slab k holds configurations bounds_out[k] .. bounds_out[k+1]-1;
+ *                          bounds_out[0] = first, the last one written is n
+ *   events_out  DEV [max_slabs+1]  offsets[bounds_out[k]]: slab k has events_out[k+1] - events_out[k] events
+ *   count_out   DEV [1]    number of slabs, or -1 if max_slabs slabs do not reach n */
+llmem_status llmem_slab_bounds(const int64_t* DEV offsets, int64_t n, int64_t max_events, int64_t first,
+                               int64_t* DEV bounds_out, int64_t* DEV events_out, int64_t max_slabs,
+                               int64_t* DEV count_out, void* cuda_stream);
+
 /* Sections 4.1 and 5: the signed byte count of every event, allocations
  * positive and frees negative, configuration i occupying
  * delta_out[offsets[i] .. offsets[i+1]).  Order: initialisation (embedding unit,

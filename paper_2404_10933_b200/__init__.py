@@ -38,7 +38,7 @@ EXPORTS = (
     "llmem_round_events", "llmem_scan_peak", "llmem_max_batch", "llmem_select_method",
     "llmem_scratch_status", "llmem_last_error", "llmem_version", "llmem_event_counts_static",
     "llmem_select_segmented", "llmem_expand_scan", "llmem_chunk_search",
-    "llmem_selftest_wait_limit", "llmem_selftest_int_rate", "llmem_checked_build",
+    "llmem_selftest_wait_limit", "llmem_selftest_int_rate", "llmem_checked_build", "llmem_slab_bounds",
 )
 STATIC_MAX_CONFIGS = 4194304
 
@@ -85,6 +85,7 @@ def lib() -> ctypes.CDLL:
         L.llmem_chunk_search.argtypes = [vp, i64, i64, i64, i32, vp, vp, vp, vp, sz, u32, vp]
         L.llmem_expand_scan.argtypes = [vp, i64, vp, i64, vp, vp, vp, vp, sz, u32, vp]
         L.llmem_select_segmented.argtypes = [vp, vp, vp, i64, i64, i32, vp, vp, vp, vp, sz, u32, vp]
+        L.llmem_slab_bounds.argtypes = [vp, i64, i64, i64, vp, vp, i64, vp, vp]
         L.llmem_selftest_wait_limit.argtypes = [vp, sz, u32, vp]
         L.llmem_selftest_int_rate.argtypes = [ctypes.c_int, u32, vp, ctypes.POINTER(i64), vp]
         L.llmem_scratch_status.argtypes = [vp, vp]
@@ -253,9 +254,10 @@ def scan_peak(delta, offsets, cfg=None, *, fuse_round: bool = False, want_index:
 
 
 def expand_scan(cfg, offsets, total_events: Optional[int] = None, *, fuse_round: bool = True, out=None,
-                want_index: bool = True, scratch=None, stream=None):
+                want_index: bool = True, scratch=None, stream=None, peak_out=None, index_out=None):
     """Materialise the event list and compute the peaks in one pass (the list is written
-    once and not read back).  Returns dict(delta, peak[n], index[n] | None, scratch)."""
+    once and not read back).  ``peak_out`` / ``index_out`` ([n] int64) receive the results when
+    given.  Returns dict(delta, peak[n], index[n] | None, scratch)."""
     torch = _torch()
     cfg = _as_cfg(cfg)
     n = cfg.shape[0]
@@ -266,8 +268,13 @@ def expand_scan(cfg, offsets, total_events: Optional[int] = None, *, fuse_round:
         out = torch.empty(total_events, dtype=torch.int64, device=cfg.device)
     else:
         _check_buffer(out, "out", torch.int64, total_events, cfg.device)
-    peak = torch.empty(n, dtype=torch.int64, device=cfg.device)
-    index = torch.empty(n, dtype=torch.int64, device=cfg.device) if want_index else None
+    if peak_out is not None:
+        _check_buffer(peak_out, "peak_out", torch.int64, n, cfg.device)
+    if index_out is not None:
+        _check_buffer(index_out, "index_out", torch.int64, n, cfg.device)
+    peak = peak_out if peak_out is not None else torch.empty(n, dtype=torch.int64, device=cfg.device)
+    index = index_out if index_out is not None else (
+        torch.empty(n, dtype=torch.int64, device=cfg.device) if want_index else None)
     if scratch is None:
         scratch, nbytes = _scratch(OP_EXPAND_SCAN, n, total_events, cfg.device)
     else:
@@ -379,10 +386,29 @@ def estimate_materialized(cfg, *, fuse_round: bool = True, stream=None):
             "total_events": total}
 
 
+def slab_bounds(offsets, max_events: int, first_config: int = 0, *, max_slabs: int = 4096, stream=None):
+    """Cut configurations [first_config, n) into contiguous slabs of at most ``max_events``
+    events (``llmem_slab_bounds``; the cut runs on the device, only the few boundaries come
+    back).  Returns (bounds, events): numpy int64 arrays, slab k = configurations
+    bounds[k] .. bounds[k+1]-1 with events[k+1] - events[k] events."""
+    torch = _torch()
+    _check_buffer(offsets, "offsets", torch.int64, 1, offsets.device)
+    n = offsets.numel() - 1
+    out = torch.empty(2 * (max_slabs + 1) + 1, dtype=torch.int64, device=offsets.device)
+    bounds, events, count = out[:max_slabs + 1], out[max_slabs + 1:2 * (max_slabs + 1)], out[-1:]
+    _check(lib().llmem_slab_bounds(_ptr(offsets), n, max_events, first_config, _ptr(bounds), _ptr(events), max_slabs,
+                                   _ptr(count), _stream_ptr(stream)))
+    host = out.cpu().numpy()
+    k = int(host[-1])
+    if k < 0:
+        raise ValueError(f"more than {max_slabs} slabs of {max_events} events: raise max_slabs or max_events")
+    return host[:k + 1].copy(), host[max_slabs + 1:max_slabs + 2 + k].copy()
+
+
 def estimate_in_slabs(cfg, max_events: int, *, first_config: int = 0, on_slab=None, stream=None):
     """The materialised path for grids whose event lists do not fit in device memory at
     once: the configurations are cut into contiguous slabs of at most ``max_events`` events
-    (``grids.slab_bounds``), and every slab is expanded, page-rounded and scanned by
+    (``llmem_slab_bounds``), and every slab is expanded, page-rounded and scanned by
     ``llmem_expand_scan`` through one list buffer and one scratch buffer that are reused.
     ``first_config`` restarts an interrupted run at a slab boundary (earlier results are then
     left at -1).  ``on_slab(lo, hi, delta, offsets)`` is called after each slab with its
@@ -392,9 +418,8 @@ def estimate_in_slabs(cfg, max_events: int, *, first_config: int = 0, on_slab=No
     cfg = _as_cfg(cfg)
     n = cfg.shape[0]
     offsets, status = event_counts(cfg, stream=stream)
-    bounds = grids.slab_bounds(offsets.cpu().numpy(), max_events, first_config)
-    off_host = offsets.cpu().numpy()
-    sizes = off_host[bounds[1:]] - off_host[bounds[:-1]]
+    bounds, events = slab_bounds(offsets, max_events, first_config, stream=stream)
+    sizes = np.diff(events)
     capacity = int(sizes.max()) if len(sizes) else 0
     delta = torch.empty(max(capacity, 1), dtype=torch.int64, device=cfg.device)
     nbytes = max([scratch_bytes(OP_EXPAND_SCAN, int(hi - lo), int(t))
@@ -405,9 +430,8 @@ def estimate_in_slabs(cfg, max_events: int, *, first_config: int = 0, on_slab=No
     for lo, hi, total in zip(bounds[:-1].tolist(), bounds[1:].tolist(), sizes.tolist()):
         part = cfg[lo:hi]
         local, _ = event_counts(part, want_status=False, stream=stream)
-        r = expand_scan(part, local, int(total), fuse_round=True, out=delta, scratch=scratch, stream=stream)
-        peak[lo:hi] = r["peak"]
-        index[lo:hi] = r["index"]
+        r = expand_scan(part, local, int(total), fuse_round=True, out=delta, scratch=scratch, stream=stream,
+                        peak_out=peak[lo:hi], index_out=index[lo:hi])
         if on_slab is not None:
             on_slab(lo, hi, r["delta"], local)
     return {"peak": peak, "index": index, "status": status, "bounds": bounds}

@@ -118,6 +118,37 @@ add_block_base_kernel(i64* __restrict__ offsets, i64 n, const u64* __restrict__ 
 }
 
 // ---------------------------------------------------------------------------
+// slabs: cutting a grid whose lists do not fit the device at once
+// ---------------------------------------------------------------------------
+// One warp cuts configurations [first, n) into contiguous slabs of at most max_events events,
+// greedily: every slab takes as many configurations as fit; one with more events than that is
+// a slab of its own.  The end of a slab is found by the warp's 32-ary search on the offsets.
+__global__ void __launch_bounds__(32)
+slab_bounds_kernel(const i64* __restrict__ offsets, i64 n, i64 max_events, i64 first, i64* __restrict__ bounds_out,
+                   i64* __restrict__ events_out, i64 max_slabs, i64* __restrict__ count_out) {
+  const int lane = threadIdx.x;
+  i64 a = first, slabs = 0;
+  if (lane == 0) {
+    bounds_out[0] = first;
+    events_out[0] = __ldg(offsets + first);
+  }
+  while (a < n && slabs < max_slabs) {
+    // smallest s with offsets[s + 1] > offsets[a] + max_events: configurations a .. s-1 fit
+    const i64 target = __ldg(offsets + a) + max_events;
+    i64 b = warp_search_cost(offsets, n, 0, target, lane);
+    if (b < a + 1) b = a + 1;
+    if (b > n) b = n;
+    ++slabs;
+    if (lane == 0) {
+      bounds_out[slabs] = b;
+      events_out[slabs] = __ldg(offsets + b);
+    }
+    a = b;
+  }
+  if (lane == 0) *count_out = a < n ? -1 : slabs;
+}
+
+// ---------------------------------------------------------------------------
 // expansion (run tables, cursor and store primitives: expand.cuh)
 // ---------------------------------------------------------------------------
 // The list is cut into n_blocks contiguous blocks of equal cost (events + kappa per segment,
@@ -352,6 +383,26 @@ extern "C" llmem_status llmem_event_counts_static(const llmem_config* cfg, int64
   if (blocks3 > cap3) blocks3 = cap3;
   add_block_base_kernel<<<(unsigned)blocks3, 256, 0, s>>>(reinterpret_cast<i64*>(offsets_out), n, block_sums, nblocks);
   return check_launch("llmem_event_counts_static");
+}
+
+extern "C" llmem_status llmem_slab_bounds(const int64_t* offsets, int64_t n, int64_t max_events, int64_t first,
+                                          int64_t* bounds_out, int64_t* events_out, int64_t max_slabs,
+                                          int64_t* count_out, void* cuda_stream) {
+  clear_error();
+  TraceRange trace("llmem_slab_bounds");
+  if (n < 0 || max_events < 1 || first < 0 || first > n || max_slabs < 1) {
+    set_error("llmem_slab_bounds: n >= 0, max_events >= 1, 0 <= first <= n and max_slabs >= 1 are required");
+    return LLMEM_ERR_ARG;
+  }
+  if (!offsets || !bounds_out || !events_out || !count_out || !aligned_to(offsets, 8) || !aligned_to(bounds_out, 8) ||
+      !aligned_to(events_out, 8) || !aligned_to(count_out, 8)) {
+    set_error("llmem_slab_bounds: offsets, bounds_out, events_out and count_out must be 8-byte aligned device pointers");
+    return LLMEM_ERR_ARG;
+  }
+  slab_bounds_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      reinterpret_cast<const i64*>(offsets), n, max_events, first, reinterpret_cast<i64*>(bounds_out),
+      reinterpret_cast<i64*>(events_out), max_slabs, reinterpret_cast<i64*>(count_out));
+  return check_launch("llmem_slab_bounds");
 }
 
 extern "C" llmem_status llmem_expand_events(const llmem_config* cfg, int64_t n, const int64_t* offsets,

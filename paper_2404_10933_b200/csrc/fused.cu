@@ -83,10 +83,21 @@ desc_table_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __rest
     build_desc(stage[threadIdx.x], cfg + i, lo, hi, round != 0);
     count = hi - lo;
   }
-  if (part_list != nullptr && count > kOwnedLaneMax) {
-    const i64 parts = (count + kOwnedPart - 1) / kOwnedPart;
-    const i64 slot = (i64)atomicAdd(part_count, (unsigned long long)parts);
-    if (slot + parts <= part_capacity) {  // always, by the size of the scratch
+  // the parts of the longer segments: one addition to the counter per warp
+  const int lane = threadIdx.x & 31;
+  const i64 parts = part_list != nullptr && count > kOwnedLaneMax ? (count + kOwnedPart - 1) / kOwnedPart : 0;
+  i64 before = parts;  // parts of this and the lower lanes
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const i64 o = __shfl_up_sync(0xffffffffu, before, d);
+    if (lane >= d) before += o;
+  }
+  const i64 in_warp = __shfl_sync(0xffffffffu, before, 31);
+  if (in_warp > 0) {
+    unsigned long long slot0 = 0;
+    if (lane == 0) slot0 = atomicAdd(part_count, (unsigned long long)in_warp);
+    const i64 slot = (i64)__shfl_sync(0xffffffffu, slot0, 0) + before - parts;
+    if (parts > 0 && slot + parts <= part_capacity) {  // always, by the size of the scratch
       for (i64 k = 0; k < parts; ++k) part_list[slot + k] = (i << 20) | k;
       stage[threadIdx.x].first_part = slot;
     }

@@ -481,6 +481,26 @@ def test_materialised_path_in_slabs(llmem):
     assert np.array_equal(again["index"].cpu().numpy()[k:], want["index"][k:])
 
 
+def test_slab_bounds_on_device_equal_the_host_cut(llmem):
+    """llmem_slab_bounds against the greedy cut written out on the host, for budgets from one
+    event (every configuration a slab of its own) to more than the whole grid, restarts, empty
+    segments, and the refusal when the slabs do not fit the output."""
+    cfgs = mixed_small_grid()
+    offsets, _ = llmem.event_counts(cfgs)
+    off = offsets.cpu().numpy()
+    n = len(cfgs)
+    for budget in (1, 300, 5000, 40_000, int(off[-1]), int(off[-1]) * 3):
+        for first in (0, 7, n - 1, n):
+            b, ev = llmem.slab_bounds(offsets, budget, first)
+            assert np.array_equal(b, grids.slab_bounds(off, budget, first))
+            assert np.array_equal(ev, off[b])
+    with pytest.raises(ValueError, match="slabs"):
+        llmem.slab_bounds(offsets, 1, 0, max_slabs=16)
+    L = llmem.lib()
+    assert L.llmem_slab_bounds(offsets.data_ptr(), n, 0, 0, offsets.data_ptr(), offsets.data_ptr(), 4,
+                               offsets.data_ptr(), None) == llmem.ERR_ARG
+
+
 CHECKED_SCRIPT = r"""
 import numpy as np, torch
 import oracle
