@@ -21,7 +21,13 @@ block reports the dominant kernel against the measured HBM copy bandwidth.
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
 Under torchrun every rank runs the same work on its own seeded grid (no exchange
-step exists in this method); times are the maximum over ranks.
+step exists in this method); times are the maximum over ranks.  With --scaling strong the
+ranks share one grid instead: contiguous shards balanced by event count, results gathered
+over NCCL and checked against the fused estimate of the whole grid.
+
+At one GPU the default run adds three short legs under "secondary": the fused estimate of
+the large sweep, the max-batch search with Algorithm 1 selection, and the whole shape grid
+through the materialised path in slabs, each with its own roofline entry.
 """
 from __future__ import annotations
 
@@ -48,7 +54,7 @@ FALLBACK_HBM_GBS = 6650.0
 # HBM-bound kernels, from an ncu capture of a 4096-configuration run (summary kept under
 # profiles/; traffic grows in proportion to the number of events).  Set an entry
 # to None when its kernel changes after the capture.
-NCU_TRAFFIC_BYTES_PER_EVENT = {"expand": 7.8238, "scan": 8.0130, "expand_scan": 7.8256}
+NCU_TRAFFIC_BYTES_PER_EVENT = {"expand": None, "scan": None, "expand_scan": None}
 
 
 def measured_peaks():
@@ -142,7 +148,7 @@ def time_oracle(cfgs, threads: int):
     return int(r["count"].sum()), dt
 
 
-def cpu_baseline(sample_configs: int = 49152):
+def cpu_baseline(sample_configs: int = grids.G5_CONFIGS):
     cores = os.cpu_count() or 1
     events, dt = time_oracle(oracle_sample(sample_configs), cores)
     one_n = max(1, sample_configs // 32)
@@ -151,7 +157,7 @@ def cpu_baseline(sample_configs: int = 49152):
             "configs_per_sec": sample_configs / dt,
             "single_thread": {"value": one_events / one_dt, "unit": UNIT, "cores": 1,
                               "sample": f"first {one_n} configurations, {one_dt:.2f} s"},
-            "sample": f"first {sample_configs} of the 65536 stress-grid configurations "
+            "sample": f"all {sample_configs} stress-grid configurations "
                       f"({events} events), level-1 oracle (explicit list, round, scan) + its bisecting search and selection, "
                       f"{cores} threads, {dt:.2f} s"}
 
@@ -377,8 +383,20 @@ def run_ours(args):
         return multi.reduce_scalar(x, "sum", device="cuda")
 
     n_cfg = args.configs
-    cfgs = grids.g5_stress(0, n_cfg, seed_offset=rank)     # weak scaling: one full grid per rank
     caps = grids.g4_capacities()
+    strong = args.scaling == "strong"
+    shard_lo, whole = 0, None
+    if strong:
+        # one grid for all ranks: contiguous shards balanced by event count (the counts come from
+        # llmem_event_counts on this rank's device; every rank computes the same cut)
+        whole = grids.g5_stress(0, n_cfg)
+        whole_offsets, _ = llmem.event_counts(whole)
+        counts = torch.diff(whole_offsets).cpu().numpy()
+        shard_lo, shard_hi = multi.shard_of(n_cfg, counts, rank, world)
+        cfgs = whole[shard_lo:shard_hi]
+        del whole_offsets
+    else:
+        cfgs = grids.g5_stress(0, n_cfg, seed_offset=rank)     # weak scaling: one full grid per rank
     hp = HotPath(llmem, torch, cfgs, caps, grids.G4_BMAX, one_pass=not args.two_pass)
 
     # ---- device-resident timing ----
@@ -416,6 +434,19 @@ def run_ours(args):
     # the two paths must agree on the device (cheap self-check outside the timed region)
     fused = llmem.estimate_batch(hp.cfg, want_status=False)
     agree = bool(torch.equal(fused["peak"], out["peak"]) and torch.equal(fused["index"], out["index"]))
+    gathered_ok = None
+    if strong:
+        # the shards' results, gathered over the process group, against the fused estimate of the
+        # whole grid computed on rank 0
+        everything = {k: multi.gather_slices(out[k], n_cfg, shard_lo, device="cuda") for k in ("peak", "index", "method", "batch")}
+        if rank == 0:
+            ref = llmem.estimate_batch(whole, want_status=False)
+            ref_sel = llmem.select_method(whole, caps, grids.G4_BMAX, want_bs_list=False, want_status=False)
+            gathered_ok = bool(torch.equal(everything["peak"], ref["peak"]) and torch.equal(everything["index"], ref["index"]) and
+                               torch.equal(everything["method"], ref_sel["method"]) and
+                               torch.equal(everything["batch"], ref_sel["batch"]))
+            del ref, ref_sel
+        del everything
 
     # ---- end to end from host buffers ----
     hp.run_e2e(min(args.warmup, 3))
@@ -462,6 +493,8 @@ def run_ours(args):
                                        "after it on the same grid (5 launches each)",
                                **{k: entry(v) for k, v in others.items()}},
         "frac_of_nominal_8000": achieved / 8000.0,
+        "note": "the measured peak is a copy (read + write); a stream that only writes, or only reads, can exceed it: "
+                "above 1 the fraction of the nominal 8 TB/s is the one to read",
     }
     step_text = ("event_counts + expand_scan (expansion, page rounding and segmented scan in one kernel, list "
                  "written to HBM once) + max_batch + select_method" if hp.one_pass else
@@ -470,136 +503,175 @@ def run_ours(args):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+        "scaling": args.scaling, "vs_baseline": None, "dtype": "int64", "data": "synthetic",
         "configs_per_sec": configs_all * args.steps / (ms * 1e-3),
         "config": {"workload": "G5 stress grid: deep/wide decoders, materialised int64 event lists",
                    "configs_per_gpu": hp.n, "events_per_gpu": hp.total, "capacities": len(caps),
-                   "bmax": grids.G4_BMAX, "parallelism": f"replicas x{world} (independent configs, no collective)",
+                   "bmax": grids.G4_BMAX,
+                   "parallelism": (f"one grid cut into {world} contiguous shards balanced by event count; results "
+                                   "gathered over NCCL outside the timed region" if strong else
+                                   f"replicas x{world} (independent configs, no collective)"),
                    "l2": "event list (8 B/event) far larger than the 126 MB L2; no flush needed",
                    "path": "one-pass" if hp.one_pass else "two-pass", "step": step_text},
         "roofline": roofline,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": hp.h2d_bytes,
-                "d2h_bytes_per_step": hp.d2h_bytes, "ms_per_step": e2e_ms / e2e_steps},
+                "d2h_bytes_per_step": hp.d2h_bytes, "ms_per_step": e2e_ms / e2e_steps,
+                "inputs": "configuration records and capacities from pinned host memory, every step",
+                "outputs": "peak[n] int64, method[n, capacities] and batch[n, capacities] int32 to pinned host memory, "
+                           "and the event total the host needs to size the list; peak positions, per-method "
+                           "batches and status stay on the device"},
         "gpu_launches": hp.kernels_per_step * args.steps,
         "clocks": clocks,
         "fused_equals_materialised": agree, "e2e_equals_resident": e2e_agree,
     }
+    if strong:
+        line["gathered_equals_whole_grid"] = gathered_ok
+    if world == 1 and args.secondary:
+        # the other grids, shortly, with their own rooflines (device memory of the headline is released first)
+        del hp, out, fused
+        torch.cuda.empty_cache()
+        line["secondary"] = {
+            "g3": leg_estimate(llmem, torch, max(20, min(args.steps, 200)), args.warmup),
+            "g4": leg_search(llmem, torch, max(5, min(args.steps, 20)), args.warmup),
+            "g2": leg_slabs(llmem, torch, max(3, min(args.steps, 5)), args.warmup),
+        }
     if args.cpu_baseline:
         line["cpu_baseline"] = cpu_baseline()
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
-    return 0 if (agree and e2e_agree) else 4
+    ok = agree and e2e_agree and gathered_ok is not False
+    if "secondary" in line:
+        ok = ok and line["secondary"]["g2"]["fused_equals_materialised"] and line["secondary"]["g4"]["selection_equals_search"]
+    return 0 if ok else 4
 
 
 # ---------------------------------------------------------------------------
 # secondary workloads: the kernels that generate events in registers (integer-ALU bound)
+# and the shape grid through the materialised path in slabs
 # ---------------------------------------------------------------------------
-# Warp instructions executed per unit of work (smsp__inst_executed.sum / units) from ncu
-# captures of these kernels on reduced grids; None once a kernel changes after the capture.
-NCU_WARP_INSTR_PER_UNIT = {"estimate_kernel": 30.88, "max_batch_kernel": 11.40, "select_kernel": 65.03}
+# Lane instructions executed per unit of work, as warp instructions with all 32 lanes busy
+# (ncu smsp__thread_inst_executed.sum / 32 / units), from captures of these kernels on reduced
+# grids (profiles/register_kernels_g3_g4_ncu.md); None once a kernel changes after the capture.
+# Counting lane instructions keeps divergence from passing for throughput: a warp instruction
+# issued for 20 of 32 lanes counts as 20/32.
+NCU_LANE_INSTR_PER_UNIT = {"estimate_kernel": None, "max_batch_kernel": None, "select_kernel": None}
 
 
-def run_register_paths(args):
-    """--workload g3: fused estimate over the 2^20-configuration sweep.
-    --workload g4: largest-batch search (2^17 shapes x 4 methods x 16 degrees x 9 capacities)
-    and Algorithm 1 selection (2^17 shapes x 16 degrees x 9 capacities).
-    Inputs are resident in HBM; L2 is flushed between timed steps (the g3 input is smaller
-    than L2).  Reports units/s and the issue-rate (integer ALU) roofline."""
-    import torch
-    import paper_2404_10933_b200 as llmem
-    llmem.lib()
-    torch.cuda.set_device(0)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    caps_np = grids.g4_capacities()
-    caps = torch.from_numpy(caps_np).cuda()
-    if args.workload == "g3":
-        n = min(args.configs, grids.G3_CONFIGS) if args.configs != grids.G5_CONFIGS else grids.G3_CONFIGS
-        host = [grids.g3_sweep(0, n)]
-        dev = [llmem.to_device(host[0])]
-        events = int(torch.diff(llmem.event_counts(dev[0])[0]).sum().item())
-        units = {"estimate_kernel": n}
-
-        def step():
-            return llmem.estimate_batch(dev[0])
-        unit_name, n_units, extra = "configs/s", n, {"virtual_events_per_config": events / n}
-        workload = "G3 large sweep: fused estimate, event runs summed in registers (no list materialised)"
-        launches = 1
-    else:
-        shapes = min(args.configs, grids.G4_SHAPES) if args.configs != grids.G5_CONFIGS else grids.G4_SHAPES
-        host = [grids.g4_search_grid(0, shapes), grids.g4_select_grid(0, shapes)]
-        dev = [llmem.to_device(h) for h in host]
-        units = {"max_batch_kernel": len(host[0]) * len(caps_np), "select_kernel": len(host[1]) * len(caps_np)}
-
-        def step():
-            a = llmem.max_batch(dev[0], caps, grids.G4_BMAX, want_status=False)
-            b = llmem.select_method(dev[1], caps, grids.G4_BMAX, want_bs_list=False, want_status=False)
-            return a, b
-        unit_name, n_units, extra = "searches/s", units["max_batch_kernel"] + 4 * units["select_kernel"], {
-            "selections": units["select_kernel"]}
-        workload = "G4 max-batch search + Algorithm 1 selection, bracketed bisection on batch 1..4096 in registers"
-        launches = 2
-    for _ in range(max(args.warmup, 3)):
-        step()
+def _gpu_id(torch):
     try:
-        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(0).uuid)
+        return "GPU-" + str(torch.cuda.get_device_properties(torch.cuda.current_device()).uuid)
     except Exception:
-        gpu_id = "0"
-    sampler = ClockSampler(gpu_id)
+        return str(torch.cuda.current_device())
+
+
+def _timed_steps(torch, step, steps, warmup, flush=None):
+    """Mean device time (ms) of `steps` calls of step(), CUDA events on the current stream, L2
+    flushed before every timed call when `flush` is given; clocks sampled meanwhile."""
+    for _ in range(max(warmup, 3)):
+        step()
+    sampler = ClockSampler(_gpu_id(torch))
     sampler.start()
     time.sleep(0.3)
     torch.cuda.synchronize()
     wall0 = time.time()
     total_ms = 0.0
-    for _ in range(args.steps):
-        flush.fill_(1)
+    for _ in range(steps):
+        if flush is not None:
+            flush.fill_(1)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         step()
         e1.record()
         torch.cuda.synchronize()
         total_ms += e0.elapsed_time(e1)
-    wall1 = time.time()
-    clocks = sampler.stop(wall0, wall1)
-    ms = total_ms / args.steps
-    # issue-rate roofline: 4 schedulers per SM, one warp instruction per cycle each
+    clocks = sampler.stop(wall0, time.time())
+    return total_ms / steps, clocks
+
+
+def _alu_roofline(torch, llmem, units, ms, clocks):
+    """Issue-rate roofline of a per-configuration kernel: achieved = lane instructions of the
+    model (as full warp instructions) per second, peak = SMs x 4 schedulers x sampled clock."""
     sm = torch.cuda.get_device_properties(0).multi_processor_count
     mhz = clocks.get("sm_mhz") or 1965.0
     peak = sm * 4 * mhz * 1e6
-    # the same ceiling measured: independent 32-bit chains (add/xor, multiply-add, alternating)
     probe = {name: llmem.int_rate(kind) for kind, name in enumerate(("add_xor", "mad", "add_mad"))}
     instr = None
-    if all(NCU_WARP_INSTR_PER_UNIT.get(k) is not None for k in units):
-        instr = sum(NCU_WARP_INSTR_PER_UNIT[k] * u for k, u in units.items())
-    line = {
-        "metric": f"{unit_name.split('/')[0]} per second ({args.workload})", "value": n_units / (ms * 1e-3),
-        "unit": unit_name, "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-        "config": {"workload": workload, "l2": "256 MB write between timed steps flushes L2", **extra},
-        "roofline": {"bound": "alu", "unit": "warp-instr/s", "peak": peak,
-                     "achieved": (instr / (ms * 1e-3)) if instr else None,
-                     "frac": (instr / (ms * 1e-3) / peak) if instr else None,
-                     "peak_source": "148 SMs x 4 schedulers x sampled SM clock (one warp instruction per cycle each)",
-                     "measured_issue_rates": probe,
-                     "frac_of_measured_add_mad": (instr / (ms * 1e-3) / probe["add_mad"]) if instr else None,
-                     "traffic": None},
-        "gpu_launches": launches * args.steps, "clocks": clocks,
-    }
-    print(json.dumps(line))
-    return 0
+    if all(NCU_LANE_INSTR_PER_UNIT.get(k) is not None for k in units):
+        instr = sum(NCU_LANE_INSTR_PER_UNIT[k] * u for k, u in units.items())
+    return {"bound": "alu", "unit": "warp-instr/s", "peak": peak,
+            "achieved": (instr / (ms * 1e-3)) if instr else None,
+            "frac": (instr / (ms * 1e-3) / peak) if instr else None,
+            "achieved_is": "lane instructions / 32 (ncu smsp__thread_inst_executed per unit x units / time): "
+                           "idle lanes of a diverged warp do not count",
+            "peak_source": "148 SMs x 4 schedulers x sampled SM clock (one warp instruction per cycle each)",
+            "measured_issue_rates": probe,
+            "frac_of_measured_add_mad": (instr / (ms * 1e-3) / probe["add_mad"]) if instr else None,
+            "traffic": None}
 
 
-def run_slab_path(args):
-    """--workload g2: the whole shape grid (3.8 M configurations, 4.6e10 events, 365 GB as
-    int64) through the materialised path in slabs of 2^32 events sharing one 32 GiB list
-    buffer.  One step = event counts of the grid, then per slab event counts, expansion with
-    fused rounding and segmented scan (llmem_expand_scan), results gathered on the device;
-    the host reads the offsets once per step to cut the slabs."""
-    import torch
-    import paper_2404_10933_b200 as llmem
-    llmem.lib()
-    torch.cuda.set_device(0)
-    shapes = 4096 if args.configs == grids.G5_CONFIGS else max(1, min(args.configs, 4096))
+def leg_estimate(llmem, torch, steps, warmup, n=None, repeat=16):
+    """Fused estimate (no list) of the large sweep; also of the sweep repeated `repeat` times
+    (2^24 configurations), where launch ramp and tail no longer weigh."""
+    n = grids.G3_CONFIGS if n is None else n
+    host = grids.g3_sweep(0, n)
+    dev = llmem.to_device(host)
+    big = dev.repeat(repeat, 1).contiguous()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    events = int(llmem.event_counts(dev)[0][-1].item())
+    ms, clocks = _timed_steps(torch, lambda: llmem.estimate_batch(dev), steps, warmup, flush)
+    ms_big, _ = _timed_steps(torch, lambda: llmem.estimate_batch(big), max(3, steps // 4), warmup, flush)
+    roof = _alu_roofline(torch, llmem, {"estimate_kernel": n}, ms, clocks)
+    roof_big = _alu_roofline(torch, llmem, {"estimate_kernel": n * repeat}, ms_big, clocks)
+    return {"metric": "configs per second (fused estimate)", "value": n / (ms * 1e-3), "unit": "configs/s",
+            "steps": steps, "ms_per_step": ms, "dtype": "int64",
+            "config": {"workload": "G3 large sweep: fused estimate, event runs summed in registers (no list materialised)",
+                       "configs": n, "virtual_events_per_config": events / n,
+                       "l2": "256 MB write between timed steps flushes L2"},
+            "roofline": roof,
+            "repeated": {"configs": n * repeat, "ms_per_step": ms_big, "value": n * repeat / (ms_big * 1e-3),
+                         "unit": "configs/s", "frac": roof_big["frac"],
+                         "frac_of_measured_add_mad": roof_big["frac_of_measured_add_mad"]},
+            "gpu_launches": steps, "clocks": clocks}
+
+
+def leg_search(llmem, torch, steps, warmup, shapes=None):
+    """Largest-batch search (shapes x 4 methods x 16 degrees x 9 capacities) and Algorithm 1
+    selection (shapes x 16 degrees x 9 capacities); the selection's batches are compared with
+    the search's on the device."""
+    shapes = grids.G4_SHAPES if shapes is None else shapes
+    caps_np = grids.g4_capacities()
+    caps = torch.from_numpy(caps_np).cuda()
+    host = [grids.g4_search_grid(0, shapes), grids.g4_select_grid(0, shapes)]
+    dev = [llmem.to_device(h) for h in host]
+    units = {"max_batch_kernel": len(host[0]) * len(caps_np), "select_kernel": len(host[1]) * len(caps_np)}
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def step():
+        a = llmem.max_batch(dev[0], caps, grids.G4_BMAX, want_status=False)
+        b = llmem.select_method(dev[1], caps, grids.G4_BMAX, want_bs_list=True, want_status=False)
+        return a, b
+    (bs, _), sel = step()
+    # the four batches Algorithm 1 compared are those of the search grid, shape by shape
+    bs4 = bs.clamp(min=0).reshape(shapes, 4, grids.G4_DEGREES, len(caps_np)).permute(0, 2, 3, 1).reshape(-1, len(caps_np), 4)
+    agree = bool(torch.equal(sel["bs_list"], bs4))
+    ms, clocks = _timed_steps(torch, step, steps, warmup, flush)
+    n_units = units["max_batch_kernel"] + 4 * units["select_kernel"]
+    return {"metric": "searches per second (max batch + Algorithm 1)", "value": n_units / (ms * 1e-3),
+            "unit": "searches/s", "steps": steps, "ms_per_step": ms, "dtype": "int64",
+            "config": {"workload": "G4 max-batch search + Algorithm 1 selection, bracketed bisection on batch 1..4096 in registers",
+                       "shapes": shapes, "searches": units["max_batch_kernel"], "selections": units["select_kernel"],
+                       "l2": "256 MB write between timed steps flushes L2"},
+            "roofline": _alu_roofline(torch, llmem, units, ms, clocks),
+            "gpu_launches": 2 * steps, "clocks": clocks, "selection_equals_search": agree}
+
+
+def leg_slabs(llmem, torch, steps, warmup, shapes=None):
+    """The whole shape grid (3.8 M configurations, 4.3e10 events, 345 GB as int64) through the
+    materialised path in slabs of 2^32 events sharing one 32 GiB list buffer.  One step = event
+    counts of the grid, slab boundaries cut on the device, then per slab event counts,
+    expansion with fused rounding and segmented scan (llmem_expand_scan)."""
+    shapes = grids.G2_SHAPES if shapes is None else max(1, min(shapes, grids.G2_SHAPES))
     cfgs = grids.g2_shape_grid(0, shapes)
     dev = llmem.to_device(cfgs)
     budget = 1 << 32
@@ -608,43 +680,41 @@ def run_slab_path(args):
     slabs = len(r["bounds"]) - 1
     fused = llmem.estimate_batch(dev)
     agree = bool(torch.equal(fused["peak"], r["peak"]) and torch.equal(fused["index"], r["index"]))
-    for _ in range(max(args.warmup, 3) - 1):
-        llmem.estimate_in_slabs(dev, budget)
-    try:
-        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(0).uuid)
-    except Exception:
-        gpu_id = "0"
-    sampler = ClockSampler(gpu_id)
-    sampler.start()
-    time.sleep(0.3)
-    torch.cuda.synchronize()
-    steps = max(1, min(args.steps, 20))
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    wall0 = time.time()
-    e0.record()
-    for _ in range(steps):
-        llmem.estimate_in_slabs(dev, budget)
-    e1.record()
-    torch.cuda.synchronize()
-    wall1 = time.time()
-    clocks = sampler.stop(wall0, wall1)
-    ms = e0.elapsed_time(e1) / steps
+    del r, fused
+    steps = max(1, min(steps, 20))
+    ms, clocks = _timed_steps(torch, lambda: llmem.estimate_in_slabs(dev, budget), steps, warmup)
     peak_gbs, peak_src = measured_peaks()
     achieved = 8.0 * events / (ms * 1e-3) / 1e9
-    line = {
-        "metric": METRIC, "value": events / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "int64", "data": "synthetic", "configs_per_sec": len(cfgs) / (ms * 1e-3),
-        "config": {"workload": "G2 shape grid, materialised int64 event lists in slabs", "configs": len(cfgs),
-                   "events": events, "slabs": slabs, "events_per_slab_max": budget,
-                   "l2": "every slab's list is far larger than the 126 MB L2"},
-        "roofline": {"bound": "hbm", "kernel": "whole step (expand_scan_kernel per slab + counts + host slab loop)",
-                     "achieved": achieved, "peak": peak_gbs, "unit": "GB/s", "frac": achieved / peak_gbs,
-                     "peak_source": peak_src, "traffic": None},
-        "gpu_launches": steps * (3 + slabs * 6), "clocks": clocks, "fused_equals_materialised": agree,
-    }
+    return {"metric": METRIC, "value": events / (ms * 1e-3), "unit": UNIT, "steps": steps, "ms_per_step": ms,
+            "dtype": "int64", "configs_per_sec": len(cfgs) / (ms * 1e-3),
+            "config": {"workload": "G2 shape grid, materialised int64 event lists in slabs", "configs": len(cfgs),
+                       "events": events, "slabs": slabs, "events_per_slab_max": budget,
+                       "l2": "every slab's list is far larger than the 126 MB L2"},
+            "roofline": {"bound": "hbm", "kernel": "whole step (per slab: counts, descriptor table, expand_scan_owned_kernel, "
+                                                   "finishing pass; host slab loop)",
+                         "achieved": achieved, "peak": peak_gbs, "unit": "GB/s", "frac": achieved / peak_gbs,
+                         "frac_of_nominal_8000": achieved / 8000.0, "peak_source": peak_src, "traffic": None},
+            "gpu_launches": steps * (4 + slabs * 7), "clocks": clocks, "fused_equals_materialised": agree}
+
+
+def run_secondary_workload(args):
+    """--workload g3 | g4 | g2 alone: one JSON line for that leg."""
+    import torch
+    import paper_2404_10933_b200 as llmem
+    llmem.lib()
+    torch.cuda.set_device(0)
+    reduced = args.configs != grids.G5_CONFIGS
+    if args.workload == "g3":
+        leg = leg_estimate(llmem, torch, args.steps, args.warmup, min(args.configs, grids.G3_CONFIGS) if reduced else None)
+    elif args.workload == "g4":
+        leg = leg_search(llmem, torch, args.steps, args.warmup, min(args.configs, grids.G4_SHAPES) if reduced else None)
+    else:
+        leg = leg_slabs(llmem, torch, args.steps, args.warmup, args.configs if reduced else None)
+    line = {"n_gpus": 1, "warmup": max(args.warmup, 3), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "data": "synthetic", **leg}
     print(json.dumps(line))
-    return 0 if agree else 4
+    ok = leg.get("fused_equals_materialised", True) and leg.get("selection_equals_search", True)
+    return 0 if ok else 4
 
 
 def main():
@@ -657,6 +727,10 @@ def main():
     ap.add_argument("--configs", type=int, default=grids.G5_CONFIGS,
                     help="configurations of the stress grid per GPU (default: the full grid)")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--scaling", choices=("weak", "strong"), default="weak",
+                    help="weak (default): every rank its own seeded grid; strong: one grid cut into shards balanced by event count")
+    ap.add_argument("--no-secondary", dest="secondary", action="store_false",
+                    help="skip the short legs on the other grids that a one-GPU run appends under 'secondary'")
     ap.add_argument("--two-pass", action="store_true",
                     help="time llmem_expand_events + llmem_scan_peak as separate kernels instead of llmem_expand_scan")
     ap.add_argument("--workload", choices=("g5", "g3", "g4", "g2"), default="g5",
@@ -665,15 +739,17 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
-    if args.workload == "g2":
-        return run_slab_path(args)
     if args.workload != "g5":
-        return run_register_paths(args)
+        return run_secondary_workload(args)
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if world == 1 and args.gpus > 1:
         # launched without torchrun: re-launch one rank per GPU
+        import socket
+        with socket.socket() as sock:  # a port nobody else on this machine is using right now
+            sock.bind(("127.0.0.1", 0))
+            port = sock.getsockname()[1]
         cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
-               "--master-addr", "127.0.0.1", "--master-port", "29511", os.path.abspath(__file__)] + sys.argv[1:]
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
         return subprocess.call(cmd)
     if int(os.environ.get("RANK", "0")) != 0:
         args.cpu_baseline = False
