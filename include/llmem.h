@@ -99,7 +99,8 @@ enum { LLMEM_OP_ESTIMATE = 0, LLMEM_OP_EVENT_COUNTS = 1, LLMEM_OP_EXPAND = 2, LL
 
 /* Bytes of scratch the operation needs for n configurations and total_events
  * events (0 where it needs none; such calls accept scratch = NULL).  For
- * LLMEM_OP_EXPAND the scratch is optional (see llmem_expand_events). */
+ * LLMEM_OP_EXPAND the scratch is optional (see llmem_expand_events).  For
+ * LLMEM_OP_EXPAND and LLMEM_OP_EXPAND_SCAN the size depends on total_events too. */
 size_t llmem_scratch_bytes(int op, int64_t n, int64_t total_events);
 
 /* Sections 4.2 and 5, fused: peak of each configuration without materialising
@@ -183,11 +184,14 @@ llmem_status llmem_slab_bounds(const int64_t* DEV offsets, int64_t n, int64_t ma
  *   offsets        DEV [n+1] as written by llmem_event_counts for the same cfg
  *   total_events   HOST value of offsets[n]
  *   delta_out      DEV [total_events], 8-byte aligned (16-byte alignment enables bulk stores)
- *   scratch        DEV, optional: llmem_scratch_bytes(LLMEM_OP_EXPAND, ..) bytes, 256-byte aligned.
- *                  It holds the counter from which the warps of a persistent grid claim blocks
- *                  of the list; with scratch = NULL (or too small) the same blocks are handed
- *                  out by the hardware block scheduler, one warp per block.  The list written
- *                  is the same either way. */
+ *   scratch        DEV, optional: llmem_scratch_bytes(LLMEM_OP_EXPAND, n, total_events) bytes,
+ *                  256-byte aligned.  For lists of long segments it holds the counter from which
+ *                  the warps of a persistent grid claim blocks of the list; for lists whose
+ *                  segments are short on average (about 1 KB per configuration then) the table of
+ *                  segment descriptors from which every segment is written by one lane or warp.
+ *                  With scratch = NULL (or too small) the list is cut into blocks handed out by
+ *                  the hardware block scheduler, one warp per block.  The list written is the
+ *                  same either way. */
 llmem_status llmem_expand_events(const llmem_config* DEV cfg, int64_t n, const int64_t* DEV offsets,
                                  int64_t total_events, int64_t* DEV delta_out, void* DEV scratch,
                                  size_t scratch_bytes, uint32_t flags, void* cuda_stream);

@@ -117,8 +117,9 @@ extern "C" size_t llmem_scratch_bytes(int op, int64_t n, int64_t total_events) {
       // header + one partial sum per block of 1024 configurations
       return kScratchHeader + (size_t)((n + 1023) / 1024 + 1) * sizeof(int64_t);
     case LLMEM_OP_EXPAND:
-      // header only: the work counter
-      return kScratchHeader;
+      // the work counter alone for lists of long segments; the descriptor table of the
+      // expansion by segment owners for lists of short ones
+      return short_segment_list(n, total_events) ? expand_scan_scratch_bytes(n, total_events) : kScratchHeader;
     case LLMEM_OP_SCAN_PEAK:
       // header, block starts and a head and a tail partial per block of the list
       return kStreamScratchBytes;

@@ -162,42 +162,58 @@ struct PageSearch {
 // ---------------------------------------------------------------------------
 // llmem_estimate_batch
 // ---------------------------------------------------------------------------
+// One configuration: status, peak and its position.
+__device__ __forceinline__ void estimate_one(const Cfg& f, i64* pk_out, i64* ix_out, int* st_out) {
+  int st = check_fields(f, true, true);
+  i64 pk = -1, ix = -1;
+  if (st == LLMEM_CFG_OK) {
+    Search q;
+    q.p = make_plan(f, f.method);
+    st = q.p.status;
+    if (st == LLMEM_CFG_OK) {
+      q.s = make_static_sums(q.p, f.pos_len > 0);
+      Dyn d;
+      bool first_wins;
+      u64 total = q.peak((u64)f.batch, &d, &first_wins);
+      if (total >= kSat) {
+        st = LLMEM_CFG_OVERFLOW;
+      } else {
+        pk = (i64)total;
+        const Plan& p = q.p;
+        // position of the peak: the last allocation of non-zero size in the
+        // iteration that attains it, or the last optimizer-state allocation
+        const u64 init_n = 2 + 2 * (u64)p.C;
+        const u64 gpart = p.gather ? 1 + (u64)p.C : 0;
+        const u64 outs = (u64)p.e_n + (u64)p.L * (u64)(p.n_x + p.n_attn + p.n_ffn);
+        const u64 allocs = gpart + outs + 3 + (p.tpback ? (u64)p.L : 0);
+        const u64 os_n = (u64)p.e_n + (u64)p.K * (u64)p.L;
+        const u64 last = (p.tpback && d.back > 0) ? allocs - 1
+                         : (d.shift > 0 ? gpart + outs + 2 : gpart + outs);
+        if (p.iters >= 2) ix = (i64)(init_n + 2 * allocs + os_n + last);
+        else if (first_wins) ix = (i64)(init_n + last);
+        else ix = (i64)(init_n + 2 * allocs + os_n - 1);
+      }
+    }
+  }
+  *pk_out = pk;
+  *ix_out = ix;
+  *st_out = st;
+}
+
+// One thread per configuration.  (Handing the configurations of a CTA's tile out in the order
+// of a counting sort by method, feed-forward kind and position embedding, so that a warp
+// evaluates one kind, does remove the divergence -- 30.5 instead of 26 of 32 lanes busy, a
+// tenth fewer warp instructions -- but the kernel waits on dependent 64-bit arithmetic rather
+// than on issue slots, and the barriers of the sort cost more than the idle lanes: 0.74 ms
+// instead of 0.69 ms for 2^24 configurations.)
 __global__ void __launch_bounds__(LLMEM_EST_THREADS, LLMEM_EST_MIN_CTAS)
 estimate_kernel(const llmem_config* __restrict__ cfg, i64 n, i64* __restrict__ peak_out,
                 i64* __restrict__ index_out, uint8_t* __restrict__ status_out) {
   for (i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (i64)gridDim.x * blockDim.x) {
-    Cfg f = load_cfg(cfg + i);
-    int st = check_fields(f, true, true);
-    i64 pk = -1, ix = -1;
-    if (st == LLMEM_CFG_OK) {
-      Search q;
-      q.p = make_plan(f, f.method);
-      st = q.p.status;
-      if (st == LLMEM_CFG_OK) {
-        q.s = make_static_sums(q.p, f.pos_len > 0);
-        Dyn d;
-        bool first_wins;
-        u64 total = q.peak((u64)f.batch, &d, &first_wins);
-        if (total >= kSat) {
-          st = LLMEM_CFG_OVERFLOW;
-        } else {
-          pk = (i64)total;
-          const Plan& p = q.p;
-          // position of the peak: the last allocation of non-zero size in the
-          // iteration that attains it, or the last optimizer-state allocation
-          const u64 init_n = 2 + 2 * (u64)p.C;
-          const u64 gpart = p.gather ? 1 + (u64)p.C : 0;
-          const u64 outs = (u64)p.e_n + (u64)p.L * (u64)(p.n_x + p.n_attn + p.n_ffn);
-          const u64 allocs = gpart + outs + 3 + (p.tpback ? (u64)p.L : 0);
-          const u64 os_n = (u64)p.e_n + (u64)p.K * (u64)p.L;
-          const u64 last = (p.tpback && d.back > 0) ? allocs - 1
-                           : (d.shift > 0 ? gpart + outs + 2 : gpart + outs);
-          if (p.iters >= 2) ix = (i64)(init_n + 2 * allocs + os_n + last);
-          else if (first_wins) ix = (i64)(init_n + last);
-          else ix = (i64)(init_n + 2 * allocs + os_n - 1);
-        }
-      }
-    }
+    const Cfg f = load_cfg(cfg + i);
+    i64 pk, ix;
+    int st;
+    estimate_one(f, &pk, &ix, &st);
     peak_out[i] = pk;
     if (index_out) index_out[i] = ix;
     if (status_out) status_out[i] = (uint8_t)st;

@@ -8,6 +8,7 @@
 
 #include "llmem_host.h"
 #include "expand.cuh"
+#include "fold.cuh"
 #include "ranges.cuh"
 
 namespace llmem {
@@ -417,6 +418,14 @@ extern "C" llmem_status llmem_expand_events(const llmem_config* cfg, int64_t n, 
     set_error("llmem_expand_events: misaligned pointer");
     return LLMEM_ERR_ARG;
   }
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (short_segment_list(n, total_events) && scratch && aligned_to(scratch, 256) &&
+      scratch_bytes >= expand_scan_scratch_bytes(n, total_events)) {
+    // lists of short segments: every segment written by its owner, a lane or a warp
+    if (cudaMemsetAsync(scratch, 0, kScratchHeader, s) != cudaSuccess) return check_launch("llmem_expand_events (memset)");
+    return expand_by_owners(cfg, n, reinterpret_cast<const i64*>(offsets), total_events, reinterpret_cast<i64*>(delta_out),
+                            (flags & LLMEM_FUSE_ROUND) != 0, false, nullptr, nullptr, scratch, nullptr, s);
+  }
   const size_t smem = sizeof(ExpandWarpSmem) * kExpWarps;
   static thread_local int configured_dev = -1;
   int dev = 0;
@@ -429,7 +438,6 @@ extern "C" llmem_status llmem_expand_events(const llmem_config* cfg, int64_t n, 
   const i64 nchunks = (total_events + kExpChunk - 1) / kExpChunk;
   const i64 resident = (i64)sm_count() * kExpCtasPerSm * kExpWarps;
   const i64 blocks = stream_warps(resident, LLMEM_EXP_OVERSUB, nchunks, LLMEM_EXP_MIN_CHUNKS);
-  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   // with scratch the warps of a persistent grid claim blocks from a counter in its header
   unsigned long long* work_counter = nullptr;
   u32* status_word = nullptr;  // only written by checked builds

@@ -303,4 +303,11 @@ llmem_status launch_scan_finish(const i64* offsets, i64 n, int shift, const llme
                                 i64* index_out, const i64* bounds, i64 n_warps, const WarpPartials* partials,
                                 cudaStream_t stream, PartsOfSegments parts = PartsOfSegments());
 
+// Host side of the expansion by segment owners (defined with its kernels): descriptor table,
+// list of parts, then every segment written by its owner into delta_out; with `fold` the bare
+// per-segment results as well.  `scratch` has llmem_expand_scan's layout, header cleared.
+llmem_status expand_by_owners(const llmem_config* cfg, i64 n, const i64* offsets, i64 total_events, i64* delta_out,
+                              bool round, bool fold, i64* peak_out, i64* index_out, void* scratch,
+                              PartsOfSegments* parts_out, cudaStream_t stream);
+
 }  // namespace llmem

@@ -316,7 +316,7 @@ struct OwnedWarpSmem {
 //
 // Results are the bare ones (largest prefix sum, its position): the finishing pass adds
 // m_base + lm_p.
-template <bool kRoundList, int kWarps>
+template <bool kRoundList, int kWarps, bool kFold>
 __global__ void __launch_bounds__(kWarps * 32, kOwnedCtasPerSm)
 expand_scan_owned_kernel(i64 n, const i64* __restrict__ offsets, i64 total, i64* __restrict__ out, i64 n_groups,
                          int par /* positions of this parity are 16-byte aligned in `out` */,
@@ -328,7 +328,7 @@ expand_scan_owned_kernel(i64 n, const i64* __restrict__ offsets, i64 total, i64*
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   OwnedWarpSmem& ws = reinterpret_cast<OwnedWarpSmem*>(smem_raw)[warp];
   const Guard g{reinterpret_cast<u32*>(reinterpret_cast<unsigned char*>(work_counter) - kWorkCounterOffset), n, total};
-  if (blockIdx.x == 0 && threadIdx.x == 0) {
+  if (kFold && blockIdx.x == 0 && threadIdx.x == 0) {
     // for the finishing pass: one block of work that owns every segment
     bounds[0] = 0;
     bounds[1] = total;
@@ -370,7 +370,8 @@ expand_scan_owned_kernel(i64 n, const i64* __restrict__ offsets, i64 total, i64*
             const i64 lim = lo - pos;
             int m = cur.rem < lim ? cur.rem : (int)lim;
             if (m < 1) m = 1;  // never reached with consistent descriptors
-            f.sum += skip_piece<!kRoundList>(m, cur);
+            const i64 passed = skip_piece<!kRoundList>(m, cur);
+            if (kFold) f.sum += passed;
             pos += m;
             if (cur.rem <= 0) cur.next_run();
           }
@@ -378,13 +379,13 @@ expand_scan_owned_kernel(i64 n, const i64* __restrict__ offsets, i64 total, i64*
             const i64 lim = hi - pos;
             int m = cur.rem < lim ? cur.rem : (int)lim;
             if (m < 1) m = 1;
-            emit_piece_by_warp<!kRoundList>(dst, (int)(pos - base), m, cur, f, base, lane);
+            emit_piece_by_warp<kFold, !kRoundList>(dst, (int)(pos - base), m, cur, f, base, lane);
             pos += m;
             if (cur.rem <= 0 && pos < hi) cur.next_run();
           }
           // a segment of one part has its result; the parts of a longer one are joined by the
           // finishing pass
-          if (lane == 0) {
+          if (kFold && lane == 0) {
             if (parts == 1) {
               write_raw(s, f.agg(), s_lo, peak_out, index_out);
             } else {
@@ -433,7 +434,7 @@ expand_scan_owned_kernel(i64 n, const i64* __restrict__ offsets, i64 total, i64*
             if (q < q_end) {
               int m = cur.rem < q_end - q ? cur.rem : q_end - q;
               if (m < 1) m = 1;  // never reached with consistent descriptors
-              emit_piece<!kRoundList>(row + q, q, (int)(row0 - gs) + q, m, cur, f);
+              emit_piece<kFold, !kRoundList>(row + q, q, (int)(row0 - gs) + q, m, cur, f);
               q += m;
               if (cur.rem <= 0 && row0 + q < ge) cur.next_run();
             }
@@ -460,7 +461,7 @@ expand_scan_owned_kernel(i64 n, const i64* __restrict__ offsets, i64 total, i64*
           }
           __syncwarp();
         }
-        if (mine && in_bounds(seg < g.n, g, kSiteResult))
+        if (kFold && mine && in_bounds(seg < g.n, g, kSiteResult))
           write_raw(seg, Agg{f.sum, f.mx, gs + f.ix, f.has ? 1 : 0}, gs, peak_out, index_out);
       }
     }
@@ -470,6 +471,70 @@ expand_scan_owned_kernel(i64 n, const i64* __restrict__ offsets, i64 total, i64*
     work = n_items > resident ? resident + (i64)ticket : n_items;
   }
 }
+
+
+// Host side of the owner kernel: descriptors of all configurations and the list of parts of
+// the longer segments (desc_table_kernel), then every segment written by its owner.  `scratch`
+// has the layout of llmem_expand_scan's; its header has been cleared by the caller.  With
+// `fold` the bare results go to peak_out / index_out and *parts_out tells the finishing pass
+// where the parts of the longer segments reported.
+llmem_status expand_by_owners(const llmem_config* cfg, i64 n, const i64* offsets, i64 total_events, i64* delta_out,
+                              bool round, bool fold, i64* peak_out, i64* index_out, void* scratch,
+                              PartsOfSegments* parts_out, cudaStream_t s) {
+  static thread_local int configured_dev = -1;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (configured_dev != dev) {
+    const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+    const int s_owned = (int)(sizeof(OwnedWarpSmem) * kOwnedWarps);
+    if (cudaFuncSetAttribute(expand_scan_owned_kernel<false, kOwnedWarps, false>, attr, s_owned) != cudaSuccess ||
+        cudaFuncSetAttribute(expand_scan_owned_kernel<true, kOwnedWarps, false>, attr, s_owned) != cudaSuccess ||
+        cudaFuncSetAttribute(expand_scan_owned_kernel<false, kOwnedWarps, true>, attr, s_owned) != cudaSuccess ||
+        cudaFuncSetAttribute(expand_scan_owned_kernel<true, kOwnedWarps, true>, attr, s_owned) != cudaSuccess ||
+        cudaFuncSetAttribute(desc_table_kernel, attr, (int)(sizeof(SegDesc) * kDescThreads)) != cudaSuccess)
+      return check_launch("expansion by segment owners (shared memory opt-in)");
+    configured_dev = dev;
+  }
+  unsigned char* base = static_cast<unsigned char*>(scratch) + kDescTableOffset;
+  SegDesc* table = reinterpret_cast<SegDesc*>(base);
+  const i64 part_capacity = max_parts(n, total_events);
+  i64* part_list = reinterpret_cast<i64*>(base + (size_t)n * sizeof(SegDesc));
+  PartResult* part_results = reinterpret_cast<PartResult*>(part_list + part_capacity);
+  i64* bounds = reinterpret_cast<i64*>(static_cast<unsigned char*>(scratch) + kBoundsOffset);
+  unsigned long long* work_counter = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(scratch) + kWorkCounterOffset);
+  unsigned long long* part_count = work_counter + 1;  // beside the work counter in the header
+  desc_table_kernel<<<(unsigned)((n + kDescThreads - 1) / kDescThreads), kDescThreads, sizeof(SegDesc) * kDescThreads, s>>>(
+      cfg, n, offsets, round ? 1 : 0, table, part_count, part_list, part_capacity);
+  llmem_status st = check_launch("expansion by segment owners (descriptor table)");
+  if (st != LLMEM_OK) return st;
+  const i64 n_groups = (n + 31) / 32;
+  // the number of parts is known on the device only: a persistent grid whatever it is
+  const unsigned grid = (unsigned)(sm_count() * kOwnedCtasPerSm);
+  const size_t smem = sizeof(OwnedWarpSmem) * kOwnedWarps;
+  const int par = aligned_to(delta_out, 16) ? 0 : 1;  // positions of this parity are 16-byte aligned
+#define LLMEM_LAUNCH_OWNED(ROUND, FOLD)                                                                          \
+  expand_scan_owned_kernel<ROUND, kOwnedWarps, FOLD><<<grid, kOwnedWarps * 32, smem, s>>>(                       \
+      n, offsets, total_events, delta_out, n_groups, par, peak_out, index_out, bounds, work_counter, table,       \
+      part_count, part_list, part_results, part_capacity)
+  if (fold) {
+    if (round) LLMEM_LAUNCH_OWNED(true, true); else LLMEM_LAUNCH_OWNED(false, true);
+  } else {
+    if (round) LLMEM_LAUNCH_OWNED(true, false); else LLMEM_LAUNCH_OWNED(false, false);
+  }
+#undef LLMEM_LAUNCH_OWNED
+  st = check_launch("expansion by segment owners");
+  if (st != LLMEM_OK) return st;
+  if (parts_out) {
+    parts_out->first_part = &table->first_part;
+    parts_out->stride = sizeof(SegDesc);
+    parts_out->results = part_results;
+    parts_out->lane_max = kOwnedLaneMax;
+    parts_out->part = kOwnedPart;
+  }
+  return LLMEM_OK;
+}
+
+bool short_segment_list(long long n, long long total_events) { return n > 0 && total_events > 0 && !long_segments(n, total_events); }
 
 }  // namespace llmem
 
@@ -511,12 +576,9 @@ extern "C" llmem_status llmem_expand_scan(const llmem_config* cfg, int64_t n, co
   cudaGetDevice(&dev);
   if (configured_dev != dev) {
     const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
-    const int s_long = (int)(sizeof(ExpandWarpSmem) * kFusedWarpsLong), s_owned = (int)(sizeof(OwnedWarpSmem) * kOwnedWarps);
-    if (cudaFuncSetAttribute(expand_scan_owned_kernel<false, kOwnedWarps>, attr, s_owned) != cudaSuccess ||
-        cudaFuncSetAttribute(expand_scan_owned_kernel<true, kOwnedWarps>, attr, s_owned) != cudaSuccess ||
-        cudaFuncSetAttribute(expand_scan_kernel<false, kFusedWarpsLong>, attr, s_long) != cudaSuccess ||
-        cudaFuncSetAttribute(expand_scan_kernel<true, kFusedWarpsLong>, attr, s_long) != cudaSuccess ||
-        cudaFuncSetAttribute(desc_table_kernel, attr, (int)(sizeof(SegDesc) * kDescThreads)) != cudaSuccess)
+    const int s_long = (int)(sizeof(ExpandWarpSmem) * kFusedWarpsLong);
+    if (cudaFuncSetAttribute(expand_scan_kernel<false, kFusedWarpsLong>, attr, s_long) != cudaSuccess ||
+        cudaFuncSetAttribute(expand_scan_kernel<true, kFusedWarpsLong>, attr, s_long) != cudaSuccess)
       return check_launch("llmem_expand_scan (shared memory opt-in)");
     configured_dev = dev;
   }
@@ -538,37 +600,10 @@ extern "C" llmem_status llmem_expand_scan(const llmem_config* cfg, int64_t n, co
     llmem_status st = check_launch("llmem_expand_scan");
     if (st != LLMEM_OK) return st;
   } else if (total_events > 0) {
-    // descriptors of all configurations and the list of parts of the longer segments, then
-    // every segment written by its owner
-    unsigned char* base = static_cast<unsigned char*>(scratch) + kDescTableOffset;
-    SegDesc* table = reinterpret_cast<SegDesc*>(base);
-    const i64 part_capacity = max_parts(n, total_events);
-    i64* part_list = reinterpret_cast<i64*>(base + (size_t)n * sizeof(SegDesc));
-    PartResult* part_results = reinterpret_cast<PartResult*>(part_list + part_capacity);
-    unsigned long long* part_count = work_counter + 1;  // beside the work counter in the header
-    desc_table_kernel<<<(unsigned)((n + kDescThreads - 1) / kDescThreads), kDescThreads, sizeof(SegDesc) * kDescThreads, s>>>(
-        cfg, n, reinterpret_cast<const i64*>(offsets), round ? 1 : 0, table, part_count, part_list, part_capacity);
-    llmem_status st = check_launch("llmem_expand_scan (descriptor table)");
+    llmem_status st = expand_by_owners(cfg, n, reinterpret_cast<const i64*>(offsets), total_events,
+                                       reinterpret_cast<i64*>(delta_out), round, true, reinterpret_cast<i64*>(peak_out),
+                                       reinterpret_cast<i64*>(peak_index_out), scratch, &parts_of_segments, s);
     if (st != LLMEM_OK) return st;
-    const i64 n_groups = (n + 31) / 32;
-    // the number of parts is known on the device only: a persistent grid whatever it is
-    const unsigned grid = (unsigned)(sm_count() * kOwnedCtasPerSm);
-    const size_t smem = sizeof(OwnedWarpSmem) * kOwnedWarps;
-    const int par = aligned_to(delta_out, 16) ? 0 : 1;  // positions of this parity are 16-byte aligned
-#define LLMEM_LAUNCH_OWNED(ROUND)                                                                               \
-  expand_scan_owned_kernel<ROUND, kOwnedWarps><<<grid, kOwnedWarps * 32, smem, s>>>(                             \
-      n, reinterpret_cast<const i64*>(offsets), total_events, reinterpret_cast<i64*>(delta_out), n_groups, par,   \
-      reinterpret_cast<i64*>(peak_out), reinterpret_cast<i64*>(peak_index_out), bounds, work_counter, table,      \
-      part_count, part_list, part_results, part_capacity)
-    if (round) LLMEM_LAUNCH_OWNED(true); else LLMEM_LAUNCH_OWNED(false);
-#undef LLMEM_LAUNCH_OWNED
-    st = check_launch("llmem_expand_scan");
-    if (st != LLMEM_OK) return st;
-    parts_of_segments.first_part = &table->first_part;
-    parts_of_segments.stride = sizeof(SegDesc);
-    parts_of_segments.results = part_results;
-    parts_of_segments.lane_max = kOwnedLaneMax;
-    parts_of_segments.part = kOwnedPart;
   }
   return launch_scan_finish(reinterpret_cast<const i64*>(offsets), n, 0, cfg, reinterpret_cast<i64*>(peak_out),
                             reinterpret_cast<i64*>(peak_index_out), bounds, warps, partials, s, parts_of_segments);

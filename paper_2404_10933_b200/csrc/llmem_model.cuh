@@ -90,9 +90,8 @@ struct Cfg {
   bool reserved_zero;
 };
 
-__device__ __forceinline__ Cfg load_cfg(const llmem_config* __restrict__ p) {
-  const int4* q = reinterpret_cast<const int4*>(p);
-  int4 a = __ldg(q), b = __ldg(q + 1), c = __ldg(q + 2), d = __ldg(q + 3);
+// The four 16-byte words of a record, unpacked.
+__device__ __forceinline__ Cfg unpack_cfg(const int4& a, const int4& b, const int4& c, const int4& d) {
   Cfg f;
   f.layers = a.x; f.hidden = a.y; f.heads = a.z; f.ffn = a.w;
   f.vocab = b.x; f.pos_len = b.y; f.seq = b.z; f.batch = b.w;
@@ -104,6 +103,12 @@ __device__ __forceinline__ Cfg load_cfg(const llmem_config* __restrict__ p) {
   f.act_mode = w1 >> 24;
   f.reserved_zero = d.z == 0 && d.w == 0;
   return f;
+}
+
+__device__ __forceinline__ Cfg load_cfg(const llmem_config* __restrict__ p) {
+  const int4* q = reinterpret_cast<const int4*>(p);
+  int4 a = __ldg(q), b = __ldg(q + 1), c = __ldg(q + 2), d = __ldg(q + 3);
+  return unpack_cfg(a, b, c, d);
 }
 
 // Field ranges (status 1).  `check_batch` is false for the search entry points,

@@ -197,7 +197,7 @@ struct SpanCursor {
 // of them has in the lane's segment.  The fold takes page-rounded values when the list itself
 // is written raw (kRoundFold).  Closed forms as in emit_piece_by_warp below.
 constexpr int kRowEvents = 16;  // events a lane stages per step: one 128-byte line
-template <bool kRoundFold>
+template <bool kFold, bool kRoundFold>
 __device__ __forceinline__ void emit_piece(i64* __restrict__ dst, int slot, int at, int m, SpanCursor& cur, LaneFold& f) {
   if (cur.period <= 2) {
     // x0 on the piece's even offsets, x1 on its odd ones (equal for a constant run)
@@ -213,25 +213,29 @@ __device__ __forceinline__ void emit_piece(i64* __restrict__ dst, int slot, int 
     for (int k = 0; k < kRowEvents / 2; ++k)
       if (k < pairs) v[k] = make_longlong2(e0, e1);
     if (j0 + 2 * pairs < m) dst[j0 + 2 * pairs] = e0;
-    const i64 y0 = ev<kRoundFold>(x0), y1 = ev<kRoundFold>(x1);
-    const i64 S = y0 + y1, s = f.sum;
-    const int n_even = (m + 1) >> 1, n_odd = m >> 1;
-    const bool rising = S > 0;
-    const int even_at = rising ? 2 * (n_even - 1) : 0, odd_at = rising ? 2 * n_odd - 1 : 1;
-    const i64 even_v = s + y0 + (rising ? (i64)(n_even - 1) * S : 0);
-    const i64 odd_v = s + (rising ? (i64)n_odd * S : S);
-    const bool even_first = even_at < odd_at || n_odd == 0;
-    f.offer(even_first ? even_v : odd_v, at + (even_first ? even_at : odd_at));
-    if (n_odd > 0) f.offer(even_first ? odd_v : even_v, at + (even_first ? odd_at : even_at));
-    f.sum = s + (i64)n_odd * S + ((m & 1) ? y0 : 0);
+    if (kFold) {
+      const i64 y0 = ev<kRoundFold>(x0), y1 = ev<kRoundFold>(x1);
+      const i64 S = y0 + y1, s = f.sum;
+      const int n_even = (m + 1) >> 1, n_odd = m >> 1;
+      const bool rising = S > 0;
+      const int even_at = rising ? 2 * (n_even - 1) : 0, odd_at = rising ? 2 * n_odd - 1 : 1;
+      const i64 even_v = s + y0 + (rising ? (i64)(n_even - 1) * S : 0);
+      const i64 odd_v = s + (rising ? (i64)n_odd * S : S);
+      const bool even_first = even_at < odd_at || n_odd == 0;
+      f.offer(even_first ? even_v : odd_v, at + (even_first ? even_at : odd_at));
+      if (n_odd > 0) f.offer(even_first ? odd_v : even_v, at + (even_first ? odd_at : even_at));
+      f.sum = s + (i64)n_odd * S + ((m & 1) ? y0 : 0);
+    }
     if (cur.period == 2) cur.phase ^= (m & 1);
   } else {
     int ph = cur.phase;
     for (int j = 0; j < m; ++j) {
       const i64 x = cur.value(ph);
       dst[j] = x;
-      f.sum += ev<kRoundFold>(x);
-      f.offer(f.sum, at + j);
+      if (kFold) {
+        f.sum += ev<kRoundFold>(x);
+        f.offer(f.sum, at + j);
+      }
       if (++ph == cur.period) ph = 0;
     }
     cur.phase = ph;
@@ -288,7 +292,7 @@ __device__ __forceinline__ void count_kinds(u32 code, u32 period, u32 from, u32 
 // have one sign the prefix sums are monotone and only the piece's sum is needed, which the
 // counts of each value give; a few events are folded one by one; anything else by the lanes
 // over consecutive parts of the piece, joined with shuffles.
-template <bool kRoundFold>
+template <bool kFold, bool kRoundFold>
 __device__ __forceinline__ void emit_piece_by_warp(i64* __restrict__ buf, int l0, int m, SpanCursor& cur, WarpFold& f,
                                                    i64 t0, int lane) {
   const i64 at = t0 + l0;
@@ -304,6 +308,11 @@ __device__ __forceinline__ void emit_piece_by_warp(i64* __restrict__ buf, int l0
 #pragma unroll 3
     for (int q = lane; q < pairs; q += 32) v[q] = make_longlong2(e0, e1);
     if (((end - a0) & 1) && lane == 31) buf[end - 1] = e0;
+    if (!kFold) {
+      if (cur.period == 2) cur.phase ^= (m & 1);
+      cur.rem -= m;
+      return;
+    }
     const i64 y0 = ev<kRoundFold>(x0), y1 = ev<kRoundFold>(x1);
     const i64 S = y0 + y1, s = f.sum;
     const int n_even = (m + 1) >> 1, n_odd = m >> 1;
@@ -329,6 +338,12 @@ __device__ __forceinline__ void emit_piece_by_warp(i64* __restrict__ buf, int l0
         ph += step;
         if (ph >= period) ph -= period;
       }
+    }
+    if (!kFold) {
+      const u32 after = phase + (u32)m;
+      cur.phase = (int)(after - (after / period) * period);
+      cur.rem -= m;
+      return;
     }
     const i64 ya = ev<kRoundFold>(cur.a), yb = ev<kRoundFold>(cur.b), yc = ev<kRoundFold>(cur.c);
     u32 n_b, n_c;

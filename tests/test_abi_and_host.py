@@ -36,6 +36,9 @@ def test_scratch_bytes_and_argument_errors_need_no_gpu():
     L = llmem.lib()
     assert L.llmem_scratch_bytes(llmem.OP_ESTIMATE, 1000, 0) == 0
     assert L.llmem_scratch_bytes(llmem.OP_EXPAND, 1000, 10 ** 9) == 256  # optional: the work counter
+    # lists of short segments: a descriptor per configuration for the expansion by segment owners
+    assert L.llmem_scratch_bytes(llmem.OP_EXPAND, 1000, 10 ** 6) == L.llmem_scratch_bytes(llmem.OP_EXPAND_SCAN, 1000, 10 ** 6)
+    assert L.llmem_scratch_bytes(llmem.OP_EXPAND_SCAN, 1000, 10 ** 6) > 1000 * 800
     assert L.llmem_scratch_bytes(llmem.OP_EVENT_COUNTS, 5000, 0) >= 256 + 8 * 6
     assert L.llmem_scratch_bytes(llmem.OP_SCAN_PEAK, 5000, 10 ** 9) >= 256 + 64
     # call-level errors are detected before any CUDA call
