@@ -54,7 +54,9 @@ FALLBACK_HBM_GBS = 6650.0
 # HBM-bound kernels, from an ncu capture of a 4096-configuration run (summary kept under
 # profiles/; traffic grows in proportion to the number of events).  Set an entry
 # to None when its kernel changes after the capture.
-NCU_TRAFFIC_BYTES_PER_EVENT = {"expand": None, "scan": None, "expand_scan": None}
+NCU_TRAFFIC_BYTES_PER_EVENT = {"expand": 7.8207, "scan": 8.0125, "expand_scan": 7.8231}
+# the same for the owner kernel that takes lists of short and medium segments (64-shape capture)
+NCU_TRAFFIC_BYTES_PER_EVENT_OWNERS = 8.03
 
 
 def measured_peaks():
@@ -555,7 +557,7 @@ def run_ours(args):
 # grids (profiles/register_kernels_g3_g4_ncu.md); None once a kernel changes after the capture.
 # Counting lane instructions keeps divergence from passing for throughput: a warp instruction
 # issued for 20 of 32 lanes counts as 20/32.
-NCU_LANE_INSTR_PER_UNIT = {"estimate_kernel": None, "max_batch_kernel": None, "select_kernel": None}
+NCU_LANE_INSTR_PER_UNIT = {"estimate_kernel": 25.24, "max_batch_kernel": 8.40, "select_kernel": 40.21}
 
 
 def _gpu_id(torch):
@@ -693,7 +695,11 @@ def leg_slabs(llmem, torch, steps, warmup, shapes=None):
             "roofline": {"bound": "hbm", "kernel": "whole step (per slab: counts, descriptor table, expand_scan_owned_kernel, "
                                                    "finishing pass; host slab loop)",
                          "achieved": achieved, "peak": peak_gbs, "unit": "GB/s", "frac": achieved / peak_gbs,
-                         "frac_of_nominal_8000": achieved / 8000.0, "peak_source": peak_src, "traffic": None},
+                         "frac_of_nominal_8000": achieved / 8000.0, "peak_source": peak_src,
+                         "traffic": (NCU_TRAFFIC_BYTES_PER_EVENT_OWNERS * events
+                                     if NCU_TRAFFIC_BYTES_PER_EVENT_OWNERS is not None else None),
+                         "traffic_note": "ncu dram bytes per event of expand_scan_owned_kernel on a 64-shape capture, scaled by events",
+                         "algorithmic_bytes": 8.0 * events},
             "gpu_launches": steps * (4 + slabs * 7), "clocks": clocks, "fused_equals_materialised": agree}
 
 
