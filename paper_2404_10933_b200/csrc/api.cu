@@ -121,8 +121,9 @@ extern "C" size_t llmem_scratch_bytes(int op, int64_t n, int64_t total_events) {
       // expansion by segment owners for lists of short ones
       return short_segment_list(n, total_events) ? expand_scan_scratch_bytes(n, total_events) : kScratchHeader;
     case LLMEM_OP_SCAN_PEAK:
-      // header, block starts and a head and a tail partial per block of the list
-      return kStreamScratchBytes;
+      // header, block starts and a head and a tail partial per block of the list; for lists of
+      // short segments also the list of parts of the longer ones
+      return scan_scratch_bytes(n, total_events);
     case LLMEM_OP_EXPAND_SCAN:
       // the same, plus a descriptor per configuration when the segments are short
       return expand_scan_scratch_bytes(n, total_events);

@@ -283,7 +283,8 @@ __device__ __forceinline__ Fold3 fold_lane_span(const i64* __restrict__ span) {
 // largest prefix sum inside the part, counted from the segment's start, and its position.
 struct PartResult {
   i64 mx, idx;
-  i64 has, pad;
+  i64 has;
+  i64 sum;  // sum of the part's events (used where the parts' prefix sums are relative to the part)
 };
 
 // Segments cut into parts, for the finishing pass: segment i has more than `lane_max` events,
@@ -293,6 +294,10 @@ struct PartsOfSegments {
   size_t stride = 0;
   const PartResult* results = nullptr;
   i64 lane_max = 0, part = 1;
+  // true: a part's mx counts from the part's own start (the scan of a given list cannot know what
+  // precedes the part) and the parts are joined in order with their sums; false: it counts
+  // from the segment's start (the expansion knows the runs before the part)
+  bool relative = false;
 };
 
 // Host launcher of the finishing pass (defined with the scan kernels): one thread per

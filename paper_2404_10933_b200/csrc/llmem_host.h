@@ -44,6 +44,9 @@ constexpr size_t kWorkCounterOffset = 64;
 // Scratch of llmem_expand_scan: header, block starts, partials and, for lists of short
 // segments, one descriptor per configuration (defined with the kernel).
 size_t expand_scan_scratch_bytes(long long n, long long total_events);
+// Scratch of llmem_scan_peak: the same header, block starts and partials and, for lists of short
+// segments, the list of parts of the longer ones (defined with the kernels).
+size_t scan_scratch_bytes(long long n, long long total_events);
 // Lists whose segments are short on average are expanded by segment owners (fused.cu), which
 // need that scratch; the others chunk by chunk.
 bool short_segment_list(long long n, long long total_events);

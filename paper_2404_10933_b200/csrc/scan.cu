@@ -257,6 +257,255 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
   }
 }
 
+// ---------------------------------------------------------------------------
+// Lists of short and medium segments: every segment scanned by its owner
+// ---------------------------------------------------------------------------
+// Segments of up to this many events are scanned by one lane each; longer ones are cut into
+// parts of this many events, each scanned by a warp (a lane's staged lines read about 1.6 TB/s
+// whatever the length, a warp's bulk copies 3.3 TB/s on 866-event and 6 TB/s on 3 k-event
+// segments: the lanes only pay below a few hundred events).
+#ifndef LLMEM_SCAN_LANE_MAX
+#define LLMEM_SCAN_LANE_MAX 384
+#endif
+#ifndef LLMEM_SCAN_PART
+#define LLMEM_SCAN_PART 4096
+#endif
+// Lists whose segments average fewer events than this are scanned by owners.
+#ifndef LLMEM_SCAN_OWNED_BELOW
+#define LLMEM_SCAN_OWNED_BELOW 8192
+#endif
+constexpr i64 kScanLaneMax = LLMEM_SCAN_LANE_MAX, kScanPart = LLMEM_SCAN_PART, kScanOwnedBelow = LLMEM_SCAN_OWNED_BELOW;
+static_assert(LLMEM_SCAN_PART % 2 == 0 && LLMEM_SCAN_PART < (1 << 20), "parts: 16-byte words, part numbers fit 20 bits");
+
+inline bool scan_by_owners(i64 n, i64 total_events) { return n > 0 && total_events > 0 && total_events / n < kScanOwnedBelow; }
+inline i64 scan_max_parts(i64 n, i64 total_events) { return total_events / kScanPart + n + 1; }
+// behind the header, block starts and partials of the chunk kernel: the first part of every
+// segment, the list of parts, one result per part
+constexpr size_t kScanPartsOffset = (kStreamScratchBytes + 255) / 256 * 256;
+
+size_t scan_scratch_bytes(long long n, long long total_events) {
+  if (!scan_by_owners(n, total_events)) return kStreamScratchBytes;
+  return kScanPartsOffset + (size_t)n * sizeof(i64) + (size_t)scan_max_parts(n, total_events) * (sizeof(i64) + sizeof(PartResult));
+}
+
+// One thread per segment: a segment too long for a lane enters its parts into the list of
+// parts (segment << 20 | part number, a segment's parts next to each other) and notes where
+// they start; the others note -1.
+__global__ void __launch_bounds__(256)
+scan_parts_kernel(const i64* __restrict__ offsets, i64 n, unsigned long long* __restrict__ part_count,
+                  i64* __restrict__ part_list, i64* __restrict__ first_part, i64 part_capacity) {
+  const i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x;
+  const int lane = threadIdx.x & 31;
+  const i64 count = i < n ? __ldg(offsets + i + 1) - __ldg(offsets + i) : 0;
+  const i64 parts = count > kScanLaneMax ? (count + kScanPart - 1) / kScanPart : 0;
+  i64 before = parts;  // parts of this and the lower lanes
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const i64 o = __shfl_up_sync(0xffffffffu, before, d);
+    if (lane >= d) before += o;
+  }
+  const i64 in_warp = __shfl_sync(0xffffffffu, before, 31);
+  i64 slot = -1;
+  if (in_warp > 0) {
+    unsigned long long slot0 = 0;
+    if (lane == 0) slot0 = atomicAdd(part_count, (unsigned long long)in_warp);
+    const i64 mine = (i64)__shfl_sync(0xffffffffu, slot0, 0) + before - parts;
+    if (parts > 0 && mine + parts <= part_capacity) {  // always, by the size of the scratch
+      for (i64 k = 0; k < parts; ++k) part_list[mine + k] = (i << 20) | k;
+      slot = mine;
+    }
+  }
+  if (i < n) first_part[i] = slot;
+}
+
+// Segmented prefix-sum + max for lists of short and medium segments.  The warps of a persistent
+// grid claim items from one counter: first the parts of the longer segments, then groups of
+// 32 consecutive segments.  In a group every segment of up to 384 events is scanned by one
+// lane: each step the warp brings the next 128-byte line of all 32 segments into shared memory
+// (eight lanes per line: 16-byte loads from 32 different lines in one instruction reach a
+// fifth of the bandwidth) and every lane folds its own line in order: no segment boundaries
+// to find in a chunk, no pieces to join.  A part is streamed by the whole
+// warp through the same two-stage ring of TMA bulk copies as in the kernel above, each lane
+// folding 26 consecutive events of a landed chunk; since a part lies inside one segment there
+// is only the fast path.  The finishing pass joins the parts of a segment in order.
+constexpr int kScanRowEvents = 16;                  // events a lane takes per step: one 128-byte line
+constexpr int kScanRowStride = kScanRowEvents + 2;  // 144 bytes: the lanes' rows fall on distinct banks
+static_assert(32 * kScanRowStride <= kScanChunk && 64 <= kScanChunk, "rows and segment ranges fit the stages");
+
+#ifndef LLMEM_SCAN_OWNED_WARPS
+#define LLMEM_SCAN_OWNED_WARPS 16
+#endif
+constexpr int kScanOwnedWarps = LLMEM_SCAN_OWNED_WARPS;
+
+template <bool kRound>
+__global__ void __launch_bounds__(kScanOwnedWarps * 32, 1)
+scan_owned_kernel(const i64* __restrict__ delta_aligned, int shift, const i64* __restrict__ offsets, i64 n, i64 total,
+                  i64* __restrict__ peak_out, i64* __restrict__ index_out, i64 n_groups,
+                  unsigned long long* __restrict__ work_counter, const unsigned long long* __restrict__ part_count,
+                  const i64* __restrict__ part_list, PartResult* __restrict__ part_results, i64 part_capacity,
+                  i64* __restrict__ bounds, u32* __restrict__ status_word) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  ScanWarpSmem& ws = reinterpret_cast<ScanWarpSmem*>(smem_raw)[warp];
+  __shared__ int abort_flags[kScanOwnedWarps];
+  const Guard guard{status_word, n, total};
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    // for the finishing pass: one block of work that owns every segment
+    bounds[0] = shift;
+    bounds[1] = (i64)shift + total;
+  }
+  if (lane == 0) {
+    for (int s = 0; s < kScanStages; ++s) mbar_init(&ws.full[s], 1);
+    abort_flags[warp] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  __syncwarp();
+  volatile int* abort_flag = &abort_flags[warp];
+  u32 phase_bits = 0;  // parity of each stage's next completion
+  bool aborted = false;
+  i64 n_parts = (i64)*part_count;
+  if (n_parts > part_capacity) n_parts = part_capacity;
+  const i64 n_items = n_parts + n_groups;
+  const i64 resident = (i64)gridDim.x * kScanOwnedWarps;
+  for (i64 item = (i64)blockIdx.x * kScanOwnedWarps + warp; item < n_items && !aborted;) {
+    if (item < n_parts) {
+      // ---- the whole warp for one part of a longer segment ----
+      const i64 entry = part_list[item];
+      const i64 s = entry >> 20, k = entry & 0xfffff;
+      if (in_bounds(s >= 0 && s < n && k <= item, guard, kSiteDescriptor)) {
+        const i64 s_lo = __ldg(offsets + s) + shift, s_hi = __ldg(offsets + s + 1) + shift;  // virtual positions
+        const i64 lo = s_lo + k * kScanPart, hi = lo + kScanPart < s_hi ? lo + kScanPart : s_hi;
+        const i64 parts = (s_hi - s_lo + kScanPart - 1) / kScanPart;
+        if (in_bounds(s_lo >= shift && s_hi <= (i64)shift + total && lo < hi, guard, kSiteLoad)) {
+          // chunks of the part, from an even position so that the copies start on 16-byte boundaries
+          const i64 c0 = lo & ~(i64)1;
+          const i64 n_chunks = (hi - c0 + kScanChunk - 1) / kScanChunk;
+          auto issue = [&](i64 c) {
+            const int st = (int)(c % kScanStages);
+            const i64 t0 = c0 + c * kScanChunk;
+            const i64 v_lo = t0 > lo ? t0 : lo, v_hi = t0 + kScanChunk < hi ? t0 + kScanChunk : hi;
+            const i64 a_lo = v_lo + (v_lo & 1), a_hi = v_hi - (v_hi & 1);
+            i64* dst = ws.stage[st];
+            if (a_lo > v_lo) dst[v_lo - t0] = delta_aligned[v_lo];
+            if (a_hi < v_hi && v_hi - 1 >= a_lo) dst[v_hi - 1 - t0] = delta_aligned[v_hi - 1];
+            if (a_hi > a_lo) {
+              const u32 bytes = (u32)((a_hi - a_lo) * 8);
+              mbar_arrive_expect_tx(&ws.full[st], bytes);
+              bulk_load(dst + (a_lo - t0), delta_aligned + a_lo, bytes, &ws.full[st]);
+            } else {
+              mbar_arrive(&ws.full[st]);
+            }
+          };
+          if (lane == 0)
+            for (i64 c = 0; c < n_chunks && c < kScanStages; ++c) issue(c);
+          SegmentFolder folder;
+          i64 consumed = 0;
+          for (i64 c = 0; c < n_chunks; ++c, ++consumed) {
+            const int st = (int)(c % kScanStages);
+            const bool ok = mbar_wait_bounded(&ws.full[st], (phase_bits >> st) & 1u, abort_flag);
+            phase_bits ^= 1u << st;
+            if (!__all_sync(0xffffffffu, ok)) { aborted = true; break; }
+            const i64* tile = ws.stage[st];
+            const i64 t0 = c0 + c * kScanChunk;
+            const i64 v_lo = t0 > lo ? t0 : lo, v_hi = t0 + kScanChunk < hi ? t0 + kScanChunk : hi;
+            if (v_lo == t0 && v_hi == t0 + kScanChunk) {
+              const Fold3 f = fold_lane_span<kRound, kScanPerLane>(tile + lane * kScanPerLane);
+              __syncwarp();  // every lane has consumed its part of the stage: refill it
+              if (lane == 0 && c + kScanStages < n_chunks) issue(c + kScanStages);
+              folder.add_spans<kScanPerLane>(f, t0, lane);
+            } else {
+              const Agg g = warp_fold_range<kRound>(tile, (int)(v_lo - t0), (int)(v_hi - t0), lane, t0);
+              folder.add_piece(g, lane);
+              __syncwarp();
+              if (lane == 0 && c + kScanStages < n_chunks) issue(c + kScanStages);
+            }
+          }
+          if (aborted) {
+            // drain: every copy that was issued must have landed before the warp goes on or exits
+            if (lane == 0) {
+              i64 issued = n_chunks < consumed + kScanStages ? n_chunks : consumed + kScanStages;
+              for (i64 c = consumed; c < issued; ++c) {
+                const int st = (int)(c % kScanStages);
+                mbar_wait_bounded(&ws.full[st], (phase_bits >> st) & 1u, nullptr);
+              }
+            }
+          } else {
+            const Agg whole = folder.take();
+            if (lane == 0) {
+              if (parts == 1) {
+                write_raw(s, whole, s_lo, peak_out, index_out);
+              } else {
+                PartResult* mine = part_results + item;
+                mine->sum = whole.sum;
+                mine->mx = whole.mx;
+                mine->idx = whole.idx;
+                mine->has = whole.valid;
+              }
+            }
+          }
+        }
+      }
+    } else {
+      // ---- one lane for each short segment of a group ----
+      const i64 seg = (item - n_parts) * 32 + lane;
+      const bool have = seg < n;
+      const i64 gs = have ? __ldg(offsets + seg) + shift : 0, ge = have ? __ldg(offsets + seg + 1) + shift : 0;
+      const bool mine = have && ge > gs && ge - gs <= kScanLaneMax &&
+                        in_bounds(gs >= shift && ge <= (i64)shift + total, guard, kSiteLoad);
+      if (__any_sync(0xffffffffu, mine)) {
+        // Rows of 16 events (one 128-byte line), one per lane, in the warp's first stage; the
+        // ranges of the lanes' segments in its second.  A step brings the next line of every
+        // segment in with 16-byte loads, eight lanes per line, so that device memory is read in
+        // whole lines although every lane then folds a list of its own.
+        i64(*rows)[kScanRowStride] = reinterpret_cast<i64(*)[kScanRowStride]>(ws.stage[0]);
+        i64* first = ws.stage[1];
+        i64* last = ws.stage[1] + 32;
+        const i64 base = gs & ~(i64)1;  // slot 0 of a lane's rows: the last even position at or before its segment
+        first[lane] = mine ? gs : 0;
+        last[lane] = mine ? ge : 0;
+        __syncwarp();
+        i64 sum = 0, mx = 0, idx = -1;
+        bool has = false;
+        for (i64 step = 0; __any_sync(0xffffffffu, mine && base + step * kScanRowEvents < ge); ++step) {
+#pragma unroll
+          for (int pass = 0; pass < 8; ++pass) {
+            const int r = (lane >> 3) + 4 * pass, vec = lane & 7;
+            const i64 lo_r = first[r], hi_r = last[r];
+            const i64 at = (lo_r & ~(i64)1) + step * kScanRowEvents + 2 * vec;
+            longlong2 x = make_longlong2(0, 0);
+            if (at >= lo_r && at + 1 < hi_r) {
+              x = __ldg(reinterpret_cast<const longlong2*>(delta_aligned + at));
+            } else {
+              if (at >= lo_r && at < hi_r) x.x = __ldg(delta_aligned + at);
+              if (at + 1 >= lo_r && at + 1 < hi_r) x.y = __ldg(delta_aligned + at + 1);
+            }
+            *reinterpret_cast<longlong2*>(&rows[r][2 * vec]) = x;
+          }
+          __syncwarp();
+          const i64 row0 = base + step * kScanRowEvents;
+          if (mine && row0 < ge) {
+            const int q_lo = row0 < gs ? (int)(gs - row0) : 0;
+            const int q_end = ge - row0 < kScanRowEvents ? (int)(ge - row0) : kScanRowEvents;
+            const i64* row = rows[lane];
+            for (int q = q_lo; q < q_end; ++q) {
+              sum += ev<kRound>(row[q]);
+              if (!has || sum > mx) { mx = sum; idx = row0 + q; has = true; }
+            }
+          }
+          __syncwarp();
+        }
+        if (mine && in_bounds(seg < guard.n, guard, kSiteResult))
+          write_raw(seg, Agg{sum, mx, idx, has ? 1 : 0}, gs, peak_out, index_out);
+      }
+    }
+    unsigned long long ticket = 0;
+    if (lane == 0 && n_items > resident) ticket = atomicAdd(work_counter, 1ull);
+    ticket = __shfl_sync(0xffffffffu, ticket, 0);
+    item = n_items > resident ? resident + (i64)ticket : n_items;
+  }
+  if (lane == 0 && (aborted || *abort_flag)) atomicExch(status_word, (u32)LLMEM_ERR_TIMEOUT);
+}
+
 // Self-test of the bounded wait: one warp waits on an mbarrier that nothing will ever
 // complete, with the given limit; the wait must give up and the warp records
 // LLMEM_ERR_TIMEOUT exactly as the scan kernel would.  Nothing else is touched.
@@ -304,13 +553,16 @@ scan_finish_kernel(const i64* __restrict__ offsets, i64 n, int shift, const llme
         // largest is the segment's
         const i64 first = *reinterpret_cast<const i64*>(reinterpret_cast<const unsigned char*>(parts.first_part) + (size_t)i * parts.stride);
         bool has = false;
+        i64 before = 0;  // sum of the parts already joined
         for (i64 j = 0; j < n_parts && first >= 0; ++j) {
           const PartResult r = parts.results[first + j];
-          if (r.has && (!has || r.mx > mx)) {
-            mx = r.mx;
+          const i64 base = parts.relative ? before : 0;
+          if (r.has && (!has || base + r.mx > mx)) {
+            mx = base + r.mx;
             idx = r.idx - a;
             has = true;
           }
+          before += r.sum;
         }
       } else if (ca == cb) {  // finished by the warp that owns it
         mx = peak_out[i];
@@ -377,7 +629,51 @@ extern "C" llmem_status llmem_scan_peak(const int64_t* delta, const int64_t* off
   const i64* delta_aligned = reinterpret_cast<const i64*>(delta) - shift;
   const bool round = (flags & LLMEM_FUSE_ROUND) != 0;
   i64 warps = 1;
-  if (total_events > 0) {
+  PartsOfSegments parts_of_segments;
+  if (scan_by_owners(n, total_events)) {
+    // lists of short and medium segments: every segment scanned by its owner
+    const size_t smem = sizeof(ScanWarpSmem) * kScanOwnedWarps;
+    static thread_local int owned_dev = -1;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (owned_dev != dev) {
+      cudaError_t e1 = cudaFuncSetAttribute(scan_owned_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      cudaError_t e2 = cudaFuncSetAttribute(scan_owned_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e1 != cudaSuccess || e2 != cudaSuccess) return check_launch("llmem_scan_peak (shared memory opt-in)");
+      owned_dev = dev;
+    }
+    unsigned char* base = static_cast<unsigned char*>(scratch) + kScanPartsOffset;
+    i64* first_part = reinterpret_cast<i64*>(base);
+    const i64 part_capacity = scan_max_parts(n, total_events);
+    i64* part_list = first_part + n;
+    PartResult* part_results = reinterpret_cast<PartResult*>(part_list + part_capacity);
+    unsigned long long* work_counter = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(scratch) + kWorkCounterOffset);
+    unsigned long long* part_count = work_counter + 1;
+    scan_parts_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(reinterpret_cast<const i64*>(offsets), n, part_count, part_list,
+                                                                 first_part, part_capacity);
+    llmem_status st = check_launch("llmem_scan_peak (parts)");
+    if (st != LLMEM_OK) return st;
+    const i64 n_groups = (n + 31) / 32;
+    const unsigned grid = (unsigned)sm_count();
+    if (round)
+      scan_owned_kernel<true><<<grid, kScanOwnedWarps * 32, smem, s>>>(
+          delta_aligned, shift, reinterpret_cast<const i64*>(offsets), n, total_events, reinterpret_cast<i64*>(peak_out),
+          reinterpret_cast<i64*>(peak_index_out), n_groups, work_counter, part_count, part_list, part_results, part_capacity,
+          bounds, status_word);
+    else
+      scan_owned_kernel<false><<<grid, kScanOwnedWarps * 32, smem, s>>>(
+          delta_aligned, shift, reinterpret_cast<const i64*>(offsets), n, total_events, reinterpret_cast<i64*>(peak_out),
+          reinterpret_cast<i64*>(peak_index_out), n_groups, work_counter, part_count, part_list, part_results, part_capacity,
+          bounds, status_word);
+    st = check_launch("llmem_scan_peak");
+    if (st != LLMEM_OK) return st;
+    parts_of_segments.first_part = first_part;
+    parts_of_segments.stride = sizeof(i64);
+    parts_of_segments.results = part_results;
+    parts_of_segments.lane_max = kScanLaneMax;
+    parts_of_segments.part = kScanPart;
+    parts_of_segments.relative = true;
+  } else if (total_events > 0) {
     const size_t smem = sizeof(ScanWarpSmem) * kScanWarps;
     static thread_local int configured_dev = -1;
     int dev = 0;
@@ -405,7 +701,7 @@ extern "C" llmem_status llmem_scan_peak(const int64_t* delta, const int64_t* off
     if (st != LLMEM_OK) return st;
   }
   return launch_scan_finish(reinterpret_cast<const i64*>(offsets), n, shift, cfg, reinterpret_cast<i64*>(peak_out),
-                            reinterpret_cast<i64*>(peak_index_out), bounds, warps, partials, s);
+                            reinterpret_cast<i64*>(peak_index_out), bounds, warps, partials, s, parts_of_segments);
 }
 
 extern "C" llmem_status llmem_selftest_wait_limit(void* scratch, size_t scratch_bytes, uint32_t limit_ms,
