@@ -133,6 +133,45 @@ def estimate(cfg: np.ndarray, level: int = 1, threads: int = 1):
     return {"peak": peak, "index": index, "status": status, "count": count}
 
 
+# ---- the DNNMem-style second estimator (Section 3.1) ---------------------------
+def dnn_event_count(cfg: np.ndarray) -> tuple[int, int]:
+    cfg = _cfgs(cfg)
+    n = ctypes.c_int64(0)
+    st = lib().oracle_dnn_event_count(_rec(cfg), ctypes.byref(n))
+    return int(st), int(n.value)
+
+
+def dnn_expand_events(cfg: np.ndarray) -> np.ndarray:
+    """Raw byte counts of the second estimator's allocations, in order."""
+    cfg = _cfgs(cfg)
+    st, n = dnn_event_count(cfg)
+    if st:
+        raise ValueError(f"status {st}")
+    out = np.zeros(n, dtype=np.int64)
+    st = lib().oracle_dnn_expand_events(_rec(cfg), _p(out), ctypes.c_int64(n))
+    assert st == 0
+    return out
+
+
+def dnn_round_events(delta: np.ndarray) -> np.ndarray:
+    out = np.ascontiguousarray(delta, dtype=np.int64).copy()
+    lib().oracle_dnn_round_events(_p(out), ctypes.c_int64(out.size))
+    return out
+
+
+def dnn_estimate(cfg: np.ndarray, threads: int = 1):
+    """Returns dict(peak, index, status, count) of the second estimator."""
+    cfg = _cfgs(cfg)
+    n = cfg.size
+    peak = np.full(n, -1, dtype=np.int64)
+    index = np.full(n, -1, dtype=np.int64)
+    status = np.zeros(n, dtype=np.uint8)
+    count = np.zeros(n, dtype=np.int64)
+    lib().oracle_dnn_estimate_many(_p(cfg), ctypes.c_int64(n), _p(peak), _p(index), _p(status), _p(count),
+                                   ctypes.c_int(threads))
+    return {"peak": peak, "index": index, "status": status, "count": count}
+
+
 def list_digest(cfg: np.ndarray, threads: int = 1):
     """Two position-weighted checksums (mod 2^64) of each configuration's page-rounded event
     list: sum d[k] (k + 1) and sum d[k] (k + 1)^2 over the positions k of the list (zeros where

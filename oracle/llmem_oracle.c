@@ -39,6 +39,15 @@
  * number: the list here is a reading, pinned only to an independent
  * enumeration of the same reading and to its reduction to m_out).
  *
+ * A second estimator (oracle_dnn_*) restates the DNNMem-style procedure that Section 3.1
+ * describes and the paper compares with: weight tensors as loaded plus a constant 64 MB
+ * buffer, then the outputs of the forward pass accumulated operator by operator, every
+ * tensor aligned to 512 bytes; no mixed precision, no chunks, no optimizer states.  The paper
+ * gives the procedure in words only: the tensor list is this file's standard-decoder
+ * inventory and the event order a reading ("parity unpinned" with respect to the paper's
+ * numbers, which need its models); pinned to an independent tensor enumeration and to the
+ * facts that the list only grows and that it stays below the LLMem estimate.
+ *
  * All arithmetic is integer.  Intermediate values use unsigned __int128 so
  * that the overflow guard (status 3) is decided exactly.
  */
@@ -488,6 +497,131 @@ int oracle_list_digest(const oracle_config *c, uint64_t *a_out, uint64_t *b_out)
   return ST_OK;
 }
 
+/* ------------------------------------------------------------------------ */
+/* the DNNMem-style estimator of Section 3.1                                 */
+/* ------------------------------------------------------------------------ */
+#define DNN_ALIGN ((u128)512)                      /* PyTorch's tensor alignment (Section 3.1) */
+#define DNN_BUFFER ((u128)64 * 1024 * 1024)        /* constant buffer of the block manager (Section 3.1) */
+
+static u128 align512(u128 x) { return ceil_div(x, DNN_ALIGN) * DNN_ALIGN; }
+
+/* The procedure models one device without sharding: only the conventional method is accepted. */
+static int dnn_validate(const oracle_config *c) {
+  int st = validate_fields(c, 1);
+  if (st) return st;
+  if (c->method != M_CDP) return ST_COMBO;
+  return ST_OK;
+}
+
+/* Allocations in order (nothing is released during the forward pass of a fine-tuning
+ * iteration: the outputs are kept for backward): the constant buffer; the weight tensors
+ * as loaded, fp16, the embeddings first, then the Linear matrices layer by layer, then the
+ * vectors (norm weights, and norm and Linear biases where the model has them) layer by
+ * layer, the final norm, the lm_head; then the outputs of the forward pass as in phase 3
+ * of the LLMem list. */
+static void dnn_walk(const oracle_config *c, const sizes_t *z, sink_t *s) {
+  u128 H = (u128)c->hidden, F = (u128)c->ffn, bias = c->has_bias;
+  emit(s, +1, DNN_BUFFER);
+  emit(s, +1, B16 * z->tok_p);
+  if (c->pos_len > 0) emit(s, +1, B16 * z->pos_p);
+  for (int64_t l = 0; l < z->L; ++l)
+    for (int k = 0; k < z->K; ++k) emit(s, +1, B16 * (k < 4 ? z->hh_p : z->hf_p));
+  for (int64_t l = 0; l < z->L; ++l) {
+    /* two norm weights; with biases also two norm biases, the four attention biases and the
+     * bias of the feed-forward output, all of the hidden size; then the biases of the
+     * feed-forward inputs, of the feed-forward size */
+    int small = 2 + (int)bias * 7, wide = (int)bias * (z->K - 5);
+    for (int k = 0; k < small; ++k) emit(s, +1, B16 * H);
+    for (int k = 0; k < wide; ++k) emit(s, +1, B16 * F);
+  }
+  for (int k = 0; k < 1 + (int)bias; ++k) emit(s, +1, B16 * H);
+  emit(s, +1, z->lm_p);
+  for (int k = 0; k < z->e_n; ++k) emit(s, +1, z->out);
+  for (int64_t l = 0; l < z->L; ++l)
+    for (int k = 0; k < z->n_ops; ++k) emit(s, +1, op_size(z, k));
+  emit(s, +1, z->logit);
+  emit(s, +1, z->shift);
+  emit(s, +1, z->shift);
+}
+
+/* raw list of the second estimator (malloc'd, caller frees) with the byte guard */
+static int dnn_build(const oracle_config *c, int64_t **list_out, int64_t *n_out) {
+  *list_out = NULL;
+  *n_out = 0;
+  int st = dnn_validate(c);
+  if (st) return st;
+  sizes_t z;
+  compute_sizes(c, &z);
+  sink_t counter = {NULL, 0, 0};
+  dnn_walk(c, &z, &counter);
+  if (counter.overflow || (u128)counter.n >= COUNT_LIMIT) return ST_OVERFLOW;
+  int64_t *d = (int64_t *)malloc((size_t)counter.n * sizeof(int64_t));
+  if (!d) return -1;
+  sink_t writer = {d, 0, 0};
+  dnn_walk(c, &z, &writer);
+  u128 run = (u128)c->base_bytes;
+  int bad = 0;
+  for (int64_t k = 0; k < writer.n && !bad; ++k) {
+    run += align512((u128)d[k]);
+    if (run >= BYTES_LIMIT) bad = 1;
+  }
+  if (bad) {
+    free(d);
+    return ST_OVERFLOW;
+  }
+  *list_out = d;
+  *n_out = writer.n;
+  return ST_OK;
+}
+
+int oracle_dnn_event_count(const oracle_config *c, int64_t *count_out) {
+  int64_t *d;
+  int st = dnn_build(c, &d, count_out);
+  free(d);
+  return st;
+}
+
+int oracle_dnn_expand_events(const oracle_config *c, int64_t *dst, int64_t capacity) {
+  int64_t *d, n;
+  int st = dnn_build(c, &d, &n);
+  if (st) return st;
+  if (capacity < n) {
+    free(d);
+    return -1;
+  }
+  memcpy(dst, d, (size_t)n * sizeof(int64_t));
+  free(d);
+  return ST_OK;
+}
+
+/* every magnitude up to a multiple of 512 bytes, the sign kept */
+void oracle_dnn_round_events(int64_t *d, int64_t n) {
+  for (int64_t k = 0; k < n; ++k) {
+    if (d[k] >= 0)
+      d[k] = (int64_t)align512((u128)d[k]);
+    else
+      d[k] = -(int64_t)align512((u128)(-(i128)d[k]));
+  }
+}
+
+/* explicit list, alignment, linear scan; m_base is added as it is */
+int oracle_dnn_estimate(const oracle_config *c, int64_t *peak_out, int64_t *index_out, int64_t *count_out) {
+  *peak_out = -1;
+  *index_out = -1;
+  if (count_out) *count_out = 0;
+  int64_t *d, n;
+  int st = dnn_build(c, &d, &n);
+  if (st) return st;
+  oracle_dnn_round_events(d, n);
+  int64_t best, arg;
+  oracle_scan_peak(d, n, &best, &arg);
+  free(d);
+  *peak_out = c->base_bytes + best;
+  *index_out = arg;
+  if (count_out) *count_out = n;
+  return ST_OK;
+}
+
 /* inventory, for the pins: e_n, K, C, embed_p, other_p, lm_p (bytes), tok_p, pos_p, hh_p, hf_p */
 int oracle_inventory(const oracle_config *c, int64_t out[10]) {
   int st = oracle_validate(c);
@@ -683,7 +817,7 @@ int oracle_select_method_bisect(const oracle_config *shape, int64_t capacity, in
 /* ------------------------------------------------------------------------ */
 typedef struct {
   int kind; /* 0 estimate (level 1), 1 collapsed, 2 max batch (linear), 3 max batch (bisect),
-               4 select (linear), 5 select (bisect), 6 list checksums */
+               4 select (linear), 5 select (bisect), 6 list checksums, 7 second estimator */
   const oracle_config *cfg;
   int64_t n;
   const int64_t *caps;
@@ -712,6 +846,13 @@ static void run_one(job_t *j, int64_t i) {
     int64_t peak;
     int st = oracle_estimate_collapsed(c, &peak);
     j->peak[i] = peak;
+    if (j->status) j->status[i] = (uint8_t)st;
+  } else if (j->kind == 7) {
+    int64_t peak, idx, cnt;
+    int st = oracle_dnn_estimate(c, &peak, &idx, &cnt);
+    j->peak[i] = peak;
+    if (j->index) j->index[i] = idx;
+    if (j->count) j->count[i] = cnt;
     if (j->status) j->status[i] = (uint8_t)st;
   } else if (j->kind == 6) {
     int st = oracle_list_digest(c, &j->digest_a[i], &j->digest_b[i]);
@@ -771,6 +912,20 @@ void oracle_estimate_many(const oracle_config *cfg, int64_t n, int64_t *peak, in
   job_t j;
   memset(&j, 0, sizeof j);
   j.kind = level == 2 ? 1 : 0;
+  j.cfg = cfg;
+  j.n = n;
+  j.peak = peak;
+  j.index = index;
+  j.status = status;
+  j.count = count;
+  run_job(&j, nthreads);
+}
+
+void oracle_dnn_estimate_many(const oracle_config *cfg, int64_t n, int64_t *peak, int64_t *index,
+                              uint8_t *status, int64_t *count, int nthreads) {
+  job_t j;
+  memset(&j, 0, sizeof j);
+  j.kind = 7;
   j.cfg = cfg;
   j.n = n;
   j.peak = peak;

@@ -191,7 +191,7 @@ expand_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict
       i64* buf = ws.buf[parity];
       // a full chunk inside one segment may repeat the one before
       const bool alternating = seg < n && gs <= tb && tb + kExpChunk <= ge &&
-                               chunk_alternates(ar, ws, desc_seg, cfg, nullptr, seg, gs, ge, tb, round != 0, lane, g);
+                               chunk_alternates(ar, ws, desc_seg, cfg, seg, gs, ge, tb, round != 0, lane, g);
       if (alternating) {
         prepare_alternating<kExpStoresInFlight>(ar, keys, parity, buf, lane);
         if (ge == te) {
@@ -216,7 +216,7 @@ expand_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict
             for (i64 e = (span_lo > pos ? span_lo : pos); e < span_hi; ++e) buf[e - tb] = 0;
             break;
           }
-          ensure_desc(ws, desc_seg, cfg, nullptr, seg, gs, ge, round != 0, lane, g);
+          ensure_desc(ws, desc_seg, cfg, seg, gs, ge, round != 0, lane, g);
           const i64 piece_end = ge < te ? ge : te;
           const i64 e = span_lo > pos ? span_lo : pos;
           const i64 e_end = span_hi < piece_end ? span_hi : piece_end;

@@ -267,6 +267,7 @@ __device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy
 // One warp's private shared memory: two chunk buffers (filled, then handed to the
 // TMA engine while the other one is being filled) and the descriptor of the
 // segment the warp is currently inside.
+static_assert(sizeof(SegDesc) % 16 == 0, "descriptors are copied in 16-byte words");
 struct ExpandWarpSmem {
   alignas(128) i64 buf[2][kExpChunk];
   SegDesc desc;
@@ -291,23 +292,15 @@ struct BufferKeys {
   }
 };
 
-// Makes sure the warp's descriptor is that of segment `seg` (range [gs, ge)): copied by the
-// whole warp from `table` (one descriptor per configuration, built beforehand by one thread
-// each) when there is one, else built here by lane 0.
-static_assert(sizeof(SegDesc) % 16 == 0, "descriptors are copied in 16-byte words");
+// Makes sure the warp's descriptor is that of segment `seg` (range [gs, ge)): built by lane 0
+// when the warp enters the segment.
 __device__ __forceinline__ void ensure_desc(ExpandWarpSmem& ws, i64& desc_seg, const llmem_config* __restrict__ cfg,
-                                            const SegDesc* __restrict__ table, i64 seg, i64 gs, i64 ge, bool round,
-                                            int lane, const Guard& g) {
+                                            i64 seg, i64 gs, i64 ge, bool round, int lane, const Guard& g) {
   if (desc_seg != seg) {
     __syncwarp();  // every lane is done with the previous descriptor
-    if (!in_bounds(seg >= 0 && seg < g.n, g, kSiteDescriptor)) {
-      if (lane == 0) ws.desc.invalid = 1;  // the segment is written as zeros
-    } else if (table) {
-      const int4* src = reinterpret_cast<const int4*>(table + seg);
-      int4* dst = reinterpret_cast<int4*>(&ws.desc);
-      for (int k = lane; k < (int)(sizeof(SegDesc) / 16); k += 32) dst[k] = __ldg(src + k);
-    } else if (lane == 0) {
-      build_desc(ws.desc, cfg + seg, gs, ge, round);
+    if (lane == 0) {
+      if (in_bounds(seg >= 0 && seg < g.n, g, kSiteDescriptor)) build_desc(ws.desc, cfg + seg, gs, ge, round);
+      else ws.desc.invalid = 1;  // the segment is written as zeros
     }
     __syncwarp();
     desc_seg = seg;
@@ -317,11 +310,10 @@ __device__ __forceinline__ void ensure_desc(ExpandWarpSmem& ws, i64& desc_seg, c
 // Does the full chunk [tb, tb + kExpChunk), which lies inside segment `seg`, consist of one
 // run of period 1 or 2?  Updates `ar` when it enters a new such run.
 __device__ __forceinline__ bool chunk_alternates(AlternatingRun& ar, ExpandWarpSmem& ws, i64& desc_seg,
-                                                 const llmem_config* __restrict__ cfg,
-                                                 const SegDesc* __restrict__ table, i64 seg, i64 gs, i64 ge, i64 tb,
+                                                 const llmem_config* __restrict__ cfg, i64 seg, i64 gs, i64 ge, i64 tb,
                                                  bool round, int lane, const Guard& g) {
   if (tb + kExpChunk <= ar.end) return true;
-  ensure_desc(ws, desc_seg, cfg, table, seg, gs, ge, round, lane, g);
+  ensure_desc(ws, desc_seg, cfg, seg, gs, ge, round, lane, g);
   if (ws.desc.invalid) return false;
   int r, o, it;
   locate(ws.desc, (u32)(tb - gs), &r, &o, &it);

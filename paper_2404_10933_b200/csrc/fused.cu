@@ -165,7 +165,7 @@ __global__ void __launch_bounds__(kFusedWarps * 32)
 expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict__ offsets, i64 total,
                    i64* __restrict__ out, i64 n_blocks, i64 kappa, int bulk_ok, i64* __restrict__ peak_out,
                    i64* __restrict__ index_out, i64* __restrict__ bounds, WarpPartials* __restrict__ partials,
-                   unsigned long long* __restrict__ work_counter, const SegDesc* __restrict__ table) {
+                   unsigned long long* __restrict__ work_counter) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   ExpandWarpSmem& ws = reinterpret_cast<ExpandWarpSmem*>(smem_raw)[warp];
@@ -200,7 +200,7 @@ expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __res
       i64* buf = ws.buf[parity];
       // a full chunk inside one segment may repeat the one before
       const bool alternating = seg < n && gs <= tb && tb + kExpChunk <= ge &&
-                               chunk_alternates(ar, ws, desc_seg, cfg, table, seg, gs, ge, tb, kRoundList, lane, g);
+                               chunk_alternates(ar, ws, desc_seg, cfg, seg, gs, ge, tb, kRoundList, lane, g);
       if (alternating) {
         prepare_alternating<kFusedStoresInFlight>(ar, keys, parity, buf, lane);
         folder.add_uniform(fold_alternating_chunk(ev<!kRoundList>(ar.x0), ev<!kRoundList>(ar.x1), tb), lane);
@@ -227,7 +227,7 @@ expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __res
             for (i64 e = (span_lo > pos ? span_lo : pos); e < span_hi; ++e) buf[e - tb] = 0;
             break;
           }
-          ensure_desc(ws, desc_seg, cfg, table, seg, gs, ge, kRoundList, lane, g);
+          ensure_desc(ws, desc_seg, cfg, seg, gs, ge, kRoundList, lane, g);
           const i64 piece_end = ge < te ? ge : te;
           const i64 e = span_lo > pos ? span_lo : pos;
           const i64 e_end = span_hi < piece_end ? span_hi : piece_end;
@@ -594,7 +594,7 @@ extern "C" llmem_status llmem_expand_scan(const llmem_config* cfg, int64_t n, co
   expand_scan_kernel<ROUND, kFusedWarpsLong><<<grid, kFusedWarpsLong * 32, smem, s>>>(                           \
       cfg, n, reinterpret_cast<const i64*>(offsets), total_events, reinterpret_cast<i64*>(delta_out), warps,    \
       kFusedSegmentCost, bulk_ok, reinterpret_cast<i64*>(peak_out), reinterpret_cast<i64*>(peak_index_out),      \
-      bounds, partials, work_counter, nullptr)
+      bounds, partials, work_counter)
     if (round) LLMEM_LAUNCH_FUSED(true); else LLMEM_LAUNCH_FUSED(false);
 #undef LLMEM_LAUNCH_FUSED
     llmem_status st = check_launch("llmem_expand_scan");

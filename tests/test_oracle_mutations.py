@@ -67,6 +67,14 @@ MUTANTS = [
      "if (best_cs < 0 || waste <= best_waste) {", 1),
     ("chunk_search_floor", "u128 waste = ceil_div(z.other_p, cs) * cs - z.other_p;",
      "u128 waste = (z.other_p / cs + 1) * cs - z.other_p;", 1),
+    ("dnn_align_down", "static u128 align512(u128 x) { return ceil_div(x, DNN_ALIGN) * DNN_ALIGN; }",
+     "static u128 align512(u128 x) { return x / DNN_ALIGN * DNN_ALIGN; }", 1),
+    ("dnn_buffer_dropped", "  emit(s, +1, DNN_BUFFER);\n", "", 1),
+    ("dnn_weights_fp32", "emit(s, +1, B16 * (k < 4 ? z->hh_p : z->hf_p));", "emit(s, +1, B32 * (k < 4 ? z->hh_p : z->hf_p));", 1),
+    ("dnn_bias_count", "int small = 2 + (int)bias * 7, wide = (int)bias * (z->K - 5);", "int small = 2 + (int)bias * 6, wide = (int)bias * (z->K - 5);", 1),
+    ("dnn_operator_kind", "for (int k = 0; k < z->n_ops; ++k) emit(s, +1, op_size(z, k));\n  emit(s, +1, z->logit);",
+     "for (int k = 0; k < z->n_ops; ++k) emit(s, +1, op_size(z, z->op_kind[k]));\n  emit(s, +1, z->logit);", 1),
+    ("dnn_accepts_sharded_methods", "  if (c->method != M_CDP) return ST_COMBO;\n  return ST_OK;", "  return ST_OK;", 1),
     ("frees_forgotten_gather", "      for (int64_t j = 0; j < C; ++j) emit(s, -1, z->gat_chunk);\n", "", 1),
 ]
 
