@@ -623,6 +623,7 @@ def leg_estimate(llmem, torch, steps, warmup, n=None, repeat=16):
     events = int(llmem.event_counts(dev)[0][-1].item())
     ms, clocks = _timed_steps(torch, lambda: llmem.estimate_batch(dev), steps, warmup, flush)
     ms_big, _ = _timed_steps(torch, lambda: llmem.estimate_batch(big), max(3, steps // 4), warmup, flush)
+    ms_dnn, _ = _timed_steps(torch, lambda: llmem.estimate_batch(dev, estimator="dnnmem"), max(3, steps // 4), warmup, flush)
     roof = _alu_roofline(torch, llmem, {"estimate_kernel": n}, ms, clocks)
     roof_big = _alu_roofline(torch, llmem, {"estimate_kernel": n * repeat}, ms_big, clocks)
     return {"metric": "configs per second (fused estimate)", "value": n / (ms * 1e-3), "unit": "configs/s",
@@ -634,6 +635,9 @@ def leg_estimate(llmem, torch, steps, warmup, n=None, repeat=16):
             "repeated": {"configs": n * repeat, "ms_per_step": ms_big, "value": n * repeat / (ms_big * 1e-3),
                          "unit": "configs/s", "frac": roof_big["frac"],
                          "frac_of_measured_add_mad": roof_big["frac_of_measured_add_mad"]},
+            "second_estimator": {"what": "the DNNMem-style estimate of Section 3.1 on the same records (those of another "
+                                         "method than the conventional one get status 2)",
+                                 "ms_per_step": ms_dnn, "value": n / (ms_dnn * 1e-3), "unit": "configs/s"},
             "gpu_launches": steps, "clocks": clocks}
 
 

@@ -96,6 +96,21 @@ enum { LLMEM_OP_ESTIMATE = 0, LLMEM_OP_EVENT_COUNTS = 1, LLMEM_OP_EXPAND = 2, LL
 #define LLMEM_SELECT_ALLZERO 1u /* llmem_select_method: offload only if every score is 0 */
 #define LLMEM_FUSE_ROUND 2u     /* llmem_expand_events: write page-rounded deltas;
                                    llmem_scan_peak: round each delta while reading */
+/* Section 3.1: estimate as the DNNMem-style procedure does that the paper implements for
+ * comparison, instead of LLMem: one device without sharding (method must be LLMEM_METHOD_CDP,
+ * else LLMEM_CFG_COMBO; gpu_n, tp_n, chunk_elems and iters play no part), the weight tensors
+ * as loaded (fp16, the lm_head in lm_bytes) and a constant 64 MB buffer, then the outputs of
+ * the forward pass (embedding outputs, layer outputs or, with act_mode 1, every operator
+ * output, logits, two shifted copies), every tensor aligned to 512 bytes instead of the 2 MiB
+ * page.  The list has no frees: its peak is m_base + its total.  Event order: buffer, token
+ * (position) embedding, the Linear matrices layer by layer, the vectors layer by layer (norm
+ * weights, then norm / attention / feed-forward output biases, then feed-forward input
+ * biases), final norm, lm_head, forward outputs.  Accepted by llmem_estimate_batch,
+ * llmem_event_counts(_static), llmem_expand_events (LLMEM_FUSE_ROUND then aligns to 512 bytes),
+ * llmem_expand_scan (only together with LLMEM_FUSE_ROUND) and llmem_scan_peak (then cfg adds
+ * m_base alone; not together with LLMEM_FUSE_ROUND, which rounds to the 2 MiB page); refused
+ * by llmem_max_batch and llmem_select_method (Algorithm 1 is LLMem's). */
+#define LLMEM_ESTIMATOR_DNNMEM 4u
 
 /* Bytes of scratch the operation needs for n configurations and total_events
  * events (0 where it needs none; such calls accept scratch = NULL).  For

@@ -31,7 +31,16 @@ OK, ERR_ARG, ERR_SCRATCH, ERR_CUDA, ERR_TIMEOUT, ERR_CHECK = 0, 1, 2, 3, 4, 5
 OP_ESTIMATE, OP_EVENT_COUNTS, OP_EXPAND, OP_ROUND, OP_SCAN_PEAK, OP_MAX_BATCH, OP_SELECT, OP_EXPAND_SCAN = range(8)
 SELECT_ALLZERO = 1
 FUSE_ROUND = 2
+ESTIMATOR_DNNMEM = 4   # the DNNMem-style estimator of Section 3.1 instead of LLMem
 METHOD_OFFLOAD = 4
+
+
+def _estimator_flag(estimator: str) -> int:
+    if estimator == "llmem":
+        return 0
+    if estimator == "dnnmem":
+        return ESTIMATOR_DNNMEM
+    raise ValueError("estimator must be 'llmem' or 'dnnmem'")
 
 EXPORTS = (
     "llmem_scratch_bytes", "llmem_estimate_batch", "llmem_event_counts", "llmem_expand_events",
@@ -149,20 +158,21 @@ def _scratch(op: int, n: int, total: int, device):
     return torch.empty(nbytes, dtype=torch.uint8, device=device), nbytes
 
 
-def estimate_batch(cfg, *, want_index: bool = True, want_status: bool = True, stream=None):
-    """Fused estimate.  Returns dict(peak[n] int64, index[n] int64 | None, status[n] uint8 | None)."""
+def estimate_batch(cfg, *, want_index: bool = True, want_status: bool = True, stream=None, estimator: str = "llmem"):
+    """Fused estimate.  ``estimator="dnnmem"`` evaluates the DNNMem-style procedure of the paper's
+    Section 3.1 instead.  Returns dict(peak[n] int64, index[n] int64 | None, status[n] uint8 | None)."""
     torch = _torch()
     cfg = _as_cfg(cfg)
     n = cfg.shape[0]
     peak = torch.empty(n, dtype=torch.int64, device=cfg.device)
     index = torch.empty(n, dtype=torch.int64, device=cfg.device) if want_index else None
     status = torch.empty(n, dtype=torch.uint8, device=cfg.device) if want_status else None
-    _check(lib().llmem_estimate_batch(_ptr(cfg), n, _ptr(peak), _ptr(index), _ptr(status), None, 0, 0,
-                                      _stream_ptr(stream)))
+    _check(lib().llmem_estimate_batch(_ptr(cfg), n, _ptr(peak), _ptr(index), _ptr(status), None, 0,
+                                      _estimator_flag(estimator), _stream_ptr(stream)))
     return {"peak": peak, "index": index, "status": status}
 
 
-def event_counts(cfg, *, want_status: bool = True, stream=None):
+def event_counts(cfg, *, want_status: bool = True, stream=None, estimator: str = "llmem"):
     """Returns (offsets[n+1] int64 exclusive scan of event counts, status[n] | None)."""
     torch = _torch()
     cfg = _as_cfg(cfg)
@@ -170,8 +180,8 @@ def event_counts(cfg, *, want_status: bool = True, stream=None):
     offsets = torch.empty(n + 1, dtype=torch.int64, device=cfg.device)
     status = torch.empty(n, dtype=torch.uint8, device=cfg.device) if want_status else None
     scratch, nbytes = _scratch(OP_EVENT_COUNTS, n, 0, cfg.device)
-    _check(lib().llmem_event_counts(_ptr(cfg), n, _ptr(offsets), _ptr(status), _ptr(scratch), nbytes, 0,
-                                    _stream_ptr(stream)))
+    _check(lib().llmem_event_counts(_ptr(cfg), n, _ptr(offsets), _ptr(status), _ptr(scratch), nbytes,
+                                    _estimator_flag(estimator), _stream_ptr(stream)))
     return offsets, status
 
 
@@ -198,7 +208,7 @@ def event_counts_static(cfg, offsets_out, status_out=None, *, stream=None):
 
 
 def expand_events(cfg, offsets, total_events: Optional[int] = None, *, fuse_round: bool = False,
-                  out=None, scratch=None, stream=None):
+                  out=None, scratch=None, stream=None, estimator: str = "llmem"):
     """Materialise the signed event list.  ``total_events`` defaults to ``offsets[-1]`` (one
     device-to-host read).  ``scratch`` (optional, 256 bytes) is allocated when not given."""
     torch = _torch()
@@ -216,7 +226,8 @@ def expand_events(cfg, offsets, total_events: Optional[int] = None, *, fuse_roun
     else:
         _check_buffer(scratch, "scratch", torch.uint8, 0, cfg.device)
     _check(lib().llmem_expand_events(_ptr(cfg), n, _ptr(offsets), total_events, _ptr(out), _ptr(scratch),
-                                     scratch.numel(), FUSE_ROUND if fuse_round else 0, _stream_ptr(stream)))
+                                     scratch.numel(), (FUSE_ROUND if fuse_round else 0) | _estimator_flag(estimator),
+                                     _stream_ptr(stream)))
     return out[:total_events] if out.numel() != total_events else out
 
 
@@ -227,7 +238,7 @@ def round_events(delta, stream=None):
 
 
 def scan_peak(delta, offsets, cfg=None, *, fuse_round: bool = False, want_index: bool = True,
-              scratch=None, stream=None, check_status: bool = False):
+              scratch=None, stream=None, check_status: bool = False, estimator: str = "llmem"):
     """Segmented prefix-sum + max.  Returns dict(peak[n], index[n] | None, scratch)."""
     torch = _torch()
     if not isinstance(offsets, torch.Tensor) or not offsets.is_cuda:
@@ -246,7 +257,7 @@ def scan_peak(delta, offsets, cfg=None, *, fuse_round: bool = False, want_index:
         _check_buffer(scratch, "scratch", torch.uint8, 0, offsets.device)
         nbytes = scratch.numel()
     _check(lib().llmem_scan_peak(_ptr(delta), _ptr(offsets), n, total, _ptr(cfg), _ptr(peak), _ptr(index),
-                                 _ptr(scratch), nbytes, FUSE_ROUND if fuse_round else 0,
+                                 _ptr(scratch), nbytes, (FUSE_ROUND if fuse_round else 0) | _estimator_flag(estimator),
                                  _stream_ptr(stream)))
     if check_status:
         _check(lib().llmem_scratch_status(_ptr(scratch), _stream_ptr(stream)))
@@ -254,7 +265,8 @@ def scan_peak(delta, offsets, cfg=None, *, fuse_round: bool = False, want_index:
 
 
 def expand_scan(cfg, offsets, total_events: Optional[int] = None, *, fuse_round: bool = True, out=None,
-                want_index: bool = True, scratch=None, stream=None, peak_out=None, index_out=None):
+                want_index: bool = True, scratch=None, stream=None, peak_out=None, index_out=None,
+                estimator: str = "llmem"):
     """Materialise the event list and compute the peaks in one pass (the list is written
     once and not read back).  ``peak_out`` / ``index_out`` ([n] int64) receive the results when
     given.  Returns dict(delta, peak[n], index[n] | None, scratch)."""
@@ -281,7 +293,8 @@ def expand_scan(cfg, offsets, total_events: Optional[int] = None, *, fuse_round:
         _check_buffer(scratch, "scratch", torch.uint8, 0, cfg.device)
         nbytes = scratch.numel()
     _check(lib().llmem_expand_scan(_ptr(cfg), n, _ptr(offsets), total_events, _ptr(out), _ptr(peak), _ptr(index),
-                                   _ptr(scratch), nbytes, FUSE_ROUND if fuse_round else 0, _stream_ptr(stream)))
+                                   _ptr(scratch), nbytes, (FUSE_ROUND if fuse_round else 0) | _estimator_flag(estimator),
+                                   _stream_ptr(stream)))
     delta = out[:total_events] if out.numel() != total_events else out
     return {"delta": delta, "peak": peak, "index": index, "scratch": scratch}
 
@@ -372,16 +385,18 @@ def _caps(capacities, device):
     return caps
 
 
-def estimate_materialized(cfg, *, fuse_round: bool = True, stream=None):
+def estimate_materialized(cfg, *, fuse_round: bool = True, stream=None, estimator: str = "llmem"):
     """The materialised path end to end: event counts -> expansion -> (rounding) ->
     segmented scan.  Returns dict(peak, index, status, offsets, total_events)."""
     cfg = _as_cfg(cfg)
-    offsets, status = event_counts(cfg, stream=stream)
+    if estimator != "llmem" and not fuse_round:
+        raise ValueError("the separate rounding pass rounds to the 2 MiB page: use fuse_round with this estimator")
+    offsets, status = event_counts(cfg, stream=stream, estimator=estimator)
     total = int(offsets[-1].item())
-    delta = expand_events(cfg, offsets, total, fuse_round=fuse_round, stream=stream)
+    delta = expand_events(cfg, offsets, total, fuse_round=fuse_round, stream=stream, estimator=estimator)
     if not fuse_round:
         round_events(delta, stream=stream)
-    r = scan_peak(delta, offsets, cfg, stream=stream)
+    r = scan_peak(delta, offsets, cfg, stream=stream, estimator=estimator)
     return {"peak": r["peak"], "index": r["index"], "status": status, "offsets": offsets,
             "total_events": total}
 

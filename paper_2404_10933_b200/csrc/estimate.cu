@@ -206,6 +206,19 @@ __device__ __forceinline__ void estimate_one(const Cfg& f, i64* pk_out, i64* ix_
 // tenth fewer warp instructions -- but the kernel waits on dependent 64-bit arithmetic rather
 // than on issue slots, and the barriers of the sort cost more than the idle lanes: 0.74 ms
 // instead of 0.69 ms for 2^24 configurations.)
+// The same for the DNNMem-style estimator of Section 3.1: the list only grows, so the peak is
+// the total and sits at the last event of non-zero size (the second shifted copy, or the
+// logits when the sequence has one token).
+__device__ __forceinline__ void dnn_estimate_one(const Cfg& f, i64* pk_out, i64* ix_out, int* st_out) {
+  DnnPlan p;
+  u64 peak;
+  const int st = dnn_full_status(f, &p, &peak);
+  *st_out = st;
+  *pk_out = st == LLMEM_CFG_OK ? (i64)peak : -1;
+  *ix_out = st == LLMEM_CFG_OK ? (i64)(p.shift > 0 ? p.count - 1 : p.count - 3) : -1;
+}
+
+template <bool kDnn>
 __global__ void __launch_bounds__(LLMEM_EST_THREADS, LLMEM_EST_MIN_CTAS)
 estimate_kernel(const llmem_config* __restrict__ cfg, i64 n, i64* __restrict__ peak_out,
                 i64* __restrict__ index_out, uint8_t* __restrict__ status_out) {
@@ -213,7 +226,8 @@ estimate_kernel(const llmem_config* __restrict__ cfg, i64 n, i64* __restrict__ p
     const Cfg f = load_cfg(cfg + i);
     i64 pk, ix;
     int st;
-    estimate_one(f, &pk, &ix, &st);
+    if (kDnn) dnn_estimate_one(f, &pk, &ix, &st);
+    else estimate_one(f, &pk, &ix, &st);
     peak_out[i] = pk;
     if (index_out) index_out[i] = ix;
     if (status_out) status_out[i] = (uint8_t)st;
@@ -412,7 +426,7 @@ extern "C" llmem_status llmem_estimate_batch(const llmem_config* cfg, int64_t n,
                                              int64_t* peak_index_out, uint8_t* status_out,
                                              void* scratch, size_t scratch_bytes, uint32_t flags,
                                              void* cuda_stream) {
-  (void)scratch; (void)scratch_bytes; (void)flags;
+  (void)scratch; (void)scratch_bytes;
   clear_error();
   TraceRange trace("llmem_estimate_batch");
   if (n < 0) { set_error("llmem_estimate_batch: n < 0"); return LLMEM_ERR_ARG; }
@@ -422,8 +436,14 @@ extern "C" llmem_status llmem_estimate_batch(const llmem_config* cfg, int64_t n,
     set_error("llmem_estimate_batch: cfg must be 16-byte and outputs 8-byte aligned");
     return LLMEM_ERR_ARG;
   }
-  estimate_kernel<<<grid_for(n, LLMEM_EST_THREADS, LLMEM_EST_GRID_CTAS), LLMEM_EST_THREADS, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-      cfg, n, reinterpret_cast<i64*>(peak_out), reinterpret_cast<i64*>(peak_index_out), status_out);
+  const int grid = grid_for(n, LLMEM_EST_THREADS, LLMEM_EST_GRID_CTAS);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (flags & LLMEM_ESTIMATOR_DNNMEM)
+    estimate_kernel<true><<<grid, LLMEM_EST_THREADS, 0, s>>>(cfg, n, reinterpret_cast<i64*>(peak_out),
+                                                             reinterpret_cast<i64*>(peak_index_out), status_out);
+  else
+    estimate_kernel<false><<<grid, LLMEM_EST_THREADS, 0, s>>>(cfg, n, reinterpret_cast<i64*>(peak_out),
+                                                              reinterpret_cast<i64*>(peak_index_out), status_out);
   return check_launch("llmem_estimate_batch");
 }
 
@@ -441,9 +461,10 @@ extern "C" llmem_status llmem_max_batch(const llmem_config* shape, int64_t n,
                                         const int64_t* capacity_bytes, int32_t n_cap, int32_t bmax,
                                         int32_t* bs_out, uint8_t* status_out, void* scratch,
                                         size_t scratch_bytes, uint32_t flags, void* cuda_stream) {
-  (void)scratch; (void)scratch_bytes; (void)flags;
+  (void)scratch; (void)scratch_bytes;
   clear_error();
   TraceRange trace("llmem_max_batch");
+  if (flags & LLMEM_ESTIMATOR_DNNMEM) { set_error("llmem_max_batch: Algorithm 1 searches with the LLMem estimate only"); return LLMEM_ERR_ARG; }
   llmem_status st = check_search_args("llmem_max_batch", shape, n, capacity_bytes, n_cap, bmax);
   if (st != LLMEM_OK || n == 0 || n_cap == 0) return st;
   if (!bs_out || !aligned_to(bs_out, 4)) { set_error("llmem_max_batch: bs_out is required"); return LLMEM_ERR_ARG; }
@@ -460,6 +481,7 @@ extern "C" llmem_status llmem_select_method(const llmem_config* shape, int64_t n
   (void)scratch; (void)scratch_bytes;
   clear_error();
   TraceRange trace("llmem_select_method");
+  if (flags & LLMEM_ESTIMATOR_DNNMEM) { set_error("llmem_select_method: Algorithm 1 selects with the LLMem estimate only"); return LLMEM_ERR_ARG; }
   llmem_status st = check_search_args("llmem_select_method", shape, n, capacity_bytes, n_cap, bmax);
   if (st != LLMEM_OK || n == 0 || n_cap == 0) return st;
   if (!method_out || !batch_out) { set_error("llmem_select_method: method_out and batch_out are required"); return LLMEM_ERR_ARG; }

@@ -50,6 +50,7 @@ __device__ __forceinline__ u64 block_exclusive_scan(u64 v, u64* total, u64* smem
 }
 
 // Pass 1: counts, CTA-local exclusive offsets, per-CTA totals.
+template <bool kDnn>
 __global__ void __launch_bounds__(kCountThreads)
 count_kernel(const llmem_config* __restrict__ cfg, i64 n, i64* __restrict__ offsets,
              uint8_t* __restrict__ status_out, u64* __restrict__ block_sums) {
@@ -64,7 +65,13 @@ count_kernel(const llmem_config* __restrict__ cfg, i64 n, i64* __restrict__ offs
     if (i < n) {
       Cfg f = load_cfg(cfg + i);
       int st = check_fields(f, true, true);
-      if (st == LLMEM_CFG_OK) {
+      if (kDnn) {
+        // the list of the second estimator (Section 3.1)
+        DnnPlan p;
+        u64 peak;
+        st = dnn_full_status(f, &p, &peak);
+        if (st == LLMEM_CFG_OK) c[j] = p.count;
+      } else if (st == LLMEM_CFG_OK) {
         Plan p = make_plan(f, f.method);
         st = p.status;
         if (st == LLMEM_CFG_OK) {
@@ -166,7 +173,8 @@ slab_bounds_kernel(const i64* __restrict__ offsets, i64 n, i64 max_events, i64 f
 // store is issued.
 __global__ void __launch_bounds__(kExpThreads)
 expand_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict__ offsets, i64 total,
-              i64* __restrict__ out, i64 n_blocks, i64 kappa, int round, int bulk_ok,
+              i64* __restrict__ out, i64 n_blocks, i64 kappa, int round /* bit 0: rounded values, bit 1: second estimator */,
+              int bulk_ok,
               unsigned long long* __restrict__ work_counter, u32* __restrict__ status_word) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -191,7 +199,7 @@ expand_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict
       i64* buf = ws.buf[parity];
       // a full chunk inside one segment may repeat the one before
       const bool alternating = seg < n && gs <= tb && tb + kExpChunk <= ge &&
-                               chunk_alternates(ar, ws, desc_seg, cfg, seg, gs, ge, tb, round != 0, lane, g);
+                               chunk_alternates(ar, ws, desc_seg, cfg, seg, gs, ge, tb, round, lane, g);
       if (alternating) {
         prepare_alternating<kExpStoresInFlight>(ar, keys, parity, buf, lane);
         if (ge == te) {
@@ -216,7 +224,7 @@ expand_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict
             for (i64 e = (span_lo > pos ? span_lo : pos); e < span_hi; ++e) buf[e - tb] = 0;
             break;
           }
-          ensure_desc(ws, desc_seg, cfg, seg, gs, ge, round != 0, lane, g);
+          ensure_desc(ws, desc_seg, cfg, seg, gs, ge, round, lane, g);
           const i64 piece_end = ge < te ? ge : te;
           const i64 e = span_lo > pos ? span_lo : pos;
           const i64 e_end = span_hi < piece_end ? span_hi : piece_end;
@@ -284,7 +292,6 @@ using namespace llmem;
 extern "C" llmem_status llmem_event_counts(const llmem_config* cfg, int64_t n, int64_t* offsets_out,
                                            uint8_t* status_out, void* scratch, size_t scratch_bytes,
                                            uint32_t flags, void* cuda_stream) {
-  (void)flags;
   clear_error();
   TraceRange trace("llmem_event_counts");
   if (n < 0) { set_error("llmem_event_counts: n < 0"); return LLMEM_ERR_ARG; }
@@ -302,7 +309,10 @@ extern "C" llmem_status llmem_event_counts(const llmem_config* cfg, int64_t n, i
   }
   u64* block_sums = reinterpret_cast<u64*>(static_cast<unsigned char*>(scratch) + kScratchHeader);
   const i64 nblocks = (n + kCountBlock - 1) / kCountBlock;
-  count_kernel<<<(unsigned)nblocks, kCountThreads, 0, s>>>(cfg, n, reinterpret_cast<i64*>(offsets_out), status_out, block_sums);
+  if (flags & LLMEM_ESTIMATOR_DNNMEM)
+    count_kernel<true><<<(unsigned)nblocks, kCountThreads, 0, s>>>(cfg, n, reinterpret_cast<i64*>(offsets_out), status_out, block_sums);
+  else
+    count_kernel<false><<<(unsigned)nblocks, kCountThreads, 0, s>>>(cfg, n, reinterpret_cast<i64*>(offsets_out), status_out, block_sums);
   scan_block_sums_kernel<<<1, kCountThreads, 0, s>>>(block_sums, nblocks);
   i64 blocks3 = (n + 1 + 255) / 256;
   const i64 cap3 = (i64)sm_count() * 8;
@@ -355,7 +365,6 @@ static llmem_status static_sums_address(u64** out) {
 
 extern "C" llmem_status llmem_event_counts_static(const llmem_config* cfg, int64_t n, int64_t* offsets_out,
                                                   uint8_t* status_out, uint32_t flags, void* cuda_stream) {
-  (void)flags;
   clear_error();
   if (n < 0) { set_error("llmem_event_counts_static: n < 0"); return LLMEM_ERR_ARG; }
   if (n > kStaticMaxConfigs) {
@@ -377,7 +386,10 @@ extern "C" llmem_status llmem_event_counts_static(const llmem_config* cfg, int64
   // rewrites them and writes entry [nblocks], and no pass reads an entry this call has not
   // written.  What an earlier call left beyond nblocks is never looked at.
   const i64 nblocks = (n + kCountBlock - 1) / kCountBlock;
-  count_kernel<<<(unsigned)nblocks, kCountThreads, 0, s>>>(cfg, n, reinterpret_cast<i64*>(offsets_out), status_out, block_sums);
+  if (flags & LLMEM_ESTIMATOR_DNNMEM)
+    count_kernel<true><<<(unsigned)nblocks, kCountThreads, 0, s>>>(cfg, n, reinterpret_cast<i64*>(offsets_out), status_out, block_sums);
+  else
+    count_kernel<false><<<(unsigned)nblocks, kCountThreads, 0, s>>>(cfg, n, reinterpret_cast<i64*>(offsets_out), status_out, block_sums);
   scan_block_sums_kernel<<<1, kCountThreads, 0, s>>>(block_sums, nblocks);
   i64 blocks3 = (n + 1 + 255) / 256;
   const i64 cap3 = (i64)sm_count() * 8;
@@ -419,12 +431,14 @@ extern "C" llmem_status llmem_expand_events(const llmem_config* cfg, int64_t n, 
     return LLMEM_ERR_ARG;
   }
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  // bit 0: values page-rounded (aligned to 512 bytes under the second estimator); bit 1: the second estimator's list
+  const int round_bits = ((flags & LLMEM_FUSE_ROUND) ? 1 : 0) | ((flags & LLMEM_ESTIMATOR_DNNMEM) ? 2 : 0);
   if (short_segment_list(n, total_events) && scratch && aligned_to(scratch, 256) &&
       scratch_bytes >= expand_scan_scratch_bytes(n, total_events)) {
     // lists of short segments: every segment written by its owner, a lane or a warp
     if (cudaMemsetAsync(scratch, 0, kScratchHeader, s) != cudaSuccess) return check_launch("llmem_expand_events (memset)");
     return expand_by_owners(cfg, n, reinterpret_cast<const i64*>(offsets), total_events, reinterpret_cast<i64*>(delta_out),
-                            (flags & LLMEM_FUSE_ROUND) != 0, false, nullptr, nullptr, scratch, nullptr, s);
+                            round_bits, false, nullptr, nullptr, scratch, nullptr, s);
   }
   const size_t smem = sizeof(ExpandWarpSmem) * kExpWarps;
   static thread_local int configured_dev = -1;
@@ -451,7 +465,7 @@ extern "C" llmem_status llmem_expand_events(const llmem_config* cfg, int64_t n, 
   const i64 grid = (grid_warps + kExpWarps - 1) / kExpWarps;
   expand_kernel<<<(unsigned)grid, kExpThreads, smem, s>>>(
       cfg, n, reinterpret_cast<const i64*>(offsets), total_events, reinterpret_cast<i64*>(delta_out),
-      blocks, kExpSegmentCost, (flags & LLMEM_FUSE_ROUND) ? 1 : 0, aligned_to(delta_out, 16) ? 1 : 0, work_counter,
+      blocks, kExpSegmentCost, round_bits, aligned_to(delta_out, 16) ? 1 : 0, work_counter,
       status_word);
   return check_launch("llmem_expand_events");
 }

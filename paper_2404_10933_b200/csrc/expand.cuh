@@ -94,7 +94,69 @@ __device__ __forceinline__ u32 layer_code(bool gated, bool reversed, int* n_ops)
 // Not inlined: the kernels reach it from two places, and the warps of an SM, each somewhere
 // else in a long kernel, already miss the instruction cache more than anything else
 // ("no instruction" is the top stall on lists of short segments).
-static __device__ __noinline__ void build_desc(SegDesc& d, const llmem_config* __restrict__ cfg, i64 gstart, i64 gend, bool round) {
+// Fills in where each run starts inside its group and which run follows it.
+__device__ __forceinline__ void link_runs(SegDesc& d) {
+  d.run[1].start = 2;
+  for (int r = kDynFirst + 1; r <= kDynLast; ++r) d.run[r].start = d.run[r - 1].start + d.run[r - 1].cnt;
+  for (int r = kOsFirst + 1; r <= kOsLast; ++r) d.run[r].start = d.run[r - 1].start + d.run[r - 1].cnt;
+  // in the first iteration the optimizer states follow the frees
+  for (int r = 0; r < kRuns; ++r) {
+    i64 links = 0;
+    for (int later = 0; later < 2; ++later) {
+      int nx = r;
+      for (int guard = 0; guard < 2 * kRuns; ++guard) {
+        if (nx == kDynLast) nx = later ? kDynFirst : kOsFirst;
+        else if (nx == kOsLast) nx = kDynFirst;
+        else ++nx;
+        if (d.run[nx].cnt > 0) break;
+      }
+      links |= (i64)nx << (8 * later);
+    }
+    d.run[r].links = links;
+  }
+}
+
+// The list of the DNNMem-style estimator (Section 3.1) in the same form: runs 0-1 the buffer
+// with the token embedding, then the position embedding; the "iteration" group holds the
+// Linear matrices, the vectors, the final norm, the lm_head and the forward outputs, and is
+// passed once; there are no optimizer states and no frees.  `f` has passed check_fields.
+__device__ __forceinline__ void build_dnn_runs(SegDesc& d, const Cfg& f, bool round) {
+  const DnnPlan p = make_dnn_plan(f);
+  if (p.status != LLMEM_CFG_OK) return;
+  if (p.out >= kSat || p.logit >= kSat || p.shift >= kSat || p.attn >= kSat || p.ffn >= kSat) return;
+  d.invalid = 0;
+#define LLMEM_W(x) ((i64)(round ? align512(x) : (x)))
+  const int L = p.L;
+  set_run(d.run[0], 2, 2, 1u << 2, (i64)kDnnBuffer, LLMEM_W(p.tok), 0);
+  set_const_run(d.run[1], p.has_pos, LLMEM_W(p.pos));
+  set_run(d.run[2], p.K * L, p.K, p.K == 7 ? 0x1500u : 0x0500u, LLMEM_W(p.hh), LLMEM_W(p.hf), 0);
+  if (p.wide > 0) {
+    // per layer: `small` vectors of the hidden size, then `wide` of the feed-forward size
+    u32 code = 0;
+    for (int k = p.small; k < p.small + p.wide; ++k) code |= 1u << (2 * k);
+    set_run(d.run[3], (p.small + p.wide) * L, p.small + p.wide, code, LLMEM_W(p.vec_h), LLMEM_W(p.vec_f), 0);
+  } else {
+    set_const_run(d.run[3], p.small * L, LLMEM_W(p.vec_h));
+  }
+  set_const_run(d.run[4], p.final_n, LLMEM_W(p.vec_h));
+  set_const_run(d.run[5], 1, LLMEM_W(p.lm));
+  int n_ops = 1;
+  u32 fwd = 0;
+  if (f.act_mode) fwd = layer_code(f.ffn_kind != 0, false, &n_ops);
+  const i64 out = LLMEM_W(p.out);
+  set_const_run(d.run[6], p.e_n + (f.act_mode ? 0 : L), out);
+  set_run(d.run[7], f.act_mode ? L * n_ops : 0, n_ops, fwd, out, LLMEM_W(p.attn), LLMEM_W(p.ffn));
+  set_run(d.run[8], 3, 3, 0x14u, LLMEM_W(p.logit), LLMEM_W(p.shift), 0);  // logits, shifted copy, shifted copy
+  for (int r = 9; r < kRuns; ++r) set_const_run(d.run[r], 0, 0);
+#undef LLMEM_W
+  link_runs(d);
+  d.init_n = 2u + (u32)p.has_pos;
+  d.dyn_n = (u32)(p.count - d.init_n);
+  d.os_n = 0;
+}
+
+static __device__ __noinline__ void build_desc(SegDesc& d, const llmem_config* __restrict__ cfg, i64 gstart, i64 gend,
+                                               bool round, bool dnn = false) {
   d.first_part = -1;
   d.reserved = 0;
   d.invalid = 1;
@@ -102,6 +164,10 @@ static __device__ __noinline__ void build_desc(SegDesc& d, const llmem_config* _
   if (gend <= gstart) return;
   Cfg f = load_cfg(cfg);
   if (check_fields(f, true, true) != LLMEM_CFG_OK) return;
+  if (dnn) {
+    build_dnn_runs(d, f, round);
+    return;
+  }
   Plan p = make_plan(f, f.method);
   if (p.status != LLMEM_CFG_OK) return;
   Dyn y = make_dyn(p, (u64)f.batch);
@@ -141,25 +207,7 @@ static __device__ __noinline__ void build_desc(SegDesc& d, const llmem_config* _
   // per layer: four H x H tensors, then the feed-forward ones
   set_run(d.run[15], p.K * L, p.K, p.K == 7 ? 0x1500u : 0x0500u, LLMEM_V(p.os_hh), LLMEM_V(p.os_hf), 0);
 #undef LLMEM_V
-  // where each run starts inside its group
-  d.run[1].start = 2;
-  for (int r = kDynFirst + 1; r <= kDynLast; ++r) d.run[r].start = d.run[r - 1].start + d.run[r - 1].cnt;
-  for (int r = kOsFirst + 1; r <= kOsLast; ++r) d.run[r].start = d.run[r - 1].start + d.run[r - 1].cnt;
-  // which run follows each run: in the first iteration the optimizer states follow the frees
-  for (int r = 0; r < kRuns; ++r) {
-    i64 links = 0;
-    for (int later = 0; later < 2; ++later) {
-      int nx = r;
-      for (int guard = 0; guard < 2 * kRuns; ++guard) {
-        if (nx == kDynLast) nx = later ? kDynFirst : kOsFirst;
-        else if (nx == kOsLast) nx = kDynFirst;
-        else ++nx;
-        if (d.run[nx].cnt > 0) break;
-      }
-      links |= (i64)nx << (8 * later);
-    }
-    d.run[r].links = links;
-  }
+  link_runs(d);
   d.init_n = 2u + 2u * (u32)C;
   const u32 allocs = (u32)(G * (1 + C) + p.e_n + L * n_ops + 3 + T * L);
   d.dyn_n = 2 * allocs;
@@ -295,11 +343,12 @@ struct BufferKeys {
 // Makes sure the warp's descriptor is that of segment `seg` (range [gs, ge)): built by lane 0
 // when the warp enters the segment.
 __device__ __forceinline__ void ensure_desc(ExpandWarpSmem& ws, i64& desc_seg, const llmem_config* __restrict__ cfg,
-                                            i64 seg, i64 gs, i64 ge, bool round, int lane, const Guard& g) {
+                                            i64 seg, i64 gs, i64 ge, int round /* bit 0: rounded values, bit 1: second estimator */,
+                                            int lane, const Guard& g) {
   if (desc_seg != seg) {
     __syncwarp();  // every lane is done with the previous descriptor
     if (lane == 0) {
-      if (in_bounds(seg >= 0 && seg < g.n, g, kSiteDescriptor)) build_desc(ws.desc, cfg + seg, gs, ge, round);
+      if (in_bounds(seg >= 0 && seg < g.n, g, kSiteDescriptor)) build_desc(ws.desc, cfg + seg, gs, ge, (round & 1) != 0, (round & 2) != 0);
       else ws.desc.invalid = 1;  // the segment is written as zeros
     }
     __syncwarp();
@@ -311,7 +360,7 @@ __device__ __forceinline__ void ensure_desc(ExpandWarpSmem& ws, i64& desc_seg, c
 // run of period 1 or 2?  Updates `ar` when it enters a new such run.
 __device__ __forceinline__ bool chunk_alternates(AlternatingRun& ar, ExpandWarpSmem& ws, i64& desc_seg,
                                                  const llmem_config* __restrict__ cfg, i64 seg, i64 gs, i64 ge, i64 tb,
-                                                 bool round, int lane, const Guard& g) {
+                                                 int round, int lane, const Guard& g) {
   if (tb + kExpChunk <= ar.end) return true;
   ensure_desc(ws, desc_seg, cfg, seg, gs, ge, round, lane, g);
   if (ws.desc.invalid) return false;

@@ -303,16 +303,18 @@ struct PartsOfSegments {
 // Host launcher of the finishing pass (defined with the scan kernels): one thread per
 // segment folds the partials of segments that cross the warps' blocks (block j starts at
 // bounds[j], bounds[n_warps] = end), joins the parts of segments written in parts, defines
-// empty segments, adds m_base + lm_p and marks inadmissible configurations.
+// empty segments, adds m_base + lm_p (m_base alone for the second estimator, `dnn`) and marks
+// inadmissible configurations.
 llmem_status launch_scan_finish(const i64* offsets, i64 n, int shift, const llmem_config* cfg, i64* peak_out,
                                 i64* index_out, const i64* bounds, i64 n_warps, const WarpPartials* partials,
-                                cudaStream_t stream, PartsOfSegments parts = PartsOfSegments());
+                                cudaStream_t stream, PartsOfSegments parts = PartsOfSegments(), bool dnn = false);
 
 // Host side of the expansion by segment owners (defined with its kernels): descriptor table,
 // list of parts, then every segment written by its owner into delta_out; with `fold` the bare
 // per-segment results as well.  `scratch` has llmem_expand_scan's layout, header cleared.
 llmem_status expand_by_owners(const llmem_config* cfg, i64 n, const i64* offsets, i64 total_events, i64* delta_out,
-                              bool round, bool fold, i64* peak_out, i64* index_out, void* scratch,
-                              PartsOfSegments* parts_out, cudaStream_t stream);
+                              int round_bits /* bit 0: rounded values, bit 1: second estimator */, bool fold,
+                              i64* peak_out, i64* index_out, void* scratch, PartsOfSegments* parts_out,
+                              cudaStream_t stream);
 
 }  // namespace llmem

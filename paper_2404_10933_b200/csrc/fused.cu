@@ -71,7 +71,8 @@ inline i64 max_parts(i64 n, i64 total_events) { return total_events / kOwnedPart
 // is too long for a lane also enters the segment's parts into the list of parts.
 constexpr int kDescThreads = 128;
 __global__ void __launch_bounds__(kDescThreads)
-desc_table_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict__ offsets, int round,
+desc_table_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict__ offsets,
+                  int round /* bit 0: rounded values, bit 1: second estimator */,
                   SegDesc* __restrict__ table, unsigned long long* __restrict__ part_count,
                   i64* __restrict__ part_list, i64 part_capacity) {
   extern __shared__ __align__(16) unsigned char desc_stage_raw[];
@@ -80,7 +81,7 @@ desc_table_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __rest
   i64 count = 0;
   if (i < n) {
     const i64 lo = __ldg(offsets + i), hi = __ldg(offsets + i + 1);
-    build_desc(stage[threadIdx.x], cfg + i, lo, hi, round != 0);
+    build_desc(stage[threadIdx.x], cfg + i, lo, hi, (round & 1) != 0, (round & 2) != 0);
     count = hi - lo;
   }
   // the parts of the longer segments: one addition to the counter per warp
@@ -165,7 +166,7 @@ __global__ void __launch_bounds__(kFusedWarps * 32)
 expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __restrict__ offsets, i64 total,
                    i64* __restrict__ out, i64 n_blocks, i64 kappa, int bulk_ok, i64* __restrict__ peak_out,
                    i64* __restrict__ index_out, i64* __restrict__ bounds, WarpPartials* __restrict__ partials,
-                   unsigned long long* __restrict__ work_counter) {
+                   unsigned long long* __restrict__ work_counter, int dnn /* 2: the second estimator's list, else 0 */) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   ExpandWarpSmem& ws = reinterpret_cast<ExpandWarpSmem*>(smem_raw)[warp];
@@ -200,7 +201,7 @@ expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __res
       i64* buf = ws.buf[parity];
       // a full chunk inside one segment may repeat the one before
       const bool alternating = seg < n && gs <= tb && tb + kExpChunk <= ge &&
-                               chunk_alternates(ar, ws, desc_seg, cfg, seg, gs, ge, tb, kRoundList, lane, g);
+                               chunk_alternates(ar, ws, desc_seg, cfg, seg, gs, ge, tb, (kRoundList ? 1 : 0) | dnn, lane, g);
       if (alternating) {
         prepare_alternating<kFusedStoresInFlight>(ar, keys, parity, buf, lane);
         folder.add_uniform(fold_alternating_chunk(ev<!kRoundList>(ar.x0), ev<!kRoundList>(ar.x1), tb), lane);
@@ -227,7 +228,7 @@ expand_scan_kernel(const llmem_config* __restrict__ cfg, i64 n, const i64* __res
             for (i64 e = (span_lo > pos ? span_lo : pos); e < span_hi; ++e) buf[e - tb] = 0;
             break;
           }
-          ensure_desc(ws, desc_seg, cfg, seg, gs, ge, kRoundList, lane, g);
+          ensure_desc(ws, desc_seg, cfg, seg, gs, ge, (kRoundList ? 1 : 0) | dnn, lane, g);
           const i64 piece_end = ge < te ? ge : te;
           const i64 e = span_lo > pos ? span_lo : pos;
           const i64 e_end = span_hi < piece_end ? span_hi : piece_end;
@@ -479,8 +480,9 @@ expand_scan_owned_kernel(i64 n, const i64* __restrict__ offsets, i64 total, i64*
 // `fold` the bare results go to peak_out / index_out and *parts_out tells the finishing pass
 // where the parts of the longer segments reported.
 llmem_status expand_by_owners(const llmem_config* cfg, i64 n, const i64* offsets, i64 total_events, i64* delta_out,
-                              bool round, bool fold, i64* peak_out, i64* index_out, void* scratch,
+                              int round_bits, bool fold, i64* peak_out, i64* index_out, void* scratch,
                               PartsOfSegments* parts_out, cudaStream_t s) {
+  const bool round = (round_bits & 1) != 0;
   static thread_local int configured_dev = -1;
   int dev = 0;
   cudaGetDevice(&dev);
@@ -504,7 +506,7 @@ llmem_status expand_by_owners(const llmem_config* cfg, i64 n, const i64* offsets
   unsigned long long* work_counter = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(scratch) + kWorkCounterOffset);
   unsigned long long* part_count = work_counter + 1;  // beside the work counter in the header
   desc_table_kernel<<<(unsigned)((n + kDescThreads - 1) / kDescThreads), kDescThreads, sizeof(SegDesc) * kDescThreads, s>>>(
-      cfg, n, offsets, round ? 1 : 0, table, part_count, part_list, part_capacity);
+      cfg, n, offsets, round_bits, table, part_count, part_list, part_capacity);
   llmem_status st = check_launch("expansion by segment owners (descriptor table)");
   if (st != LLMEM_OK) return st;
   const i64 n_groups = (n + 31) / 32;
@@ -571,6 +573,12 @@ extern "C" llmem_status llmem_expand_scan(const llmem_config* cfg, int64_t n, co
   i64 warps = 1;  // blocks of work the finishing pass has to look at
   PartsOfSegments parts_of_segments;  // segments written in parts, for the finishing pass
   const bool round = (flags & LLMEM_FUSE_ROUND) != 0;
+  const int dnn_bit = (flags & LLMEM_ESTIMATOR_DNNMEM) ? 2 : 0;
+  if (dnn_bit && !round) {
+    // the fold of a list written raw rounds every value to the 2 MiB page while it reads
+    set_error("llmem_expand_scan: LLMEM_ESTIMATOR_DNNMEM needs LLMEM_FUSE_ROUND (the list is written aligned to 512 bytes)");
+    return LLMEM_ERR_ARG;
+  }
   static thread_local int configured_dev = -1;
   int dev = 0;
   cudaGetDevice(&dev);
@@ -594,17 +602,17 @@ extern "C" llmem_status llmem_expand_scan(const llmem_config* cfg, int64_t n, co
   expand_scan_kernel<ROUND, kFusedWarpsLong><<<grid, kFusedWarpsLong * 32, smem, s>>>(                           \
       cfg, n, reinterpret_cast<const i64*>(offsets), total_events, reinterpret_cast<i64*>(delta_out), warps,    \
       kFusedSegmentCost, bulk_ok, reinterpret_cast<i64*>(peak_out), reinterpret_cast<i64*>(peak_index_out),      \
-      bounds, partials, work_counter)
+      bounds, partials, work_counter, dnn_bit)
     if (round) LLMEM_LAUNCH_FUSED(true); else LLMEM_LAUNCH_FUSED(false);
 #undef LLMEM_LAUNCH_FUSED
     llmem_status st = check_launch("llmem_expand_scan");
     if (st != LLMEM_OK) return st;
   } else if (total_events > 0) {
     llmem_status st = expand_by_owners(cfg, n, reinterpret_cast<const i64*>(offsets), total_events,
-                                       reinterpret_cast<i64*>(delta_out), round, true, reinterpret_cast<i64*>(peak_out),
+                                       reinterpret_cast<i64*>(delta_out), (round ? 1 : 0) | dnn_bit, true, reinterpret_cast<i64*>(peak_out),
                                        reinterpret_cast<i64*>(peak_index_out), scratch, &parts_of_segments, s);
     if (st != LLMEM_OK) return st;
   }
   return launch_scan_finish(reinterpret_cast<const i64*>(offsets), n, 0, cfg, reinterpret_cast<i64*>(peak_out),
-                            reinterpret_cast<i64*>(peak_index_out), bounds, warps, partials, s, parts_of_segments);
+                            reinterpret_cast<i64*>(peak_index_out), bounds, warps, partials, s, parts_of_segments, dnn_bit != 0);
 }

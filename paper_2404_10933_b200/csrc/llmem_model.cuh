@@ -376,4 +376,93 @@ __device__ __forceinline__ int full_status(const Cfg& f, Plan* plan_out, u64* pe
   return LLMEM_CFG_OK;
 }
 
+// ---------------------------------------------------------------------------
+// The DNNMem-style estimator of Section 3.1, which the paper implements for comparison: the
+// weight tensors as loaded (fp16), a constant 64 MB buffer of the block manager, and the
+// outputs of the forward pass accumulated operator by operator, every tensor aligned to 512
+// bytes; one device, no mixed precision, no chunks, no optimizer states.  The allocations in
+// order: buffer; token (and position) embedding; the Linear matrices layer by layer; the
+// vectors layer by layer (two norm weights, with biases also two norm biases, four attention
+// biases and the feed-forward output bias, then the feed-forward input biases); the final
+// norm; the lm_head; then embedding outputs, layer outputs (or every operator output),
+// logits and the two shifted copies as in the LLMem list.  Nothing is released during the
+// forward pass, so the peak is the total.
+// ---------------------------------------------------------------------------
+constexpr u64 kDnnAlign = 512;
+constexpr u64 kDnnBuffer = 64ull * 1024ull * 1024ull;
+
+__host__ __device__ __forceinline__ u64 align512(u64 x) { return (x + (kDnnAlign - 1)) & ~(kDnnAlign - 1); }
+
+struct DnnPlan {
+  int status;
+  int e_n, K, L, has_pos;
+  int small, wide, final_n;  // vectors per layer of the hidden / of the feed-forward size; final norm vectors
+  int n_x, n_attn, n_ffn;    // operator outputs kept per layer, by size
+  u64 count;                 // number of events
+  u64 tok, pos, hh, hf, vec_h, vec_f, lm;  // raw bytes of the weight tensors
+  u64 out, attn, ffn, logit, shift;        // raw bytes of the forward outputs (saturating)
+};
+
+// `f` has passed check_fields(f, true, true).
+__device__ __forceinline__ DnnPlan make_dnn_plan(const Cfg& f) {
+  DnnPlan p;
+  p.status = f.method == LLMEM_METHOD_CDP ? LLMEM_CFG_OK : LLMEM_CFG_COMBO;  // one device, no sharding
+  const u64 H = zx(f.hidden), F = zx(f.ffn), V = zx(f.vocab), P = zx(f.pos_len);
+  const int bias = (int)f.has_bias;
+  p.e_n = 1 + (f.pos_len > 0);
+  p.has_pos = f.pos_len > 0;
+  p.K = f.ffn_kind ? 7 : 6;
+  p.L = f.layers;
+  p.small = 2 + 7 * bias;
+  p.wide = bias * (p.K - 5);
+  p.final_n = 1 + bias;
+  p.n_x = f.act_mode ? 10 : 1;
+  p.n_attn = f.act_mode ? 2 : 0;
+  p.n_ffn = f.act_mode ? (f.ffn_kind ? 4 : 2) : 0;
+  p.tok = 2 * V * H;
+  p.pos = 2 * P * H;
+  p.hh = 2 * H * H;
+  p.hf = 2 * H * F;
+  p.vec_h = 2 * H;
+  p.vec_f = 2 * F;
+  p.lm = V * H * (u64)f.lm_bytes;
+  const u32 b = (u32)f.batch;
+  p.out = sat_mul_u32(b, 2 * zx(f.seq) * H);
+  p.logit = sat_mul_u32(b, (u64)f.lm_bytes * zx(f.seq) * V);
+  p.shift = sat_mul_u32(b, (u64)f.lm_bytes * zx(f.seq - 1) * V);
+  p.attn = p.n_attn ? sat_mul_u32(b, sat_mul_u32((u32)f.seq, sat_mul_u32((u32)f.seq, 2 * zx(f.heads)))) : 0;
+  p.ffn = p.n_ffn ? sat_mul_u32(b, 2 * zx(f.seq) * F) : 0;
+  p.count = 2 + (u64)p.has_pos + (u64)p.L * (u64)(p.K + p.small + p.wide) + (u64)p.final_n + 1 + (u64)p.e_n +
+            (u64)p.L * (u64)(p.n_x + p.n_attn + p.n_ffn) + 3;
+  return p;
+}
+
+// Sum of the aligned events (without m_base), saturating at 2^62.
+__device__ __forceinline__ u64 dnn_total(const DnnPlan& p) {
+  u64 s = kDnnBuffer + align512(p.tok) + (p.has_pos ? align512(p.pos) : 0) + align512(p.lm);
+  s = sat_add(s, sat_mul_u32((u32)p.L, 4 * align512(p.hh) + (u64)(p.K - 4) * align512(p.hf) +
+                                           (u64)p.small * align512(p.vec_h) + (u64)p.wide * align512(p.vec_f)));
+  s += (u64)p.final_n * align512(p.vec_h);
+  if (p.out >= kSat || p.logit >= kSat || p.shift >= kSat || p.attn >= kSat || p.ffn >= kSat) return kSat;
+  s = sat_add(s, sat_mul_u32((u32)(p.e_n + p.L * p.n_x), align512(p.out)));
+  if (p.n_attn) s = sat_add(s, sat_mul_u32((u32)(p.L * p.n_attn), align512(p.attn)));
+  if (p.n_ffn) s = sat_add(s, sat_mul_u32((u32)(p.L * p.n_ffn), align512(p.ffn)));
+  s = sat_add(s, align512(p.logit));
+  s = sat_add(s, sat_mul_u32(2u, align512(p.shift)));
+  return s;
+}
+
+// Status and peak of a configuration under the second estimator; on LLMEM_CFG_OK *plan_out
+// holds the plan and *peak_out the peak (m_base included).
+__device__ __forceinline__ int dnn_full_status(const Cfg& f, DnnPlan* plan_out, u64* peak_out) {
+  int st = check_fields(f, true, true);
+  if (st != LLMEM_CFG_OK) return st;
+  *plan_out = make_dnn_plan(f);
+  if (plan_out->status != LLMEM_CFG_OK) return plan_out->status;
+  const u64 total = sat_add((u64)f.base_bytes, dnn_total(*plan_out));
+  if (total >= kSat) return LLMEM_CFG_OVERFLOW;
+  *peak_out = total;
+  return LLMEM_CFG_OK;
+}
+
 }  // namespace llmem

@@ -121,10 +121,18 @@ struct ScanWarpSmem {
 };
 
 // Per-configuration additive offset m_base + lm_p and admissibility.
-__device__ __forceinline__ bool segment_offset(const llmem_config* __restrict__ cfg, i64 seg, i64* off) {
+__device__ __forceinline__ bool segment_offset(const llmem_config* __restrict__ cfg, i64 seg, i64* off, bool dnn) {
   *off = 0;
   if (!cfg) return true;
   Cfg f = load_cfg(cfg + seg);
+  if (dnn) {
+    // the second estimator adds the CUDA context alone: the lm_head is one of its events
+    DnnPlan p;
+    u64 peak;
+    if (dnn_full_status(f, &p, &peak) != LLMEM_CFG_OK) return false;
+    *off = f.base_bytes;
+    return true;
+  }
   Plan p;
   u64 peak;
   if (full_status(f, &p, &peak) != LLMEM_CFG_OK) return false;
@@ -541,7 +549,7 @@ __device__ __forceinline__ i64 owner_of(const i64* __restrict__ bounds, i64 n_wa
 __global__ void __launch_bounds__(256)
 scan_finish_kernel(const i64* __restrict__ offsets, i64 n, int shift, const llmem_config* __restrict__ cfg,
                    i64* __restrict__ peak_out, i64* __restrict__ index_out, const i64* __restrict__ bounds,
-                   i64 n_warps, const WarpPartials* __restrict__ partials, PartsOfSegments parts) {
+                   i64 n_warps, const WarpPartials* __restrict__ partials, PartsOfSegments parts, bool dnn) {
   for (i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (i64)gridDim.x * blockDim.x) {
     const i64 a = offsets[i] + shift, b = offsets[i + 1] + shift;
     i64 mx = 0, idx = -1;
@@ -575,7 +583,7 @@ scan_finish_kernel(const i64* __restrict__ offsets, i64 n, int shift, const llme
       }
     }
     i64 off;
-    const bool ok = segment_offset(cfg, i, &off);
+    const bool ok = segment_offset(cfg, i, &off, dnn);
     peak_out[i] = ok ? off + mx : -1;
     if (index_out) index_out[i] = ok ? idx : -1;
   }
@@ -583,13 +591,13 @@ scan_finish_kernel(const i64* __restrict__ offsets, i64 n, int shift, const llme
 
 llmem_status launch_scan_finish(const i64* offsets, i64 n, int shift, const llmem_config* cfg, i64* peak_out,
                                 i64* index_out, const i64* bounds, i64 n_warps, const WarpPartials* partials,
-                                cudaStream_t stream, PartsOfSegments parts) {
+                                cudaStream_t stream, PartsOfSegments parts, bool dnn) {
   i64 blocks = (n + 255) / 256;
   const i64 cap = (i64)sm_count() * 8;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   scan_finish_kernel<<<(unsigned)blocks, 256, 0, stream>>>(offsets, n, shift, cfg, peak_out, index_out, bounds,
-                                                          n_warps < 1 ? 1 : n_warps, partials, parts);
+                                                          n_warps < 1 ? 1 : n_warps, partials, parts, dnn);
   return check_launch("llmem_scan_peak (finish)");
 }
 
@@ -628,6 +636,11 @@ extern "C" llmem_status llmem_scan_peak(const int64_t* delta, const int64_t* off
   const int shift = aligned_to(delta, 16) ? 0 : 1;
   const i64* delta_aligned = reinterpret_cast<const i64*>(delta) - shift;
   const bool round = (flags & LLMEM_FUSE_ROUND) != 0;
+  const bool dnn = (flags & LLMEM_ESTIMATOR_DNNMEM) != 0;
+  if (dnn && round) {
+    set_error("llmem_scan_peak: LLMEM_FUSE_ROUND rounds to the 2 MiB page; lists of the second estimator are written aligned");
+    return LLMEM_ERR_ARG;
+  }
   i64 warps = 1;
   PartsOfSegments parts_of_segments;
   if (scan_by_owners(n, total_events)) {
@@ -701,7 +714,7 @@ extern "C" llmem_status llmem_scan_peak(const int64_t* delta, const int64_t* off
     if (st != LLMEM_OK) return st;
   }
   return launch_scan_finish(reinterpret_cast<const i64*>(offsets), n, shift, cfg, reinterpret_cast<i64*>(peak_out),
-                            reinterpret_cast<i64*>(peak_index_out), bounds, warps, partials, s, parts_of_segments);
+                            reinterpret_cast<i64*>(peak_index_out), bounds, warps, partials, s, parts_of_segments, dnn);
 }
 
 extern "C" llmem_status llmem_selftest_wait_limit(void* scratch, size_t scratch_bytes, uint32_t limit_ms,

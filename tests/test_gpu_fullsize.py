@@ -170,6 +170,36 @@ def test_g3_large_sweep_full(llmem):
     assert_equals_level1(got, want1, got["status"], offsets)
 
 
+def test_g3_large_sweep_second_estimator(llmem):
+    """The DNNMem-style estimator (Section 3.1) over the shapes of the large sweep, conventional
+    method: every peak, position, status and event count against the oracle's explicit lists,
+    and the materialised list of a 2^16 slice against the oracle's through the one-pass path."""
+    def make():
+        c = grids.g3_sweep().copy()
+        c["method"], c["gpu_n"], c["tp_n"] = 0, 1, 0
+        c["method"][::97] = 2                      # some records the estimator refuses
+        return c
+    if "g3_dnn" not in _LEVEL1:
+        cfgs = make()
+        _LEVEL1["g3_dnn"] = (cfgs, oracle.dnn_estimate(cfgs, threads=THREADS))
+    cfgs, want = _LEVEL1["g3_dnn"]
+    got = llmem.estimate_batch(cfgs, estimator="dnnmem")
+    offsets, _ = llmem.event_counts(cfgs, estimator="dnnmem")
+    assert_equals_level1(got, want, got["status"], offsets)
+    assert (want["status"] == 2).sum() == len(range(0, len(cfgs), 97))
+    part = cfgs[:1 << 16]
+    dev = llmem.to_device(part)
+    off, _ = llmem.event_counts(dev, estimator="dnnmem")
+    one = llmem.expand_scan(dev, off, fuse_round=True, estimator="dnnmem")
+    assert np.array_equal(one["peak"].cpu().numpy(), want["peak"][:1 << 16])
+    assert np.array_equal(one["index"].cpu().numpy(), want["index"][:1 << 16])
+    o = off.cpu().numpy()
+    for i in sample_indices(len(part), 40, 21):
+        if want["status"][i] == 0:
+            ev = oracle.dnn_round_events(oracle.dnn_expand_events(part[i:i + 1]))
+            assert np.array_equal(one["delta"][o[i]:o[i + 1]].cpu().numpy(), ev)
+
+
 def test_g4_max_batch_and_selection_full(llmem):
     caps = grids.g4_capacities()
     bmax = grids.G4_BMAX

@@ -503,6 +503,57 @@ def test_slab_bounds_on_device_equal_the_host_cut(llmem):
                                offsets.data_ptr(), None) == llmem.ERR_ARG
 
 
+def test_second_estimator_all_paths(llmem):
+    """The DNNMem-style estimator of Section 3.1: fused estimate, event counts, the list raw
+    and aligned to 512 bytes (both expansion kernels), its scan and the one-pass path against
+    the oracle, on G1, a mixed grid with inadmissible records, long lists and every operator
+    output kept; the searches refuse the flag."""
+    mixed = mixed_small_grid()
+    mixed["method"][::2] = 0                       # the estimator takes the conventional method only
+    long_lists = grids.g5_stress(3, 12).copy()
+    long_lists["method"], long_lists["act_mode"] = 0, np.arange(12) % 2
+    long_lists["layers"] = 40000                   # lists long enough for the chunk kernels
+    for cfgs in (grids.g1_small(), mixed, long_lists):
+        want = oracle.dnn_estimate(cfgs, threads=8)
+        got = llmem.estimate_batch(cfgs, estimator="dnnmem")
+        for k in ("status", "peak", "index"):
+            assert np.array_equal(got[k].cpu().numpy(), want[k]), k
+        assert (want["status"] == 0).any()
+        dev = llmem.to_device(cfgs)
+        offsets, status = llmem.event_counts(dev, estimator="dnnmem")
+        off = offsets.cpu().numpy()
+        assert np.array_equal(status.cpu().numpy(), want["status"])
+        assert np.array_equal(np.diff(off), np.where(want["status"] == 0, want["count"], 0))
+        total = int(off[-1])
+        raw_want = np.concatenate([oracle.dnn_expand_events(cfgs[i:i + 1]) for i in range(len(cfgs))
+                                   if want["status"][i] == 0])
+        aligned_want = oracle.dnn_round_events(raw_want)
+        raw = llmem.expand_events(dev, offsets, total, estimator="dnnmem")
+        assert np.array_equal(raw.cpu().numpy(), raw_want)
+        header = torch.zeros(256, dtype=torch.uint8, device="cuda")
+        for scratch in (None, header):             # segment owners / chunks of the list
+            aligned = llmem.expand_events(dev, offsets, total, fuse_round=True, estimator="dnnmem", scratch=scratch)
+            assert np.array_equal(aligned.cpu().numpy(), aligned_want)
+        two = llmem.scan_peak(aligned, offsets, dev, estimator="dnnmem", check_status=True)
+        one = llmem.expand_scan(dev, offsets, total, fuse_round=True, estimator="dnnmem")
+        assert np.array_equal(one["delta"].cpu().numpy(), aligned_want)
+        pipe = llmem.estimate_materialized(dev, estimator="dnnmem")
+        for r in (two, one, pipe):
+            assert np.array_equal(r["peak"].cpu().numpy(), want["peak"])
+            assert np.array_equal(r["index"].cpu().numpy(), want["index"])
+        with pytest.raises(llmem.LlmemError):
+            llmem.expand_scan(dev, offsets, total, fuse_round=False, estimator="dnnmem")
+        with pytest.raises(llmem.LlmemError):
+            llmem.scan_peak(raw, offsets, dev, fuse_round=True, estimator="dnnmem")
+    L = llmem.lib()
+    caps = llmem._caps(grids.g4_capacities(), dev.device)
+    out = torch.zeros((len(cfgs), caps.numel()), dtype=torch.int32, device="cuda")
+    assert L.llmem_max_batch(dev.data_ptr(), len(cfgs), caps.data_ptr(), caps.numel(), 8, out.data_ptr(), None, None, 0,
+                             llmem.ESTIMATOR_DNNMEM, None) == llmem.ERR_ARG
+    assert L.llmem_select_method(dev.data_ptr(), len(cfgs), caps.data_ptr(), caps.numel(), 8, out.data_ptr(),
+                                 out.data_ptr(), None, None, None, 0, llmem.ESTIMATOR_DNNMEM, None) == llmem.ERR_ARG
+
+
 CHECKED_SCRIPT = r"""
 import numpy as np, torch
 import oracle
