@@ -557,7 +557,7 @@ def run_ours(args):
 # grids (profiles/register_kernels_g3_g4_ncu.md); None once a kernel changes after the capture.
 # Counting lane instructions keeps divergence from passing for throughput: a warp instruction
 # issued for 20 of 32 lanes counts as 20/32.
-NCU_LANE_INSTR_PER_UNIT = {"estimate_kernel": 25.24, "max_batch_kernel": 8.40, "select_kernel": 40.21}
+NCU_LANE_INSTR_PER_UNIT = {"estimate_kernel": 21.78, "max_batch_kernel": 8.40, "select_kernel": 40.21}
 
 
 def _gpu_id(torch):

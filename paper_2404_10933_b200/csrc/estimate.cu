@@ -167,19 +167,20 @@ __device__ __forceinline__ void estimate_one(const Cfg& f, i64* pk_out, i64* ix_
   int st = check_fields(f, true, true);
   i64 pk = -1, ix = -1;
   if (st == LLMEM_CFG_OK) {
-    Search q;
-    q.p = make_plan(f, f.method);
-    st = q.p.status;
+    // only the peak is wanted: plain sums and products that remember whether one was too large
+    StickyMath m;
+    const Plan p = make_plan(m, f, f.method);
+    st = p.status;
     if (st == LLMEM_CFG_OK) {
-      q.s = make_static_sums(q.p, f.pos_len > 0);
-      Dyn d;
+      const StaticSums s = make_static_sums(m, p, f.pos_len > 0);
+      const Dyn d = make_dyn(m, p, (u64)f.batch);
       bool first_wins;
-      u64 total = q.peak((u64)f.batch, &d, &first_wins);
-      if (total >= kSat) {
+      const u64 rel = relative_peak(m, p, s, m.add(s.gather, dyn_sum(m, p, d)), &first_wins);
+      const u64 total = m.add(p.offset, rel);
+      if (m.too_large(total)) {
         st = LLMEM_CFG_OVERFLOW;
       } else {
         pk = (i64)total;
-        const Plan& p = q.p;
         // position of the peak: the last allocation of non-zero size in the
         // iteration that attains it, or the last optimizer-state allocation
         const u64 init_n = 2 + 2 * (u64)p.C;
@@ -200,12 +201,12 @@ __device__ __forceinline__ void estimate_one(const Cfg& f, i64* pk_out, i64* ix_
   *st_out = st;
 }
 
-// One thread per configuration.  (Handing the configurations of a CTA's tile out in the order
-// of a counting sort by method, feed-forward kind and position embedding, so that a warp
-// evaluates one kind, does remove the divergence -- 30.5 instead of 26 of 32 lanes busy, a
-// tenth fewer warp instructions -- but the kernel waits on dependent 64-bit arithmetic rather
-// than on issue slots, and the barriers of the sort cost more than the idle lanes: 0.74 ms
-// instead of 0.69 ms for 2^24 configurations.)
+// One thread per configuration.  The lanes of a warp hold configurations of different methods,
+// so the model forms the quotients by the partition degrees in every lane and selects (a
+// division that three lanes in four need is not worth a branch): on a random mix of the four
+// methods 29.6 of 32 lanes are busy per instruction.  Handing the configurations of a CTA's
+// tile out in the order of a counting sort by method was tried before that and lost to the
+// barriers of the sort.
 // The same for the DNNMem-style estimator of Section 3.1: the list only grows, so the peak is
 // the total and sits at the last event of non-zero size (the second shifted copy, or the
 // logits when the sequence has one token).

@@ -65,6 +65,37 @@ __device__ __forceinline__ u64 sat_mul_u32(u32 a, u64 b) {
   return (hi >= (1ull << 30) || t < lo || t >= kSat) ? kSat : t;
 }
 
+// The model's sums and products under two policies.  SatMath clamps every result at 2^62, so
+// a value can be carried on and compared (the searches do).  StickyMath computes the plain
+// 64-bit result and only remembers whether some result reached 2^62: every quantity is
+// non-negative and enters the peak, so "some result reached 2^62" and "the peak reached 2^62"
+// are the same statement, and where the peak is all that is asked for the clamps (two
+// compares and two selects per operation) shrink to one OR.  Operands must be exact (below
+// 2^62) or follow a result that has already been recorded as too large.
+struct SatMath {
+  __device__ __forceinline__ u64 add(u64 a, u64 b) { return sat_add(a, b); }
+  __device__ __forceinline__ u64 mul(u32 a, u64 b) { return sat_mul_u32(a, b); }
+  __device__ __forceinline__ bool too_large(u64 total) const { return total >= kSat; }
+};
+
+struct StickyMath {
+  u32 top = 0;   // bits 64.. of some result
+  u32 word = 0;  // bits 32..63 of some result: too large when bit 30 or 31 is set
+  __device__ __forceinline__ u64 add(u64 a, u64 b) {
+    const u64 s = a + b;  // a, b < 2^62: no wrap
+    word |= (u32)(s >> 32);
+    return s;
+  }
+  __device__ __forceinline__ u64 mul(u32 a, u64 b) {
+    const u64 lo = (u64)a * (u32)b;
+    const u64 upper = (u64)a * (u32)(b >> 32) + (lo >> 32);  // the product >> 32; b < 2^62: no wrap
+    top |= (u32)(upper >> 32);
+    word |= (u32)upper;
+    return (upper << 32) | (u32)lo;
+  }
+  __device__ __forceinline__ bool too_large(u64) const { return (top | (word >> 30)) != 0; }
+};
+
 // zero-extension of a field that check_fields has shown to be non-negative: tells the
 // compiler that the upper half is zero, so products of two such values are one widening multiply
 __device__ __forceinline__ u64 zx(int v) { return (u64)(u32)v; }
@@ -111,6 +142,19 @@ __device__ __forceinline__ Cfg load_cfg(const llmem_config* __restrict__ p) {
   return unpack_cfg(a, b, c, d);
 }
 
+// Whether d divides x, for 1 <= x <= 2^20 and d >= 1, without the integer division routine:
+// both numbers are exact in single precision, the quotient of a fast division is within
+// 2^20 * 3 * 2^-24 < 1/2 of the true one, so it rounds to the true quotient whenever that is an
+// integer, and one exact multiplication tells.  (A d above x gives quotient 0 or 1 and fails.)
+__device__ __forceinline__ bool divides(int d, int x) {
+  const int dc = d < (1 << 21) ? d : (1 << 21);
+  const float two23 = 8388608.0f;
+  const float xf = __uint_as_float(0x4b000000u | (u32)x) - two23;
+  const float df = __uint_as_float(0x4b000000u | (u32)dc) - two23;
+  const u32 q = __float_as_uint(__fdividef(xf, df) + two23) & 0x007fffffu;  // nearest integer
+  return q * (u32)dc == (u32)x;
+}
+
 // Field ranges (status 1).  `check_batch` is false for the search entry points,
 // which choose the batch themselves; `check_method` is false for selection.
 __device__ __forceinline__ int check_fields(const Cfg& f, bool check_batch, bool check_method) {
@@ -121,7 +165,7 @@ __device__ __forceinline__ int check_fields(const Cfg& f, bool check_batch, bool
             f.base_bytes >= 0 && f.base_bytes <= (1ll << 60) && f.gpu_n >= 1 &&
             (f.lm_bytes == 2 || f.lm_bytes == 4) && f.ffn_kind <= 1 && f.has_bias <= 1 &&
             f.iters >= 1 && f.act_mode <= 1 && f.reserved_zero;
-  if (ok) ok = (f.hidden % f.heads) == 0;
+  if (ok) ok = divides(f.heads, f.hidden);
   if (ok && check_batch) ok = f.batch >= 1 && f.batch <= (1 << 26);
   if (ok && check_method) ok = f.method <= 3;
   return ok ? LLMEM_CFG_OK : LLMEM_CFG_FIELD;
@@ -209,19 +253,22 @@ __device__ __forceinline__ u64 chunk_count(u64 a, u64 b) {
   return q + (r != 0 ? 1 : 0);
 }
 
-__device__ __forceinline__ u64 shard_bytes(u64 bytes, u32 method, const Recip& n) {
-  return method == LLMEM_METHOD_CDP ? bytes : ceil_div(bytes, n);
-}
+// Bytes of a tensor's shard on one device: the whole tensor for CDP (the caller passes the
+// reciprocal of 1), ceil(bytes / gpu_n) otherwise.  No branch on the method: the lanes of a
+// warp hold different methods, and a division skipped by some of them is not time saved.
+__device__ __forceinline__ u64 shard_bytes(u64 bytes, const Recip& n) { return ceil_div(bytes, n); }
 
 // fp16 bytes of a unit of x elements that exist only while computing:
 // ADP holds the whole of param fp16 (m_p,16 undivided in m_peak^dp);
 // DP+TP holds m_p,16 * (1 - tp_n/gpu_n) (m_peak^dp+tp).
-__device__ __forceinline__ u64 gathered_bytes(u64 x, u32 method, const Recip& n, u32 t) {
-  u64 whole = 2 * x;
-  u64 kept = ceil_div(whole, n);
-  if (method == LLMEM_METHOD_ADP) return whole - kept;
-  if (method == LLMEM_METHOD_DPTP) return whole - floor_div(whole * t, n) - kept;  // whole * t < 2^55
-  return 0;
+// `kept` = ceil(2 x / gpu_n), the shard that stays; `n` the reciprocal of gpu_n.
+__device__ __forceinline__ u64 gathered_bytes(u64 x, u32 method, const Recip& n, u32 t, u64 kept) {
+  const u64 whole = 2 * x;
+  const u64 tp_share = floor_div(whole * t, n);  // whole * t < 2^56
+  u64 g = 0;
+  if (method == LLMEM_METHOD_ADP) g = whole - kept;
+  if (method == LLMEM_METHOD_DPTP) g = whole - tp_share - kept;
+  return g;
 }
 
 // Table 1, other_p: every parameter outside the input embedding and lm_head of a standard
@@ -236,11 +283,12 @@ __device__ __forceinline__ u64 other_params(const Cfg& f) {
 }
 
 // a1: parameter inventory and event sizes.  `f` has passed check_fields.
-__device__ __forceinline__ Plan make_plan(const Cfg& f, u32 method) {
+template <class Math>
+__device__ __forceinline__ Plan make_plan(Math& m, const Cfg& f, u32 method) {
   Plan p;
   p.status = check_combo(method, f.gpu_n, f.tp_n);
   const u64 H = zx(f.hidden), F = zx(f.ffn), V = zx(f.vocab), P = zx(f.pos_len);
-  const Recip rn = make_recip(f.gpu_n);
+  const Recip rn = make_recip(method == LLMEM_METHOD_CDP ? 1u : f.gpu_n);
   p.e_n = 1 + (f.pos_len > 0);
   p.K = f.ffn_kind ? 7 : 6;
   p.gather = (method == LLMEM_METHOD_ADP || method == LLMEM_METHOD_DPTP);
@@ -256,16 +304,16 @@ __device__ __forceinline__ Plan make_plan(const Cfg& f, u32 method) {
   const u64 cs = (u64)f.chunk_elems;
   const u64 chunks = chunk_count(other_p, cs);
   p.offset = (u64)f.base_bytes + tok_p * (u64)f.lm_bytes;  // < 2^60 + 2^49
-  p.p16_embed = shard_bytes(2 * embed_p, method, rn);
-  p.p32_embed = shard_bytes(4 * embed_p, method, rn);
-  p.p16_chunk = shard_bytes(2 * cs, method, rn);
-  p.p32_chunk = shard_bytes(4 * cs, method, rn);
-  p.gat_embed = gathered_bytes(embed_p, method, rn, p.tp);
-  p.gat_chunk = gathered_bytes(cs, method, rn, p.tp);
-  p.os_tok = shard_bytes(8 * tok_p, method, rn);
-  p.os_pos = shard_bytes(8 * pos_p, method, rn);
-  p.os_hh = shard_bytes(8 * hh_p, method, rn);
-  p.os_hf = shard_bytes(8 * hf_p, method, rn);
+  p.p16_embed = shard_bytes(2 * embed_p, rn);
+  p.p32_embed = shard_bytes(4 * embed_p, rn);
+  p.p16_chunk = shard_bytes(2 * cs, rn);
+  p.p32_chunk = shard_bytes(4 * cs, rn);
+  p.gat_embed = gathered_bytes(embed_p, method, rn, p.tp, p.p16_embed);
+  p.gat_chunk = gathered_bytes(cs, method, rn, p.tp, p.p16_chunk);
+  p.os_tok = shard_bytes(8 * tok_p, rn);
+  p.os_pos = shard_bytes(8 * pos_p, rn);
+  p.os_hh = shard_bytes(8 * hh_p, rn);
+  p.os_hf = shard_bytes(8 * hf_p, rn);
   p.out1 = 2 * zx(f.seq) * H;                              // <= 2^47
   p.logit1 = (u64)f.lm_bytes * zx(f.seq) * V;              // <= 2^54
   p.shift1 = (u64)f.lm_bytes * zx(f.seq - 1) * V;
@@ -275,7 +323,7 @@ __device__ __forceinline__ Plan make_plan(const Cfg& f, u32 method) {
   p.n_x = f.act_mode ? 10 : 1;
   p.n_attn = f.act_mode ? 2 : 0;
   p.n_ffn = f.act_mode ? (f.ffn_kind ? 4 : 2) : 0;
-  p.attn1 = sat_mul_u32((u32)f.seq, sat_mul_u32((u32)f.seq, 2 * zx(f.heads)));
+  p.attn1 = f.act_mode ? m.mul((u32)f.seq, m.mul((u32)f.seq, 2 * zx(f.heads))) : 0;
   p.ffn1 = 2 * zx(f.seq) * F;                              // <= 2^49
   if (chunks >= kCountLimit) {
     p.C = 0;
@@ -291,28 +339,38 @@ __device__ __forceinline__ Plan make_plan(const Cfg& f, u32 method) {
   return p;
 }
 
+__device__ __forceinline__ Plan make_plan(const Cfg& f, u32 method) {
+  SatMath m;
+  return make_plan(m, f, method);
+}
+
 // Batch-dependent raw sizes (saturating).
 struct Dyn {
   u64 out, logit, shift, back, attn, ffn;
 };
 
-__device__ __forceinline__ Dyn make_dyn(const Plan& p, u64 batch) {
+template <class Math>
+__device__ __forceinline__ Dyn make_dyn(Math& m, const Plan& p, u64 batch) {
   Dyn d;
   const u32 b32 = (u32)batch;  // batch <= 2^26
-  d.out = sat_mul_u32(b32, p.out1);
-  d.logit = sat_mul_u32(b32, p.logit1);
-  d.shift = sat_mul_u32(b32, p.shift1);
+  d.out = m.mul(b32, p.out1);
+  d.logit = m.mul(b32, p.logit1);
+  d.shift = m.mul(b32, p.shift1);
   // ceil(out * (tp-1) / tp) = out - floor(out / tp)   (m_back^tp, one layer's share); the
-  // reciprocal is exact below 2^56, and a saturated output makes the whole peak overflow
-  d.back = 0;
-  if (p.tpback) {
-    if (d.out >= kSat) d.back = kSat;
-    else if (d.out < (1ull << 56)) d.back = d.out - floor_div(d.out, Recip{p.tp_recip, p.tp});
-    else d.back = d.out - d.out / p.tp;
-  }
-  d.attn = p.n_attn ? sat_mul_u32(b32, p.attn1) : 0;
-  d.ffn = p.n_ffn ? sat_mul_u32(b32, p.ffn1) : 0;
+  // reciprocal is exact below 2^56, and a saturated output makes the whole peak overflow.
+  // The quotient is formed in every lane (no branch on the method), the rare wide one apart.
+  u64 share = floor_div(d.out, Recip{p.tp_recip, p.tp});
+  if (p.tpback && d.out >= (1ull << 56)) share = d.out / p.tp;
+  d.back = p.tpback ? d.out - share : 0;
+  if (p.tpback && d.out >= kSat) d.back = kSat;
+  d.attn = p.n_attn ? m.mul(b32, p.attn1) : 0;
+  d.ffn = p.n_ffn ? m.mul(b32, p.ffn1) : 0;
   return d;
+}
+
+__device__ __forceinline__ Dyn make_dyn(const Plan& p, u64 batch) {
+  SatMath m;
+  return make_dyn(m, p, batch);
 }
 
 // Batch-independent sums of rounded events.
@@ -320,42 +378,60 @@ struct StaticSums {
   u64 init, gather, os;
 };
 
-__device__ __forceinline__ StaticSums make_static_sums(const Plan& p, bool has_pos) {
+template <class Math>
+__device__ __forceinline__ StaticSums make_static_sums(Math& m, const Plan& p, bool has_pos) {
   StaticSums s;
-  s.init = sat_add(sat_add(page_round(p.p16_embed), page_round(p.p32_embed)),
-                   sat_mul_u32(p.C, page_round(p.p16_chunk) + page_round(p.p32_chunk)));
-  s.gather = p.gather ? sat_add(page_round(p.gat_embed), sat_mul_u32(p.C, page_round(p.gat_chunk))) : 0;
+  s.init = m.add(m.add(page_round(p.p16_embed), page_round(p.p32_embed)),
+                 m.mul(p.C, page_round(p.p16_chunk) + page_round(p.p32_chunk)));
+  s.gather = p.gather ? m.add(page_round(p.gat_embed), m.mul(p.C, page_round(p.gat_chunk))) : 0;
   const u64 per_layer = 4 * page_round(p.os_hh) + (u64)(p.K - 4) * page_round(p.os_hf);  // < 2^48
-  s.os = sat_add(page_round(p.os_tok) + (has_pos ? page_round(p.os_pos) : 0),
-                 sat_mul_u32((u32)p.L, per_layer));
+  s.os = m.add(page_round(p.os_tok) + (has_pos ? page_round(p.os_pos) : 0), m.mul((u32)p.L, per_layer));
   return s;
 }
 
+__device__ __forceinline__ StaticSums make_static_sums(const Plan& p, bool has_pos) {
+  SatMath m;
+  return make_static_sums(m, p, has_pos);
+}
+
 // Sum of the rounded batch-dependent allocations of one iteration (phases 3 and 4).
-__device__ __forceinline__ u64 dyn_sum(const Plan& p, const Dyn& d) {
-  u64 s = sat_mul_u32((u32)(p.e_n + p.L * p.n_x), page_round(d.out));
-  if (p.n_attn) s = sat_add(s, sat_mul_u32((u32)(p.L * p.n_attn), page_round(d.attn)));
-  if (p.n_ffn) s = sat_add(s, sat_mul_u32((u32)(p.L * p.n_ffn), page_round(d.ffn)));
-  s = sat_add(s, page_round(d.logit));
-  s = sat_add(s, sat_mul_u32(2u, page_round(d.shift)));
-  if (p.tpback) s = sat_add(s, sat_mul_u32((u32)p.L, page_round(d.back)));
+template <class Math>
+__device__ __forceinline__ u64 dyn_sum(Math& m, const Plan& p, const Dyn& d) {
+  u64 s = m.mul((u32)(p.e_n + p.L * p.n_x), page_round(d.out));
+  if (p.n_attn) s = m.add(s, m.mul((u32)(p.L * p.n_attn), page_round(d.attn)));
+  if (p.n_ffn) s = m.add(s, m.mul((u32)(p.L * p.n_ffn), page_round(d.ffn)));
+  s = m.add(s, page_round(d.logit));
+  s = m.add(s, m.mul(2u, page_round(d.shift)));
+  if (p.tpback) s = m.add(s, m.mul((u32)p.L, page_round(d.back)));
   return s;
+}
+
+__device__ __forceinline__ u64 dyn_sum(const Plan& p, const Dyn& d) {
+  SatMath m;
+  return dyn_sum(m, p, d);
 }
 
 // Largest prefix sum (without the offset) given the phase sums.  Iteration 1
 // peaks before the optimizer states exist; they are allocated after its frees and
-// stay; every later iteration peaks on top of them.
-__device__ __forceinline__ u64 relative_peak(const Plan& p, const StaticSums& s, u64 dyn_total,
+// stay; every later iteration peaks on top of them.  Only sums that the result is at least
+// as large as are formed, so that a sum which is too large makes the result too large.
+template <class Math>
+__device__ __forceinline__ u64 relative_peak(Math& m, const Plan& p, const StaticSums& s, u64 dyn_total,
                                              bool* first_iteration_wins) {
-  const u64 first = sat_add(s.init, dyn_total);
-  const u64 after = sat_add(s.init, s.os);
-  const u64 later = sat_add(after, dyn_total);
+  const u64 after = m.add(s.init, s.os);
   if (p.iters >= 2) {
     *first_iteration_wins = false;
-    return later;
+    return m.add(after, dyn_total);
   }
+  const u64 first = m.add(s.init, dyn_total);
   *first_iteration_wins = first >= after;
   return first >= after ? first : after;
+}
+
+__device__ __forceinline__ u64 relative_peak(const Plan& p, const StaticSums& s, u64 dyn_total,
+                                             bool* first_iteration_wins) {
+  SatMath m;
+  return relative_peak(m, p, s, dyn_total, first_iteration_wins);
 }
 
 // Complete admissibility check of a configuration for estimation: field ranges,
