@@ -59,10 +59,11 @@ struct PageSearch {
   u32 n_out, n_back;         // outputs kept per iteration; TP backward buffers (0 if none or tp = 1)
   int b_safe;                // probes stay within 1..b_safe; 0: nothing can fit
   bool single_iter;
-  double batches_per_page;   // cu_p / W: batches per page of batch-dependent memory (guided search)
-  double dyn_events;         // N: batch-dependent events of one iteration
+  double rate_up, rate_dn;   // cu_p / W for a W not above, and one not below, the bytes a sample adds
+  double dyn_events;         // N: at least the number of batch-dependent events of one iteration
 
-  __device__ __forceinline__ void init(const Plan& p, const StaticSums& s, int bmax) {
+  // `too_large`: one of the batch-independent sums (or the per-sample score size) reached 2^62
+  __device__ __forceinline__ void init(const Plan& p, const StaticSums& s, int bmax, bool too_large) {
     out1 = p.out1; logit1 = p.logit1; shift1 = p.shift1;
     offset = p.offset;
     n_out = (u32)(p.e_n + p.L * p.n_x);
@@ -78,10 +79,10 @@ struct PageSearch {
       r1 = (u32)(out1 - q1 * p.tp);
     }
     single_iter = p.iters < 2;
-    if (s.init >= kSat || s.os >= kSat || s.gather >= kSat) {
+    if (too_large) {
       b_safe = 0;
       fixed_a = fixed_b = 0;
-      batches_per_page = dyn_events = 0.0;
+      rate_up = rate_dn = dyn_events = 0.0;
       return;
     }
     const u64 init_p = s.init >> 21, os_p = s.os >> 21, gat_p = s.gather >> 21;
@@ -89,14 +90,18 @@ struct PageSearch {
     fixed_a = single_iter ? init_p + gat_p : init_p + os_p + gat_p;
     fixed_b = init_p + os_p;
     u64 big = out1 > logit1 ? out1 : logit1;  // >= 2
-    if (attn1 > big) big = attn1;               // may be saturated: then nothing fits
+    if (attn1 > big) big = attn1;
     if (ffn1 > big) big = ffn1;
     const u64 lim = (kSat - 1) / big;                // largest b with b * big < 2^62
     b_safe = lim < (u64)bmax ? (int)lim : bmax;
+    // bytes one more sample adds to the batch-dependent events, without the backward buffers;
+    // those add  out - floor(out / tp)  per layer, which lies between b (out1 - q1 - 1) and
+    // b (out1 - q1)
     const double w = (double)n_out * (double)out1 + (double)logit1 + 2.0 * (double)shift1 +
-                     (double)n_attn * (double)attn1 + (double)n_ffn * (double)ffn1 +
-                     (double)n_back * (double)(out1 - q1);
-    batches_per_page = (double)kPage / w;
+                     (double)n_attn * (double)attn1 + (double)n_ffn * (double)ffn1;
+    const double back_hi = n_back ? (double)(out1 - q1) : 0.0;  // out1 >= 2 q1 >= q1 + 1 when tp >= 2
+    rate_up = (double)kPage / (w + (double)n_back * (back_hi - (n_back ? 1.0 : 0.0)));
+    rate_dn = (double)kPage / (w + (double)n_back * back_hi);
     dyn_events = (double)(n_out + n_attn + n_ffn + 2 * n_back + 3);
   }
 
@@ -121,10 +126,13 @@ struct PageSearch {
   // increments b until the peak exceeds m_total; the peak never decreases with b, so any
   // search that ends with "b fits, b + 1 does not" finds the same b.  The page count is
   // almost linear in b: with W the bytes all batch-dependent events take per sample and N
-  // their number,  b W / cu_p <= dyn pages(b) <= b W / cu_p + N,  which brackets the answer
-  // within about N cu_p / W + 2 batches.  The bracket is computed in floating point, made
-  // certain by probing its two ends (so the result does not depend on rounding there), and
-  // bisected: four or five probes instead of log2(bmax).
+  // their number,  b W / cu_p <= dyn pages(b) < b W / cu_p + N  (every event rounds up by
+  // less than a page).  So with R pages of room nothing above R cu_p / W fits and everything
+  // up to (R - N) cu_p / W does.  Both bounds are computed in double precision: the sums and
+  // products behind them are of positive terms, fewer than twenty roundings of 2^-53 each,
+  // and the bounds are widened by 2^-40, far more than that, before they are cut to integers,
+  // so the bracket is certain.  For most shapes it holds one candidate and no probe is needed;
+  // otherwise it is bisected with exact page counts.
   __device__ __forceinline__ int largest_batch(i64 capacity) const {
     const u64 cap = capacity >= (i64)kSat ? kSat - 1 : (u64)(capacity < 0 ? 0 : capacity);
     if (capacity < 0 || cap < offset || b_safe == 0) return 0;
@@ -136,20 +144,11 @@ struct PageSearch {
 
   template <bool kActs>
   __device__ __forceinline__ int guided(u64 budget) const {
-    const double room = (double)(budget - fixed_a);
-    const double hi_d = room * batches_per_page, lo_d = (room - dyn_events) * batches_per_page;
-    int hi = hi_d >= (double)b_safe ? b_safe : (int)hi_d + 1;
-    if (hi > b_safe) hi = b_safe;
-    int lo = lo_d <= 2.0 ? 0 : (int)lo_d - 1;
-    if (lo > hi) lo = hi;
-    // invariant of the bisection: lo fits (or is 0) and nothing above hi fits
-    if (lo > 0 && pages<kActs>((u32)lo) > budget) {
-      hi = lo - 1;
-      lo = 0;
-    } else if (hi < b_safe && pages<kActs>((u32)hi + 1) <= budget) {
-      lo = hi + 1;
-      hi = b_safe;
-    }
+    const double room = (double)(budget - fixed_a);  // below 2^41: exact
+    const double up = room * rate_up * (1.0 + 0x1p-40);
+    int hi = up >= (double)b_safe ? b_safe : (int)up;  // nothing above hi fits
+    const double dn = (room - dyn_events) * rate_dn * (1.0 - 0x1p-40);
+    int lo = dn < 1.0 ? 0 : (dn >= (double)hi ? hi : (int)dn);  // lo fits (or is 0)
     while (lo < hi) {
       const int mid = lo + (hi - lo + 1) / 2;
       if (pages<kActs>((u32)mid) <= budget) lo = mid;
@@ -247,9 +246,13 @@ max_batch_kernel(const llmem_config* __restrict__ shape, i64 n, const i64* __res
     int st = check_fields(f, false, true);
     PageSearch q;
     if (st == LLMEM_CFG_OK) {
-      const Plan p = make_plan(f, f.method);
+      StickyMath m;
+      const Plan p = make_plan(m, f, f.method);
       st = p.status;
-      if (st == LLMEM_CFG_OK) q.init(p, make_static_sums(p, f.pos_len > 0), bmax);
+      if (st == LLMEM_CFG_OK) {
+        const StaticSums s = make_static_sums(m, p, f.pos_len > 0);
+        q.init(p, s, bmax, m.too_large(0));
+      }
     }
     int* out = bs_out + i * n_cap;
     if (st != LLMEM_CFG_OK) {
@@ -286,9 +289,13 @@ select_kernel(const llmem_config* __restrict__ shape, i64 n, const i64* __restri
       gpu_n = f.gpu_n;
       tp_n = f.tp_n;
       if (st == LLMEM_CFG_OK) {
-        const Plan p = make_plan(f, k);
+        StickyMath m;
+        const Plan p = make_plan(m, f, k);
         usable = p.status == LLMEM_CFG_OK;  // a method that cannot be configured scores 0
-        if (usable) q.init(p, make_static_sums(p, f.pos_len > 0), bmax);
+        if (usable) {
+          const StaticSums s = make_static_sums(m, p, f.pos_len > 0);
+          q.init(p, s, bmax, m.too_large(0));
+        }
       }
     }
     for (int m = 0; m < n_cap; ++m) {

@@ -340,6 +340,42 @@ def test_search_edge_capacities_and_ranges(llmem):
             assert np.array_equal(got[k].cpu().numpy(), want[k]), k
 
 
+def test_search_bracket_at_its_boundaries(llmem):
+    """The search cuts a floating-point bracket to integers and probes only inside it: capacities
+    exactly at, one byte below and one page below the peak of a batch, for batches from 1 to
+    2^20, on shapes whose bytes per sample range from a few bytes (wide brackets) to gigabytes
+    (brackets of one candidate), every method, TP degrees that do not divide the output."""
+    rng = np.random.default_rng(606)
+    shapes = fuzz_configs(40, 7)
+    small = shapes[:12].copy()
+    small["seq"], small["hidden"], small["heads"], small["vocab"] = 1, 3, 1, 5      # few bytes per sample
+    small["layers"] = rng.integers(1, 40, size=12)
+    odd = shapes[12:24].copy()
+    odd["method"], odd["gpu_n"], odd["tp_n"] = 2, rng.choice([3, 5, 7, 11, 13], size=12), 0
+    odd["seq"] = rng.choice([1, 3, 7, 129], size=12)
+    shapes = np.concatenate([shapes, small, odd])
+    bmax = 1 << 20
+    checked = 0
+    for i in range(len(shapes)):
+        one = shapes[i:i + 1]
+        caps = []
+        for b in (1, 2, 3, 17, 255, 4097, 65535, (1 << 20) - 1, 1 << 20):
+            at = one.copy(); at["batch"] = b
+            est = oracle.estimate(at, level=2)
+            if est["status"][0] == 0:
+                pk = int(est["peak"][0])
+                caps += [pk, pk - 1, pk - (1 << 21), pk + (1 << 21) - 1]
+        if not caps:
+            continue
+        caps = np.array(sorted(set(caps)), dtype=np.int64)
+        want_bs, want_st = oracle.max_batch(one, caps, bmax, level=2)
+        got_bs, got_st = llmem.max_batch(one, caps, bmax)
+        assert np.array_equal(got_st.cpu().numpy(), want_st)
+        assert np.array_equal(got_bs.cpu().numpy(), want_bs), (i, caps, got_bs.cpu().numpy(), want_bs)
+        checked += caps.size
+    assert checked > 1000
+
+
 def test_segmented_selection_random_groups(llmem):
     rng = np.random.default_rng(10933)
     sizes = rng.integers(0, 40, size=300)
@@ -426,6 +462,44 @@ def test_fuzz_all_entry_points(llmem):
         got_sel = llmem.select_method(cfgs, caps, 1 << 20, allzero=allzero)
         for k in ("method", "batch", "bs_list", "status"):
             assert np.array_equal(got_sel[k].cpu().numpy(), want_sel[k]), k
+
+
+def heads_and_hidden_pairs(n, seed):
+    """hidden in 1 .. 2^20 against divisors, near-divisors, itself, heads above hidden and heads
+    up to 2^31 - 1; records with tiny event lists."""
+    rng = np.random.default_rng(seed)
+    c = np.repeat(grids.g1_small()[:1], n)
+    lo = np.arange(n) % 2 == 0
+    h = np.where(lo, rng.integers(1, 1 << 10, size=n), rng.integers(1, 1 << 5, size=n))
+    k = np.where(lo, rng.integers(1, 1 << 10, size=n), rng.integers(1, 1 << 15, size=n))
+    hidden = h * k                                              # <= 2^20
+    kind = (np.arange(n) // 2) % 8
+    heads = np.select(
+        [kind == 0, kind == 1, kind == 2, kind == 3, kind == 4, kind == 5, kind == 6],
+        [h, k, h + 1, np.maximum(1, k - 1), hidden, hidden + rng.integers(1, 1 << 20, size=n),
+         rng.integers(1 << 21, 1 << 31, size=n)],
+        default=rng.integers(1, (1 << 20) + 1, size=n))
+    hidden[:4] = [1, 1 << 20, (1 << 20) - 1, 720720]
+    heads[:4] = [1, 1 << 20, (1 << 20) - 1, (1 << 31) - 1]
+    c["hidden"], c["heads"] = hidden, heads
+    c["layers"], c["ffn"], c["vocab"], c["seq"], c["batch"] = 1, 64, 64, 8, 1
+    c["chunk_elems"] = 1 << 40
+    return c
+
+
+def test_heads_must_divide_hidden_every_pair_class(llmem):
+    """The field check decides hidden % heads == 0 without an integer division."""
+    c = heads_and_hidden_pairs(1 << 18, 77)
+    want = oracle.estimate(c, threads=16)
+    ok = (c["hidden"] % c["heads"]) == 0
+    assert np.array_equal(want["status"] == 0, ok) and 0.3 < ok.mean() < 0.7
+    got = llmem.estimate_batch(c)
+    assert np.array_equal(got["status"].cpu().numpy(), want["status"])
+    assert np.array_equal(got["peak"].cpu().numpy(), want["peak"])
+    caps = np.array([1 << 34], dtype=np.int64)
+    got_bs, got_st = llmem.max_batch(c[:4096], caps, 64)
+    want_bs, want_st = oracle.max_batch(c[:4096], caps, 64, level=2, threads=8)
+    assert np.array_equal(got_st.cpu().numpy(), want_st) and np.array_equal(got_bs.cpu().numpy(), want_bs)
 
 
 def test_bounded_wait_gives_up_and_reports(llmem):
