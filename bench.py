@@ -707,8 +707,64 @@ def leg_slabs(llmem, torch, steps, warmup, shapes=None):
             "gpu_launches": steps * (4 + slabs * 7), "clocks": clocks, "fused_equals_materialised": agree}
 
 
+# lists of the shape grid by length: [lo, hi) events per list
+LENGTH_CLASSES = ((1, 150), (150, 400), (400, 1500), (1500, 6000), (6000, 25000), (25000, 1 << 31))
+
+
+def leg_classes(llmem, torch, steps, warmup, only=None):
+    """Throughput by list length: about 4e8 events of shape-grid configurations from one length
+    class each (the class's configurations repeated), through llmem_expand_scan,
+    llmem_expand_events and llmem_scan_peak with CUDA events; `only` picks one class by number
+    (for a profiler capture).  The lists (3.2 GB) are larger than L2."""
+    import numpy as np
+    cfgs = grids.g2_shape_grid(0, 512)
+    counts = torch.diff(llmem.event_counts(llmem.to_device(cfgs))[0]).cpu().numpy()
+    target = 400_000_000
+    rows = []
+    for k, (lo, hi) in enumerate(LENGTH_CLASSES):
+        if only is not None and k != only:
+            continue
+        idx = np.nonzero((counts >= lo) & (counts < hi))[0]
+        idx = idx[:int(np.searchsorted(np.cumsum(counts[idx]), target)) + 1]
+        sub = np.tile(cfgs[idx], max(1, int(target // max(1, counts[idx].sum()))))
+        dev = llmem.to_device(sub)
+        offsets, _ = llmem.event_counts(dev)
+        total = int(offsets[-1].item())
+        delta = torch.empty(total, dtype=torch.int64, device="cuda")
+        scratch = torch.empty(max(llmem.scratch_bytes(op, len(sub), total)
+                                  for op in (llmem.OP_SCAN_PEAK, llmem.OP_EXPAND_SCAN, llmem.OP_EXPAND)),
+                              dtype=torch.uint8, device="cuda")
+        fused = llmem.estimate_batch(dev)
+        row = {"events_per_list": [lo, hi], "lists": len(sub), "events": total, "mean_events": total / len(sub)}
+        calls = (("expand_scan", lambda: llmem.expand_scan(dev, offsets, total, fuse_round=True, out=delta, scratch=scratch)),
+                 ("expand", lambda: llmem.expand_events(dev, offsets, total, fuse_round=True, out=delta, scratch=scratch)),
+                 ("scan", lambda: llmem.scan_peak(delta, offsets, dev, scratch=scratch)))
+        for name, call in calls:  # the scan reads the list the expansion before it wrote
+            best = None
+            for it in range(max(warmup, 1) + max(steps, 1)):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                res = call()
+                e1.record()
+                torch.cuda.synchronize()
+                if it >= max(warmup, 1):
+                    best = e0.elapsed_time(e1) if best is None else min(best, e0.elapsed_time(e1))
+            if name != "expand" and not (torch.equal(res["peak"], fused["peak"]) and torch.equal(res["index"], fused["index"])):
+                raise SystemExit(f"{name} disagrees with the fused estimate on class {lo}..{hi}")
+            row[name] = {"ms": best, "gbs": 8.0 * total / best / 1e6}
+        rows.append(row)
+        del dev, delta, scratch
+    peak_gbs, peak_src = measured_peaks()
+    return {"metric": METRIC, "unit": UNIT, "steps": steps, "dtype": "int64",
+            "value": sum(r["events"] for r in rows) / sum(r["expand_scan"]["ms"] * 1e-3 for r in rows),
+            "ms_per_step": sum(r["expand_scan"]["ms"] for r in rows),
+            "config": {"workload": "shape-grid lists by length class, 4e8 events each: expand_scan / expand / scan",
+                       "l2": "each list (3.2 GB) is larger than the 126 MB L2"},
+            "classes": rows, "peak": peak_gbs, "peak_source": peak_src}
+
+
 def run_secondary_workload(args):
-    """--workload g3 | g4 | g2 alone: one JSON line for that leg."""
+    """--workload g3 | g4 | g2 | classes alone: one JSON line for that leg."""
     import torch
     import paper_2404_10933_b200 as llmem
     llmem.lib()
@@ -718,6 +774,8 @@ def run_secondary_workload(args):
         leg = leg_estimate(llmem, torch, args.steps, args.warmup, min(args.configs, grids.G3_CONFIGS) if reduced else None)
     elif args.workload == "g4":
         leg = leg_search(llmem, torch, args.steps, args.warmup, min(args.configs, grids.G4_SHAPES) if reduced else None)
+    elif args.workload == "classes":
+        leg = leg_classes(llmem, torch, min(args.steps, 10), min(args.warmup, 3), args.length_class)
     else:
         leg = leg_slabs(llmem, torch, args.steps, args.warmup, args.configs if reduced else None)
     line = {"n_gpus": 1, "warmup": max(args.warmup, 3), "higher_is_better": True, "scaling": "weak",
@@ -743,9 +801,12 @@ def main():
                     help="skip the short legs on the other grids that a one-GPU run appends under 'secondary'")
     ap.add_argument("--two-pass", action="store_true",
                     help="time llmem_expand_events + llmem_scan_peak as separate kernels instead of llmem_expand_scan")
-    ap.add_argument("--workload", choices=("g5", "g3", "g4", "g2"), default="g5",
+    ap.add_argument("--workload", choices=("g5", "g3", "g4", "g2", "classes"), default="g5",
                     help="g5 (default): the full hot path on the stress grid; g3 / g4: the in-register kernels; "
-                         "g2: the shape grid through the materialised path in slabs")
+                         "g2: the shape grid through the materialised path in slabs; classes: the three list "
+                         "entry points on shape-grid lists of one length class at a time")
+    ap.add_argument("--length-class", type=int, default=None, choices=range(len(LENGTH_CLASSES)),
+                    help="with --workload classes: only this class (0 = the shortest lists)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
