@@ -54,9 +54,9 @@ FALLBACK_HBM_GBS = 6650.0
 # HBM-bound kernels, from an ncu capture of a 4096-configuration run (summary kept under
 # profiles/; traffic grows in proportion to the number of events).  Set an entry
 # to None when its kernel changes after the capture.
-NCU_TRAFFIC_BYTES_PER_EVENT = {"expand": 7.8207, "scan": 8.0125, "expand_scan": 7.8231}
+NCU_TRAFFIC_BYTES_PER_EVENT = {"expand": 7.8251, "scan": 8.0143, "expand_scan": 7.8269}
 # the same for the owner kernel that takes lists of short and medium segments (64-shape capture)
-NCU_TRAFFIC_BYTES_PER_EVENT_OWNERS = 8.03
+NCU_TRAFFIC_BYTES_PER_EVENT_OWNERS = 8.0225
 
 
 def measured_peaks():
@@ -557,7 +557,7 @@ def run_ours(args):
 # grids (profiles/register_kernels_g3_g4_ncu.md); None once a kernel changes after the capture.
 # Counting lane instructions keeps divergence from passing for throughput: a warp instruction
 # issued for 20 of 32 lanes counts as 20/32.
-NCU_LANE_INSTR_PER_UNIT = {"estimate_kernel": 21.78, "max_batch_kernel": 8.40, "select_kernel": 40.21}
+NCU_LANE_INSTR_PER_UNIT = {"estimate_kernel": 21.78, "max_batch_kernel": 5.34, "select_kernel": 27.58}
 
 
 def _gpu_id(torch):
@@ -665,7 +665,7 @@ def leg_search(llmem, torch, steps, warmup, shapes=None):
     n_units = units["max_batch_kernel"] + 4 * units["select_kernel"]
     return {"metric": "searches per second (max batch + Algorithm 1)", "value": n_units / (ms * 1e-3),
             "unit": "searches/s", "steps": steps, "ms_per_step": ms, "dtype": "int64",
-            "config": {"workload": "G4 max-batch search + Algorithm 1 selection, bracketed bisection on batch 1..4096 in registers",
+            "config": {"workload": "G4 max-batch search + Algorithm 1 selection, batch 1..4096, a certain bracket from the near-linear page count and probes inside it, in registers",
                        "shapes": shapes, "searches": units["max_batch_kernel"], "selections": units["select_kernel"],
                        "l2": "256 MB write between timed steps flushes L2"},
             "roofline": _alu_roofline(torch, llmem, units, ms, clocks),
