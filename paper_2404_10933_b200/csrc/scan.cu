@@ -273,7 +273,7 @@ scan_kernel(const i64* __restrict__ delta_aligned /* 16-byte aligned base */, in
 // whatever the length, a warp's bulk copies 3.3 TB/s on 866-event and 6 TB/s on 3 k-event
 // segments: the lanes only pay below a few hundred events).
 #ifndef LLMEM_SCAN_LANE_MAX
-#define LLMEM_SCAN_LANE_MAX 384
+#define LLMEM_SCAN_LANE_MAX 768
 #endif
 #ifndef LLMEM_SCAN_PART
 #define LLMEM_SCAN_PART 4096
@@ -328,7 +328,7 @@ scan_parts_kernel(const i64* __restrict__ offsets, i64 n, unsigned long long* __
 
 // Segmented prefix-sum + max for lists of short and medium segments.  The warps of a persistent
 // grid claim items from one counter: first the parts of the longer segments, then groups of
-// 32 consecutive segments.  In a group every segment of up to 384 events is scanned by one
+// 32 consecutive segments.  In a group every segment of up to 768 events is scanned by one
 // lane: each step the warp brings the next 128-byte line of all 32 segments into shared memory
 // (eight lanes per line: 16-byte loads from 32 different lines in one instruction reach a
 // fifth of the bandwidth) and every lane folds its own line in order: no segment boundaries
@@ -474,22 +474,33 @@ scan_owned_kernel(const i64* __restrict__ delta_aligned, int shift, const i64* _
         __syncwarp();
         i64 sum = 0, mx = 0, idx = -1;
         bool has = false;
-        for (i64 step = 0; __any_sync(0xffffffffu, mine && base + step * kScanRowEvents < ge); ++step) {
+        // The lines of the next step are requested before the rows of this one are folded, so
+        // that the loads are in flight during the fold.
+        longlong2 x[8];
+        auto fetch = [&](i64 step) {
 #pragma unroll
           for (int pass = 0; pass < 8; ++pass) {
             const int r = (lane >> 3) + 4 * pass, vec = lane & 7;
             const i64 lo_r = first[r], hi_r = last[r];
             const i64 at = (lo_r & ~(i64)1) + step * kScanRowEvents + 2 * vec;
-            longlong2 x = make_longlong2(0, 0);
+            x[pass] = make_longlong2(0, 0);
             if (at >= lo_r && at + 1 < hi_r) {
-              x = __ldg(reinterpret_cast<const longlong2*>(delta_aligned + at));
+              x[pass] = __ldg(reinterpret_cast<const longlong2*>(delta_aligned + at));
             } else {
-              if (at >= lo_r && at < hi_r) x.x = __ldg(delta_aligned + at);
-              if (at + 1 >= lo_r && at + 1 < hi_r) x.y = __ldg(delta_aligned + at + 1);
+              if (at >= lo_r && at < hi_r) x[pass].x = __ldg(delta_aligned + at);
+              if (at + 1 >= lo_r && at + 1 < hi_r) x[pass].y = __ldg(delta_aligned + at + 1);
             }
-            *reinterpret_cast<longlong2*>(&rows[r][2 * vec]) = x;
           }
+        };
+        bool more = true;  // the group has a segment with events: step 0 exists
+        fetch(0);
+        for (i64 step = 0; more; ++step) {
+#pragma unroll
+          for (int pass = 0; pass < 8; ++pass)
+            *reinterpret_cast<longlong2*>(&rows[(lane >> 3) + 4 * pass][2 * (lane & 7)]) = x[pass];
           __syncwarp();
+          more = __any_sync(0xffffffffu, mine && base + (step + 1) * kScanRowEvents < ge);
+          if (more) fetch(step + 1);
           const i64 row0 = base + step * kScanRowEvents;
           if (mine && row0 < ge) {
             const int q_lo = row0 < gs ? (int)(gs - row0) : 0;

@@ -162,8 +162,8 @@ def test_scan_of_arbitrary_lists_and_alignments(llmem):
     rng = np.random.default_rng(2404)
     lens = [0, 1, 2, 4607, 4608, 4609, 0, 0, 9216, 13824, 5, 70000, 3, 0, 4608 * 3 - 1, 1, 18, 17, 19,
             250000, 0]
-    # around the limits of the scan by owners: a lane's segment (384), a warp's part (4096), its chunks (832)
-    lens += [383, 384, 385, 831, 832, 833, 4095, 4096, 4097, 8191, 8192, 8193, 2 * 4096 + 833]
+    # around the limits of the scan by owners: a lane's segment (768), a warp's part (4096), its chunks (832)
+    lens += [383, 384, 385, 767, 768, 769, 831, 832, 833, 4095, 4096, 4097, 8191, 8192, 8193, 2 * 4096 + 833]
     lens += rng.integers(0, 300, size=400).tolist()
     lens += [0]
     offsets = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
