@@ -115,7 +115,8 @@ enum { LLMEM_OP_ESTIMATE = 0, LLMEM_OP_EVENT_COUNTS = 1, LLMEM_OP_EXPAND = 2, LL
 /* Bytes of scratch the operation needs for n configurations and total_events
  * events (0 where it needs none; such calls accept scratch = NULL).  For
  * LLMEM_OP_EXPAND the scratch is optional (see llmem_expand_events).  For
- * LLMEM_OP_EXPAND and LLMEM_OP_EXPAND_SCAN the size depends on total_events too. */
+ * LLMEM_OP_EXPAND, LLMEM_OP_SCAN_PEAK and LLMEM_OP_EXPAND_SCAN the size depends on
+ * total_events too (lists of short segments keep per-segment records there). */
 size_t llmem_scratch_bytes(int op, int64_t n, int64_t total_events);
 
 /* Sections 4.2 and 5, fused: peak of each configuration without materialising
@@ -222,7 +223,8 @@ llmem_status llmem_round_events(int64_t* DEV delta, int64_t total_events, void* 
  * offset + 0 and index -1; with cfg, an inadmissible cfg[i] yields -1 / -1.
  *   delta          DEV [total_events]; any signed values whose prefix sums stay within int64
  *   cfg            DEV [n], nullable (then the offset is 0)
- *   scratch        required; holds a device status word readable with llmem_scratch_status */
+ *   scratch        required, llmem_scratch_bytes(LLMEM_OP_SCAN_PEAK, n, total_events) bytes;
+ *                  holds a device status word readable with llmem_scratch_status */
 llmem_status llmem_scan_peak(const int64_t* DEV delta, const int64_t* DEV offsets, int64_t n,
                              int64_t total_events, const llmem_config* DEV cfg,
                              int64_t* DEV peak_out, int64_t* DEV peak_index_out, void* DEV scratch,
