@@ -376,6 +376,55 @@ def test_search_bracket_at_its_boundaries(llmem):
     assert checked > 1000
 
 
+def configs_near_the_byte_limit(n_per=256):
+    """Records whose peak crosses 2^62 bytes as the batch grows: through the logits, through
+    the score-sized operator outputs, through m_base; every method."""
+    base = grids.g1_small()[:1].copy()
+    k = np.arange(n_per)
+    a = np.repeat(base, n_per)
+    a["lm_bytes"], a["seq"], a["vocab"], a["hidden"], a["heads"], a["ffn"], a["layers"] = 4, 1 << 26, 1 << 26, 64, 1, 256, 2
+    a["batch"], a["method"] = k + 1, k % 4
+    a["gpu_n"] = np.where(a["method"] == 3, 4, 1 + k % 7)
+    a["tp_n"] = np.where(a["method"] == 3, 2, 0)
+    b = np.repeat(base, n_per)
+    b["act_mode"], b["seq"], b["hidden"], b["heads"], b["ffn"], b["vocab"] = 1, 1 << 20, 1 << 10, 1 << 10, 1 << 12, 1000
+    b["layers"], b["batch"], b["method"] = 1 + k % 64, 1 + k // 4, k % 4
+    b["gpu_n"] = np.where(b["method"] == 3, 4, 1 + k % 5)
+    b["tp_n"] = np.where(b["method"] == 3, 2, 0)
+    c = np.repeat(base, n_per)
+    c["base_bytes"], c["lm_bytes"], c["seq"], c["vocab"] = 1 << 60, 4, 1 << 25, 1 << 26
+    c["batch"], c["iters"] = k + 1, 1 + k % 2
+    out = np.concatenate([a, b, c])
+    out["chunk_elems"] = 1 << 30
+    return out
+
+
+def test_results_around_the_byte_limit(llmem):
+    """Status 3 exactly from 2^62 bytes on, the exact peak below: the fused estimate remembers
+    an overflow instead of clamping, the counts clamp, the searches exclude such batches."""
+    cfgs = configs_near_the_byte_limit()
+    want = oracle.estimate(cfgs, level=2, threads=8)
+    for part in range(3):
+        st = want["status"][part * 256:(part + 1) * 256]
+        assert (st == 0).sum() > 60 and (st == 3).sum() > 60
+    assert want["peak"].max() > 0.98 * 2.0 ** 62
+    got = llmem.estimate_batch(cfgs)
+    assert np.array_equal(got["status"].cpu().numpy(), want["status"])
+    assert np.array_equal(got["peak"].cpu().numpy(), want["peak"])
+    offsets, status = llmem.event_counts(cfgs)
+    assert np.array_equal(status.cpu().numpy(), want["status"])
+    caps = np.array([(1 << 62) - 1, 1 << 61, 1 << 60, 3 << 59], dtype=np.int64)
+    for bmax in (300, 1 << 26):
+        want_bs, want_st = oracle.max_batch(cfgs, caps, bmax, level=2, threads=8)
+        got_bs, got_st = llmem.max_batch(cfgs, caps, bmax)
+        assert np.array_equal(got_st.cpu().numpy(), want_st)
+        assert np.array_equal(got_bs.cpu().numpy(), want_bs), bmax
+    want_sel = oracle.select_method(cfgs, caps, 1 << 26, level=2, threads=8)
+    got_sel = llmem.select_method(cfgs, caps, 1 << 26)
+    for key in ("method", "batch", "bs_list", "status"):
+        assert np.array_equal(got_sel[key].cpu().numpy(), want_sel[key]), key
+
+
 def test_segmented_selection_random_groups(llmem):
     rng = np.random.default_rng(10933)
     sizes = rng.integers(0, 40, size=300)
