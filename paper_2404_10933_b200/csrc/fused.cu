@@ -55,7 +55,6 @@ constexpr i64 kFusedSegmentCost = LLMEM_FUSED_SEGMENT_COST;
 #define LLMEM_OWNED_PART 8192
 #endif
 constexpr i64 kOwnedLaneMax = LLMEM_OWNED_LANE_MAX, kOwnedPart = LLMEM_OWNED_PART;
-static_assert(LLMEM_OWNED_PART % 16 == 0 && LLMEM_OWNED_PART < (1 << 20), "parts: whole lines, part numbers fit 20 bits");
 
 // Scratch of the owner kernel behind the header, block starts and partials of the chunk
 // kernels: one descriptor per configuration, then the list of parts (segment << 20 | part
@@ -296,16 +295,15 @@ struct OwnedWarpSmem {
 };
 
 // One-pass expansion + scan in which every event has one owner that needs nobody else.  The
-// warps of a persistent grid claim items of work from one counter: first the parts of the
-// longer segments (the list of parts the table kernel made), then groups of 32 consecutive
-// segments.
+// warps of a persistent grid claim items of work from one counter: first the groups of 32
+// consecutive segments, then the parts of the longer segments (the list of parts the table
+// kernel made).
 //
 // A part (up to 8192 events of one segment) is written by a whole warp, run by run, with
 // coalesced 16-byte stores straight to device memory; the fold of a run is taken once, in
 // closed form, by all lanes alike, so a part costs a few thousand instructions however many
 // events it has.  The prefix sum at which a part begins is the sum of the runs before it,
-// taken from their closed forms.  The warp that reports a segment's last outstanding part
-// joins the parts' results.
+// taken from their closed forms.  The finishing pass joins the results of a segment's parts.
 //
 // In a group, the segments short enough for a lane (most of a list of small decoders) are
 // written by one lane each: the lane walks its segment's runs with a cursor of its own, stages
@@ -336,13 +334,18 @@ expand_scan_owned_kernel(i64 n, const i64* __restrict__ offsets, i64 total, i64*
   }
   i64 n_parts = (i64)*part_count;
   if (n_parts > part_capacity) n_parts = part_capacity;
-  const i64 n_items = n_parts + n_groups;
-  const i64 resident = (i64)gridDim.x * kWarps;
-  for (i64 work = (i64)blockIdx.x * kWarps + warp; work < n_items;) {
-    // the parts come first: they are the long items, so what ends the kernel is short
-    const bool is_part = work < n_parts;
-    const i64 item = work;
-    if (is_part) {
+  // One queue, handed out item by item from the counter in the scratch header: the groups of
+  // short segments first (a group of 32 lists written by lanes takes longer than a part
+  // written by a warp, so the items that end the kernel are the short ones), then the parts.
+  const i64 n_items = n_groups + n_parts;
+  for (;;) {
+    unsigned long long ticket = 0;
+    if (lane == 0) ticket = atomicAdd(work_counter, 1ull);
+    const i64 work = (i64)__shfl_sync(0xffffffffu, ticket, 0);
+    if (work >= n_items) break;
+    const bool on_groups = work < n_groups;
+    const i64 item = on_groups ? work : work - n_groups;
+    if (!on_groups) {
       // ---- the whole warp for one part of a longer segment ----
       const i64 entry = part_list[item];
       const i64 s = entry >> 20, k = entry & 0xfffff;
@@ -401,7 +404,7 @@ expand_scan_owned_kernel(i64 n, const i64* __restrict__ offsets, i64 total, i64*
       }
     } else {
       // ---- one lane for each short segment of a group ----
-      const i64 seg = (item - n_parts) * 32 + lane;
+      const i64 seg = item * 32 + lane;
       const bool have = seg < n;
       const i64 gs = have ? __ldg(offsets + seg) : 0, ge = have ? __ldg(offsets + seg + 1) : 0;
       const bool in_list = have && in_bounds(gs >= 0 && ge <= total, g, kSiteStore);
@@ -466,10 +469,6 @@ expand_scan_owned_kernel(i64 n, const i64* __restrict__ offsets, i64 total, i64*
           write_raw(seg, Agg{f.sum, f.mx, gs + f.ix, f.has ? 1 : 0}, gs, peak_out, index_out);
       }
     }
-    unsigned long long ticket = 0;
-    if (lane == 0 && n_items > resident) ticket = atomicAdd(work_counter, 1ull);
-    ticket = __shfl_sync(0xffffffffu, ticket, 0);
-    work = n_items > resident ? resident + (i64)ticket : n_items;
   }
 }
 

@@ -327,8 +327,8 @@ scan_parts_kernel(const i64* __restrict__ offsets, i64 n, unsigned long long* __
 }
 
 // Segmented prefix-sum + max for lists of short and medium segments.  The warps of a persistent
-// grid claim items from one counter: first the parts of the longer segments, then groups of
-// 32 consecutive segments.  In a group every segment of up to 768 events is scanned by one
+// grid claim items from one counter: first the groups of 32 consecutive segments, then the
+// parts of the longer segments.  In a group every segment of up to 768 events is scanned by one
 // lane: each step the warp brings the next 128-byte line of all 32 segments into shared memory
 // (eight lanes per line: 16-byte loads from 32 different lines in one instruction reach a
 // fifth of the bandwidth) and every lane folds its own line in order: no segment boundaries
@@ -373,10 +373,16 @@ scan_owned_kernel(const i64* __restrict__ delta_aligned, int shift, const i64* _
   bool aborted = false;
   i64 n_parts = (i64)*part_count;
   if (n_parts > part_capacity) n_parts = part_capacity;
-  const i64 n_items = n_parts + n_groups;
-  const i64 resident = (i64)gridDim.x * kScanOwnedWarps;
-  for (i64 item = (i64)blockIdx.x * kScanOwnedWarps + warp; item < n_items && !aborted;) {
-    if (item < n_parts) {
+  // groups first, item by item from the counter (see expand_scan_owned_kernel)
+  const i64 n_items = n_groups + n_parts;
+  while (!aborted) {
+    unsigned long long ticket = 0;
+    if (lane == 0) ticket = atomicAdd(work_counter, 1ull);
+    const i64 work = (i64)__shfl_sync(0xffffffffu, ticket, 0);
+    if (work >= n_items) break;
+    const bool on_groups = work < n_groups;
+    const i64 item = on_groups ? work : work - n_groups;
+    if (!on_groups) {
       // ---- the whole warp for one part of a longer segment ----
       const i64 entry = part_list[item];
       const i64 s = entry >> 20, k = entry & 0xfffff;
@@ -455,7 +461,7 @@ scan_owned_kernel(const i64* __restrict__ delta_aligned, int shift, const i64* _
       }
     } else {
       // ---- one lane for each short segment of a group ----
-      const i64 seg = (item - n_parts) * 32 + lane;
+      const i64 seg = item * 32 + lane;
       const bool have = seg < n;
       const i64 gs = have ? __ldg(offsets + seg) + shift : 0, ge = have ? __ldg(offsets + seg + 1) + shift : 0;
       const bool mine = have && ge > gs && ge - gs <= kScanLaneMax &&
@@ -517,10 +523,6 @@ scan_owned_kernel(const i64* __restrict__ delta_aligned, int shift, const i64* _
           write_raw(seg, Agg{sum, mx, idx, has ? 1 : 0}, gs, peak_out, index_out);
       }
     }
-    unsigned long long ticket = 0;
-    if (lane == 0 && n_items > resident) ticket = atomicAdd(work_counter, 1ull);
-    ticket = __shfl_sync(0xffffffffu, ticket, 0);
-    item = n_items > resident ? resident + (i64)ticket : n_items;
   }
   if (lane == 0 && (aborted || *abort_flag)) atomicExch(status_word, (u32)LLMEM_ERR_TIMEOUT);
 }
