@@ -56,7 +56,7 @@ FALLBACK_HBM_GBS = 6650.0
 # to None when its kernel changes after the capture.
 NCU_TRAFFIC_BYTES_PER_EVENT = {"expand": 7.8251, "scan": 8.0143, "expand_scan": 7.8269}
 # the same for the owner kernel that takes lists of short and medium segments (64-shape capture)
-NCU_TRAFFIC_BYTES_PER_EVENT_OWNERS = 8.0225
+NCU_TRAFFIC_BYTES_PER_EVENT_OWNERS = 8.0487
 
 
 def measured_peaks():
