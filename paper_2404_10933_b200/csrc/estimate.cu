@@ -63,7 +63,8 @@ struct PageSearch {
   double dyn_events;         // N: at least the number of batch-dependent events of one iteration
 
   // `too_large`: one of the batch-independent sums (or the per-sample score size) reached 2^62
-  __device__ __forceinline__ void init(const Plan& p, const StaticSums& s, int bmax, bool too_large) {
+  // `big_limit` = floor((2^62 - 1) / bmax), the same for every configuration of a call
+  __device__ __forceinline__ void init(const Plan& p, const StaticSums& s, int bmax, bool too_large, u64 big_limit) {
     out1 = p.out1; logit1 = p.logit1; shift1 = p.shift1;
     offset = p.offset;
     n_out = (u32)(p.e_n + p.L * p.n_x);
@@ -92,8 +93,8 @@ struct PageSearch {
     u64 big = out1 > logit1 ? out1 : logit1;  // >= 2
     if (attn1 > big) big = attn1;
     if (ffn1 > big) big = ffn1;
-    const u64 lim = (kSat - 1) / big;                // largest b with b * big < 2^62
-    b_safe = lim < (u64)bmax ? (int)lim : bmax;
+    // the largest b <= bmax with b * big < 2^62: bmax itself unless a per-sample size is huge
+    b_safe = big <= big_limit ? bmax : (int)((kSat - 1) / big);
     // bytes one more sample adds to the batch-dependent events, without the backward buffers;
     // those add  out - floor(out / tp)  per layer, which lies between b (out1 - q1 - 1) and
     // b (out1 - q1)
@@ -240,7 +241,7 @@ estimate_kernel(const llmem_config* __restrict__ cfg, i64 n, i64* __restrict__ p
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256, LLMEM_SEARCH_MIN_CTAS)
 max_batch_kernel(const llmem_config* __restrict__ shape, i64 n, const i64* __restrict__ caps,
-                 int n_cap, int bmax, int* __restrict__ bs_out, uint8_t* __restrict__ status_out) {
+                 int n_cap, int bmax, u64 big_limit, int* __restrict__ bs_out, uint8_t* __restrict__ status_out) {
   for (i64 i = (i64)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (i64)gridDim.x * blockDim.x) {
     Cfg f = load_cfg(shape + i);
     int st = check_fields(f, false, true);
@@ -251,7 +252,7 @@ max_batch_kernel(const llmem_config* __restrict__ shape, i64 n, const i64* __res
       st = p.status;
       if (st == LLMEM_CFG_OK) {
         const StaticSums s = make_static_sums(m, p, f.pos_len > 0);
-        q.init(p, s, bmax, m.too_large(0));
+        q.init(p, s, bmax, m.too_large(0), big_limit);
       }
     }
     int* out = bs_out + i * n_cap;
@@ -270,7 +271,7 @@ max_batch_kernel(const llmem_config* __restrict__ shape, i64 n, const i64* __res
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256, LLMEM_SEARCH_MIN_CTAS)
 select_kernel(const llmem_config* __restrict__ shape, i64 n, const i64* __restrict__ caps, int n_cap,
-              int bmax, u32 flags, int* __restrict__ method_out, int* __restrict__ batch_out,
+              int bmax, u64 big_limit, u32 flags, int* __restrict__ method_out, int* __restrict__ batch_out,
               int* __restrict__ bs_list_out, uint8_t* __restrict__ status_out) {
   const i64 quads_per_grid = ((i64)gridDim.x * blockDim.x) >> 2;
   const u32 k = threadIdx.x & 3;  // method of this lane
@@ -294,7 +295,7 @@ select_kernel(const llmem_config* __restrict__ shape, i64 n, const i64* __restri
         usable = p.status == LLMEM_CFG_OK;  // a method that cannot be configured scores 0
         if (usable) {
           const StaticSums s = make_static_sums(m, p, f.pos_len > 0);
-          q.init(p, s, bmax, m.too_large(0));
+          q.init(p, s, bmax, m.too_large(0), big_limit);
         }
       }
     }
@@ -477,7 +478,7 @@ extern "C" llmem_status llmem_max_batch(const llmem_config* shape, int64_t n,
   if (st != LLMEM_OK || n == 0 || n_cap == 0) return st;
   if (!bs_out || !aligned_to(bs_out, 4)) { set_error("llmem_max_batch: bs_out is required"); return LLMEM_ERR_ARG; }
   max_batch_kernel<<<grid_for(n, 256, LLMEM_SEARCH_GRID_CTAS), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-      shape, n, reinterpret_cast<const i64*>(capacity_bytes), n_cap, bmax, bs_out, status_out);
+      shape, n, reinterpret_cast<const i64*>(capacity_bytes), n_cap, bmax, (kSat - 1) / (u64)bmax, bs_out, status_out);
   return check_launch("llmem_max_batch");
 }
 
@@ -494,7 +495,7 @@ extern "C" llmem_status llmem_select_method(const llmem_config* shape, int64_t n
   if (st != LLMEM_OK || n == 0 || n_cap == 0) return st;
   if (!method_out || !batch_out) { set_error("llmem_select_method: method_out and batch_out are required"); return LLMEM_ERR_ARG; }
   select_kernel<<<grid_for(4 * n, 256, LLMEM_SEARCH_GRID_CTAS), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-      shape, n, reinterpret_cast<const i64*>(capacity_bytes), n_cap, bmax, flags, method_out,
+      shape, n, reinterpret_cast<const i64*>(capacity_bytes), n_cap, bmax, (kSat - 1) / (u64)bmax, flags, method_out,
       batch_out, bs_list_out, status_out);
   return check_launch("llmem_select_method");
 }
