@@ -557,7 +557,7 @@ def run_ours(args):
 # grids (profiles/register_kernels_g3_g4_ncu.md); None once a kernel changes after the capture.
 # Counting lane instructions keeps divergence from passing for throughput: a warp instruction
 # issued for 20 of 32 lanes counts as 20/32.
-NCU_LANE_INSTR_PER_UNIT = {"estimate_kernel": 21.78, "max_batch_kernel": 5.34, "select_kernel": 27.58}
+NCU_LANE_INSTR_PER_UNIT = {"estimate_kernel": 21.78, "max_batch_kernel": 5.14, "select_kernel": 26.76}
 
 
 def _gpu_id(torch):
