@@ -55,6 +55,7 @@ constexpr i64 kFusedSegmentCost = LLMEM_FUSED_SEGMENT_COST;
 #define LLMEM_OWNED_PART 8192
 #endif
 constexpr i64 kOwnedLaneMax = LLMEM_OWNED_LANE_MAX, kOwnedPart = LLMEM_OWNED_PART;
+static_assert(LLMEM_OWNED_PART % 16 == 0 && LLMEM_OWNED_PART < (1 << 20), "parts: whole lines, part numbers fit 20 bits");
 
 // Scratch of the owner kernel behind the header, block starts and partials of the chunk
 // kernels: one descriptor per configuration, then the list of parts (segment << 20 | part
