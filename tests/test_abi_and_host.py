@@ -182,3 +182,31 @@ def test_checked_build_exports_the_same_entry_points():
         getattr(D, name)
     D.llmem_checked_build.restype = ctypes.c_int
     assert D.llmem_checked_build() == 1
+
+
+def test_bench_constants_are_the_figures_of_the_committed_profiles():
+    """bench.py scales profiler counters (DRAM bytes per event, lane instructions per unit) that
+    were captured on reduced cases; the figures it uses must be the ones the summaries under
+    profiles/ state, so that neither can be updated without the other."""
+    import importlib.util
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    spec = importlib.util.spec_from_file_location("bench_module", os.path.join(root, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+
+    def rows(name):
+        with open(os.path.join(root, "profiles", name)) as f:
+            return [[c.strip() for c in line.strip().strip("|").split("|")] for line in f if line.startswith("|")]
+
+    g5 = [r for r in rows("expand_scan_g5_4096cfg_ncu.md") if r[0].startswith("traffic per event")]
+    assert len(g5) == 1
+    one_pass, expand, scan = (float(c.split()[0]) for c in g5[0][1:4])
+    assert bench.NCU_TRAFFIC_BYTES_PER_EVENT == {"expand": expand, "scan": scan, "expand_scan": one_pass}
+    owners = [r for r in rows("expand_scan_owned_g2_64shapes_ncu.md") if r[0].startswith("traffic per event")]
+    assert len(owners) == 1 and float(owners[0][2].split()[0]) == bench.NCU_TRAFFIC_BYTES_PER_EVENT_OWNERS
+    table = rows("register_kernels_g3_g4_ncu.md")
+    head = next(r for r in table if r[0] == "kernel" and "lane instr / 32 / unit" in r)
+    col = head.index("lane instr / 32 / unit")
+    for kernel, value in bench.NCU_LANE_INSTR_PER_UNIT.items():
+        row = next(r for r in table if r[0].startswith(kernel) and len(r) == len(head))
+        assert float(row[col]) == value, kernel
