@@ -537,6 +537,8 @@ def run_ours(args):
             "g4": leg_search(llmem, torch, max(5, min(args.steps, 20)), args.warmup),
             "g2": leg_slabs(llmem, torch, max(3, min(args.steps, 5)), args.warmup),
         }
+        torch.cuda.empty_cache()
+        line["secondary"]["classes"] = leg_classes(llmem, torch, 3, 1)
     if args.cpu_baseline:
         line["cpu_baseline"] = cpu_baseline()
     print(json.dumps(line))
