@@ -417,12 +417,16 @@ def run_ours(args):
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     wall0 = time.time()
     start.record()
+    marks = []  # an event after every step: where the time of the region went, step by step
     for _ in range(args.steps):
         out = hp.step()
+        marks.append(torch.cuda.Event(enable_timing=True))
+        marks[-1].record()
     stop.record()
     barrier()
     wall1 = time.time()
     ms = max_over_ranks(start.elapsed_time(stop))
+    per_step = [a.elapsed_time(b) for a, b in zip([start] + marks[:-1], marks)]
     clocks = sampler.stop(wall0, wall1) if rank == 0 else None
     total_events_all = sum_over_ranks(float(hp.total))
     configs_all = sum_over_ranks(float(hp.n))
@@ -505,6 +509,9 @@ def run_ours(args):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "step_ms": {"median": statistics.median(per_step), "min": min(per_step), "max": max(per_step),
+                    "note": "device time of the single timed steps on this rank (ms_per_step is the whole region / steps: "
+                            "one pause of the box inside a short region shows as a large max here)"},
         "scaling": args.scaling, "vs_baseline": None, "dtype": "int64", "data": "synthetic",
         "configs_per_sec": configs_all * args.steps / (ms * 1e-3),
         "config": {"workload": "G5 stress grid: deep/wide decoders, materialised int64 event lists",
